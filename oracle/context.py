@@ -1,0 +1,86 @@
+"""Upstream and downstream context of the filter, as numpy float64: TEST INFRASTRUCTURE ONLY.
+
+The vision-encoding stage (Local Spatial Merging, Key Retaining; Sec. 3.3) produces the
+tokens and the key set O that the prefill filter consumes; the decoding stage (output-aware
+cache policy, Sec. 3.5) consumes the filter's kept sets.  The paper leaves their constants and
+several details unstated, so every function here is a stated reading and is checked only
+against internal invariants: PARITY UNPINNED for ``local_spatial_merge``, ``key_set`` and
+``cache_policy``.  ``kv_cache_mb`` is pinned to the token/MB pairs of Tables 3 and 6.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Sequence, Tuple
+
+import numpy as np
+
+
+def kv_cache_mb(tokens: int, layers: int = 32, hidden: int = 4096, bytes_per_el: int = 2) -> float:
+    """KV-cache size of `tokens` tokens in MB (10^6 bytes): K and V, every layer (Eq. 2)."""
+    return tokens * 2 * layers * hidden * bytes_per_el / 1e6
+
+
+def local_spatial_merge(tokens: np.ndarray, grid: int, window: int = 2, tau: float = 0.8
+                        ) -> Tuple[np.ndarray, np.ndarray]:
+    """Local Spatial Merging (Sec. 3.3, Eq. 5).
+
+    tokens [grid*grid, C] in raster order.  The grid is cut into non-overlapping
+    window x window squares; for each square S_w = mean over unordered pairs of the cosine
+    similarity of its tokens; if S_w > tau the square is replaced by the plain average of
+    its tokens, placed at the square's first raster slot.  Returns (merged tokens
+    [M', C], source slot of each output token [M']).
+    """
+    x = np.asarray(tokens, np.float64)
+    assert x.shape[0] == grid * grid and grid % window == 0
+    keep_rows: List[np.ndarray] = []
+    slots: List[int] = []
+    unit = x / np.maximum(np.linalg.norm(x, axis=1, keepdims=True), 1e-300)
+    for wy in range(0, grid, window):
+        for wx in range(0, grid, window):
+            ids = [(wy + dy) * grid + (wx + dx) for dy in range(window) for dx in range(window)]
+            sims = [float(unit[a] @ unit[b]) for ai, a in enumerate(ids) for b in ids[ai + 1:]]
+            if np.mean(sims) > tau:
+                keep_rows.append(x[ids].mean(axis=0))
+                slots.append(ids[0])
+            else:
+                for t in ids:
+                    keep_rows.append(x[t])
+                    slots.append(t)
+    order = np.argsort(np.asarray(slots), kind="stable")
+    return np.stack(keep_rows)[order], np.asarray(slots, np.int64)[order]
+
+
+def key_set(q_cls: np.ndarray, k: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Key Retaining (Sec. 3.3, Eq. 6-7).
+
+    q_cls [H, D], k [H, M, D]: a_cls = head mean of softmax(q_cls k^T / sqrt(D)) over the M
+    patch tokens; O = {j : a_cls[j] > mu} with the adaptive threshold read as Tukey's upper
+    fence mu = Q3 + 1.5 (Q3 - Q1) of a_cls.  Returns (O ascending, a_cls).
+    """
+    q = np.asarray(q_cls, np.float64)
+    kk = np.asarray(k, np.float64)
+    z = np.einsum("hd,hmd->hm", q, kk) / np.sqrt(q.shape[-1])
+    z -= z.max(axis=1, keepdims=True)
+    p = np.exp(z)
+    p /= p.sum(axis=1, keepdims=True)
+    a = p.mean(axis=0)
+    q1, q3 = np.quantile(a, [0.25, 0.75])
+    mu = q3 + 1.5 * (q3 - q1)
+    return np.nonzero(a > mu)[0].astype(np.int32), a
+
+
+def cache_policy(kept_per_layer: Sequence[np.ndarray], n_layers: int, first_sparse_layer: int = 2
+                 ) -> Dict[int, np.ndarray]:
+    """Output-aware cache policy (Sec. 3.5).
+
+    kept_per_layer[l] = vision tokens (original indices, ascending) that layer l's KV cache
+    holds after prefill.  S_few is the set still retained at the last layer.  During decoding
+    the layers with 0-based index >= first_sparse_layer ("following the second layer") keep, of
+    the vision tokens, only S_few; earlier layers keep what prefill left them.
+    """
+    assert len(kept_per_layer) == n_layers
+    s_few = np.asarray(kept_per_layer[-1])
+    out = {}
+    for l in range(n_layers):
+        cur = np.asarray(kept_per_layer[l])
+        out[l] = cur if l < first_sparse_layer else np.intersect1d(cur, s_few)
+    return out
