@@ -1,0 +1,167 @@
+/*
+ * mustdrop.h - C ABI of the B200 (sm_100a) vision-token filter.
+ *
+ * The library implements the prefill-stage, text-guided dual-attention filtering of vision
+ * tokens of MustDrop (arXiv 2411.10803, Sec. 3.4 "Dual-Attention Filtering Guided by
+ * Language") as a batched operation at one pruning layer:
+ *
+ *     mustdrop_score    text-query x key attention -> per-vision-token importance (Eq. 1, 8, 10)
+ *     mustdrop_select   dual criteria + key set -> retained indices             (Eq. 9, 10, Sec. 3.3)
+ *     mustdrop_compact  gather the retained hidden states and per-head K/V     (Table 3: tokens in the KV cache)
+ *
+ * Conventions shared by all calls
+ *   - Pointers marked (host) are plain host memory.  Every other data pointer is DEVICE
+ *     memory, 16-byte aligned, allocated and freed by the caller.  The library allocates only
+ *     the host-side plan; it never allocates device memory and never synchronises, except
+ *     mustdrop_device_status.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls enqueue work and return; issuing score, select, compact in that order on one
+ *     stream is the whole protocol.
+ *   - Host-detectable problems return a non-OK status and launch nothing.  Conditions only
+ *     the device can see (a key index outside [0, n_vis)) are recorded in a status word in
+ *     the workspace and never trap.
+ *   - Sequence layout (Sec. 3.1, "Prefilling"): the n_vis vision tokens occupy positions
+ *     [vis_start, vis_start+n_vis), the n_txt text tokens [txt_start, txt_start+n_txt),
+ *     vis_start+n_vis <= txt_start, txt_start+n_txt <= seq_len.
+ *   - A plan is immutable; concurrent calls are safe when they use distinct workspaces.
+ */
+#ifndef MUSTDROP_H_
+#define MUSTDROP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mustdrop_plan mustdrop_plan_t; /* opaque, host memory, owned by the library */
+
+typedef enum {
+  MUSTDROP_OK = 0,
+  MUSTDROP_ERR_INVALID_ARG = 1,   /* null or misaligned pointer, non-positive size, bad span, bad threshold */
+  MUSTDROP_ERR_UNSUPPORTED = 2,   /* head_dim != 128, n_txt > 128, n_vis > 4096, odd strides */
+  MUSTDROP_ERR_BUDGET = 3,        /* budget < key_max or budget > n_vis (BUDGET mode) */
+  MUSTDROP_ERR_WORKSPACE = 4,     /* null workspace */
+  MUSTDROP_ERR_CUDA = 5,          /* a CUDA runtime call failed; see mustdrop_last_cuda_error */
+  MUSTDROP_ERR_TIMEOUT = 6,       /* device status only: a bounded wait inside a kernel ran out */
+  MUSTDROP_ERR_BAD_KEY_INDEX = 7  /* device status only: an index outside [0, n_vis) was ignored */
+} mustdrop_status_t;
+
+typedef enum { MUSTDROP_MODE_BUDGET = 0, MUSTDROP_MODE_THRESHOLD = 1 } mustdrop_mode_t;
+
+/* Which criteria decide (Table 4, rows b, c, d). */
+typedef enum {
+  MUSTDROP_CRIT_DUAL = 0,
+  MUSTDROP_CRIT_GLOBAL_ONLY = 1,
+  MUSTDROP_CRIT_INDIVIDUAL_ONLY = 2
+} mustdrop_criteria_t;
+
+typedef struct {
+  int32_t batch;      /* B, independent requests */
+  int32_t n_heads;    /* H */
+  int32_t head_dim;   /* D, must be 128 */
+  int32_t hidden;     /* elements per hidden-state row (any positive multiple of 8) */
+  int32_t seq_len;    /* L */
+  int32_t vis_start;  /* first vision position */
+  int32_t n_vis;      /* M, 1..4096 */
+  int32_t txt_start;  /* first text position */
+  int32_t n_txt;      /* N, 1..128 */
+  int32_t causal;     /* 1: text query i attends keys 0..txt_start+i (the model's prefill mask); 0: all L keys */
+  float   scale;      /* logit scale; 0 => 1/sqrt(head_dim) (Eq. 1) */
+  int32_t mode;       /* mustdrop_mode_t */
+  int32_t criteria;   /* mustdrop_criteria_t */
+  int32_t budget;     /* Kp: tokens kept per request in BUDGET mode, key set included */
+  float   gamma;      /* Eq. 9 threshold; 0 => 1/n_vis */
+  float   alpha;      /* Eq. 10 threshold; 0 => 2/seq_len */
+  int32_t key_max;    /* capacity of key_idx per request; 0 = no key set */
+  int32_t reserved;   /* must be 0 */
+  /* Strides in ELEMENTS (bf16); 0 => contiguous.  Head rows themselves are contiguous
+   * (head_dim elements).  Every stride must be a multiple of 8 (16 bytes). */
+  int64_t k_stride_b, k_stride_h, k_stride_l;       /* K      [B,H,L,D] */
+  int64_t v_stride_b, v_stride_h, v_stride_l;       /* V      [B,H,L,D] */
+  int64_t hid_stride_b, hid_stride_l;               /* hidden [B,L,hidden] */
+} mustdrop_config_t;
+
+/*
+ * Validate a configuration and build a plan (host only; nothing is launched).
+ * config, plan_out and workspace_bytes are (host).  `*workspace_bytes` receives the size of
+ * the device workspace the other calls need (>= 256, a multiple of 256).  The workspace must
+ * be zeroed once before first use (its first bytes are the device status word); after that
+ * the calls keep it consistent.  The plan records the CUDA device current at this call.
+ */
+mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t *config, mustdrop_plan_t **plan_out,
+                                       size_t *workspace_bytes);
+
+mustdrop_status_t mustdrop_plan_destroy(mustdrop_plan_t *plan);
+
+/*
+ * Importance of every vision token (Sec. 3.4).
+ *   z^h[i][l] = scale * <q_text[b][h][i], k[b][h][l]>                      (Eq. 1)
+ *   p^h[i][.] = softmax over the keys visible to text query i (all vision keys, and the text
+ *               keys up to and including its own when causal)             (Eq. 1, "attention map")
+ *   a[i][j]   = mean over heads of p^h[i][vis_start + j]
+ *   g_out[b][j] = sum_i a[i][j]                                            (Eq. 8)
+ *   i_out[b][j] = max_i a[i][j]                                            (Eq. 10)
+ * q_text bf16 [B,H,N,D] contiguous; k bf16 [B,H,L,D] (plan strides); g_out, i_out fp32 [B,M].
+ * fp32 accumulation from bf16 inputs.
+ */
+mustdrop_status_t mustdrop_score(const mustdrop_plan_t *plan, const void *q_text, const void *k,
+                                 float *g_out, float *i_out, void *workspace, void *cuda_stream);
+
+/*
+ * Dual criteria, key set and selection (Eq. 9, Eq. 10; the key set O of Sec. 3.3 is always kept).
+ *   T = sum_j g[j];  gt = gamma * T;  D = { j : g[j] <= gt }               (Eq. 9)
+ *   THRESHOLD mode: token j is dropped iff j in D and i[j] < alpha and j not in O.
+ *   BUDGET mode: s[j] = max(g[j]/gt, i[j]/alpha) (fp32, one rounding per operation); O is kept,
+ *   then the tokens with the largest s, lower index first among equals, until exactly
+ *   `budget` tokens are kept.  GLOBAL_ONLY / INDIVIDUAL_ONLY use one of the two terms.
+ * g, i fp32 [B,M]; key_idx int32 [B,key_max] vision-relative (entries outside [0,M) and repeats
+ * are ignored, the former also recorded as MUSTDROP_ERR_BAD_KEY_INDEX), key_cnt int32 [B];
+ * both may be NULL when key_max == 0.
+ * kept_idx int32 [B,cap], cap = budget (BUDGET) or n_vis (THRESHOLD): strictly ascending,
+ * vision-relative; entries at and beyond kept_cnt[b] are left untouched.  kept_cnt int32 [B].
+ * s_out: NULL or fp32 [B,M], receives s.
+ */
+mustdrop_status_t mustdrop_select(const mustdrop_plan_t *plan, const float *g, const float *i,
+                                  const int32_t *key_idx, const int32_t *key_cnt,
+                                  int32_t *kept_idx, int32_t *kept_cnt, float *s_out,
+                                  void *workspace, void *cuda_stream);
+
+/*
+ * Gather-compaction of the retained tokens (pruned tokens leave the sequence and the KV
+ * cache; Table 3).  For r < kept_cnt[b]:
+ *   hidden_out[b][r][:]  = hidden[b][vis_start + kept_idx[b][r]][:]
+ *   k_out[b][h][r][:]    = k[b][h][vis_start + kept_idx[b][r]][:]          (v likewise)
+ * hidden bf16 [B,L,hidden], k, v bf16 [B,H,L,D] (plan strides); outputs contiguous
+ * hidden_out [B,cap,hidden], k_out, v_out [B,H,cap,D].  Rows r >= kept_cnt[b] are left
+ * untouched.  Any of the three (source, destination) pairs may be NULL together to skip it.
+ * An index outside [0, n_vis) is skipped and, when workspace is not NULL, recorded in its
+ * device status word.
+ */
+mustdrop_status_t mustdrop_compact(const mustdrop_plan_t *plan, const int32_t *kept_idx,
+                                   const int32_t *kept_cnt, const void *hidden, const void *k,
+                                   const void *v, void *hidden_out, void *k_out, void *v_out,
+                                   void *workspace, void *cuda_stream);
+
+/*
+ * Read the device status word of a workspace (synchronises `cuda_stream`).
+ * code_out (host) receives MUSTDROP_OK or the first device-detected condition, detail_out
+ * (host, may be NULL) an operation-specific detail (BAD_KEY_INDEX: request * 65536 + slot).
+ */
+mustdrop_status_t mustdrop_device_status(const mustdrop_plan_t *plan, const void *workspace,
+                                         void *cuda_stream, int32_t *code_out, int32_t *detail_out);
+
+/* Static description of a status code. */
+const char *mustdrop_status_string(mustdrop_status_t status);
+
+/* cudaError_t value of the last failed CUDA call made by this library on this thread (0 if none). */
+int32_t mustdrop_last_cuda_error(void);
+
+/* Name of the score kernel variant the plan selected (static string; for logs and benchmarks). */
+const char *mustdrop_plan_score_variant(const mustdrop_plan_t *plan);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MUSTDROP_H_ */

@@ -1,0 +1,205 @@
+// C-ABI layer: configuration checks, plan object, argument checks, kernel dispatch.
+// The operations themselves are defined by Sec. 3.4 (Eq. 8-10) of the paper; see mustdrop.h.
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "mustdrop_internal.h"
+
+namespace {
+
+thread_local int32_t g_last_cuda_error = 0;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline mustdrop_status_t cuda_fail(cudaError_t e) {
+  g_last_cuda_error = static_cast<int32_t>(e);
+  return MUSTDROP_ERR_CUDA;
+}
+
+inline bool valid_plan(const mustdrop_plan_t* p) { return p != nullptr && p->magic == mustdrop::kPlanMagic; }
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" {
+
+mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan_t** plan_out,
+                                       size_t* workspace_bytes) {
+  using namespace mustdrop;
+  if (c == nullptr || plan_out == nullptr || workspace_bytes == nullptr) return MUSTDROP_ERR_INVALID_ARG;
+  *plan_out = nullptr;
+  *workspace_bytes = 0;
+  if (c->batch <= 0 || c->n_heads <= 0 || c->head_dim <= 0 || c->hidden <= 0 || c->seq_len <= 0 ||
+      c->n_vis <= 0 || c->n_txt <= 0 || c->vis_start < 0 || c->txt_start < 0 || c->key_max < 0 ||
+      c->reserved != 0)
+    return MUSTDROP_ERR_INVALID_ARG;
+  // the vision span precedes the text span and both lie inside the sequence
+  if (static_cast<int64_t>(c->vis_start) + c->n_vis > c->txt_start ||
+      static_cast<int64_t>(c->txt_start) + c->n_txt > c->seq_len)
+    return MUSTDROP_ERR_INVALID_ARG;
+  if (c->causal != 0 && c->causal != 1) return MUSTDROP_ERR_INVALID_ARG;
+  if (c->mode != MUSTDROP_MODE_BUDGET && c->mode != MUSTDROP_MODE_THRESHOLD) return MUSTDROP_ERR_INVALID_ARG;
+  if (c->criteria < MUSTDROP_CRIT_DUAL || c->criteria > MUSTDROP_CRIT_INDIVIDUAL_ONLY)
+    return MUSTDROP_ERR_INVALID_ARG;
+  if (!(c->scale >= 0.0f) || !std::isfinite(c->scale)) return MUSTDROP_ERR_INVALID_ARG;
+  if (!(c->gamma >= 0.0f) || !std::isfinite(c->gamma) || !(c->alpha >= 0.0f) || !std::isfinite(c->alpha))
+    return MUSTDROP_ERR_INVALID_ARG;
+  const int64_t strides[] = {c->k_stride_b, c->k_stride_h, c->k_stride_l, c->v_stride_b,
+                             c->v_stride_h, c->v_stride_l, c->hid_stride_b, c->hid_stride_l};
+  for (int64_t s : strides)
+    if (s < 0) return MUSTDROP_ERR_INVALID_ARG;
+  if (c->batch > 65535) return MUSTDROP_ERR_UNSUPPORTED;
+  if (c->head_dim != kHeadDim || c->n_txt > kMaxTxt || c->n_vis > kMaxVis || (c->hidden % 8) != 0)
+    return MUSTDROP_ERR_UNSUPPORTED;
+  for (int64_t s : strides)
+    if (s % 8 != 0) return MUSTDROP_ERR_UNSUPPORTED;
+  if (c->mode == MUSTDROP_MODE_BUDGET) {
+    if (c->budget <= 0 || c->budget > c->n_vis || c->budget < c->key_max) return MUSTDROP_ERR_BUDGET;
+  }
+
+  mustdrop_plan_t* p = new (std::nothrow) mustdrop_plan_t();
+  if (p == nullptr) return MUSTDROP_ERR_INVALID_ARG;
+  p->magic = kPlanMagic;
+  p->config = *c;
+  Resolved& r = p->r;
+  r.B = c->batch; r.H = c->n_heads; r.D = c->head_dim; r.hidden = c->hidden; r.L = c->seq_len;
+  r.vis_start = c->vis_start; r.M = c->n_vis; r.txt_start = c->txt_start; r.N = c->n_txt;
+  r.causal = c->causal; r.mode = c->mode; r.criteria = c->criteria; r.budget = c->budget;
+  r.key_max = c->key_max;
+  r.cap = (c->mode == MUSTDROP_MODE_BUDGET) ? c->budget : c->n_vis;
+  r.scale = (c->scale == 0.0f) ? 1.0f / sqrtf(static_cast<float>(c->head_dim)) : c->scale;
+  r.scale_log2e = r.scale * 1.4426950408889634f;
+  r.gamma = (c->gamma == 0.0f) ? 1.0f / static_cast<float>(c->n_vis) : c->gamma;
+  r.alpha = (c->alpha == 0.0f) ? 2.0f / static_cast<float>(c->seq_len) : c->alpha;
+  r.k_sl = c->k_stride_l ? c->k_stride_l : c->head_dim;
+  r.k_sh = c->k_stride_h ? c->k_stride_h : static_cast<int64_t>(c->seq_len) * r.k_sl;
+  r.k_sb = c->k_stride_b ? c->k_stride_b : static_cast<int64_t>(c->n_heads) * r.k_sh;
+  r.v_sl = c->v_stride_l ? c->v_stride_l : c->head_dim;
+  r.v_sh = c->v_stride_h ? c->v_stride_h : static_cast<int64_t>(c->seq_len) * r.v_sl;
+  r.v_sb = c->v_stride_b ? c->v_stride_b : static_cast<int64_t>(c->n_heads) * r.v_sh;
+  r.hid_sl = c->hid_stride_l ? c->hid_stride_l : c->hidden;
+  r.hid_sb = c->hid_stride_b ? c->hid_stride_b : static_cast<int64_t>(c->seq_len) * r.hid_sl;
+  if (r.k_sl < c->head_dim || r.v_sl < c->head_dim || r.hid_sl < c->hidden) {
+    delete p;
+    return MUSTDROP_ERR_INVALID_ARG;
+  }
+
+  // The device is only consulted for the SM count; a box without a GPU still gets a plan.
+  p->device = -1;
+  p->sm_count = 148;
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
+      p->device = dev;
+      p->sm_count = sms;
+    }
+  }
+  (void)cudaGetLastError();
+
+  p->score_variant = kScoreTwoPassMma;
+  size_t off = kWsStatusBytes;
+  p->ws_rowstats_off = off;
+  off += round_up(sizeof(float) * 2 * static_cast<size_t>(r.B) * r.H * r.N, 256);
+  p->ws_bytes = off;
+  *workspace_bytes = p->ws_bytes;
+  *plan_out = p;
+  return MUSTDROP_OK;
+}
+
+mustdrop_status_t mustdrop_plan_destroy(mustdrop_plan_t* plan) {
+  if (plan == nullptr) return MUSTDROP_OK;
+  if (!valid_plan(plan)) return MUSTDROP_ERR_INVALID_ARG;
+  plan->magic = 0;
+  delete plan;
+  return MUSTDROP_OK;
+}
+
+mustdrop_status_t mustdrop_score(const mustdrop_plan_t* plan, const void* q_text, const void* k, float* g_out,
+                                 float* i_out, void* workspace, void* cuda_stream) {
+  if (!valid_plan(plan) || q_text == nullptr || k == nullptr || g_out == nullptr || i_out == nullptr)
+    return MUSTDROP_ERR_INVALID_ARG;
+  if (workspace == nullptr) return MUSTDROP_ERR_WORKSPACE;
+  if (!aligned16(q_text) || !aligned16(k) || !aligned16(g_out) || !aligned16(i_out) || !aligned16(workspace))
+    return MUSTDROP_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  void* rowstats = static_cast<unsigned char*>(workspace) + plan->ws_rowstats_off;
+  cudaError_t e = mustdrop::launch_score_two_pass(*plan, q_text, k, g_out, i_out, rowstats, stream);
+  return e == cudaSuccess ? MUSTDROP_OK : cuda_fail(e);
+}
+
+mustdrop_status_t mustdrop_select(const mustdrop_plan_t* plan, const float* g, const float* i,
+                                  const int32_t* key_idx, const int32_t* key_cnt, int32_t* kept_idx,
+                                  int32_t* kept_cnt, float* s_out, void* workspace, void* cuda_stream) {
+  if (!valid_plan(plan) || g == nullptr || i == nullptr || kept_idx == nullptr || kept_cnt == nullptr)
+    return MUSTDROP_ERR_INVALID_ARG;
+  if (plan->r.key_max > 0 && (key_idx == nullptr || key_cnt == nullptr)) return MUSTDROP_ERR_INVALID_ARG;
+  if (workspace == nullptr) return MUSTDROP_ERR_WORKSPACE;
+  if (!aligned16(g) || !aligned16(i) || !aligned16(kept_idx) || !aligned16(kept_cnt) || !aligned16(workspace) ||
+      (key_idx && !aligned16(key_idx)) || (key_cnt && !aligned16(key_cnt)) || (s_out && !aligned16(s_out)))
+    return MUSTDROP_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e =
+      mustdrop::launch_select(*plan, g, i, key_idx, key_cnt, kept_idx, kept_cnt, s_out, workspace, stream);
+  return e == cudaSuccess ? MUSTDROP_OK : cuda_fail(e);
+}
+
+mustdrop_status_t mustdrop_compact(const mustdrop_plan_t* plan, const int32_t* kept_idx, const int32_t* kept_cnt,
+                                   const void* hidden, const void* k, const void* v, void* hidden_out,
+                                   void* k_out, void* v_out, void* workspace, void* cuda_stream) {
+  if (!valid_plan(plan) || kept_idx == nullptr || kept_cnt == nullptr) return MUSTDROP_ERR_INVALID_ARG;
+  if ((hidden == nullptr) != (hidden_out == nullptr) || (k == nullptr) != (k_out == nullptr) ||
+      (v == nullptr) != (v_out == nullptr))
+    return MUSTDROP_ERR_INVALID_ARG;
+  const void* ptrs[] = {kept_idx, kept_cnt, hidden, k, v, hidden_out, k_out, v_out, workspace};
+  for (const void* q : ptrs)
+    if (q != nullptr && !aligned16(q)) return MUSTDROP_ERR_INVALID_ARG;
+  if (hidden == nullptr && k == nullptr && v == nullptr) return MUSTDROP_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = mustdrop::launch_compact(*plan, kept_idx, kept_cnt, hidden, k, v, hidden_out, k_out, v_out,
+                                           workspace, stream);
+  return e == cudaSuccess ? MUSTDROP_OK : cuda_fail(e);
+}
+
+mustdrop_status_t mustdrop_device_status(const mustdrop_plan_t* plan, const void* workspace, void* cuda_stream,
+                                         int32_t* code_out, int32_t* detail_out) {
+  if (!valid_plan(plan) || code_out == nullptr) return MUSTDROP_ERR_INVALID_ARG;
+  if (workspace == nullptr) return MUSTDROP_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int32_t host[2] = {0, 0};
+  cudaError_t e = cudaMemcpyAsync(host, workspace, sizeof(host), cudaMemcpyDeviceToHost, stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  *code_out = host[0];
+  if (detail_out != nullptr) *detail_out = host[1];
+  return MUSTDROP_OK;
+}
+
+const char* mustdrop_status_string(mustdrop_status_t s) {
+  switch (s) {
+    case MUSTDROP_OK: return "ok";
+    case MUSTDROP_ERR_INVALID_ARG: return "invalid argument";
+    case MUSTDROP_ERR_UNSUPPORTED: return "unsupported configuration";
+    case MUSTDROP_ERR_BUDGET: return "budget smaller than the key set capacity or larger than n_vis";
+    case MUSTDROP_ERR_WORKSPACE: return "workspace missing";
+    case MUSTDROP_ERR_CUDA: return "CUDA runtime error";
+    case MUSTDROP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case MUSTDROP_ERR_BAD_KEY_INDEX: return "index outside [0, n_vis) ignored";
+  }
+  return "unknown status";
+}
+
+int32_t mustdrop_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* mustdrop_plan_score_variant(const mustdrop_plan_t* plan) {
+  if (!valid_plan(plan)) return "invalid plan";
+  switch (plan->score_variant) {
+    case mustdrop::kScoreTwoPassMma: return "two_pass_mma";
+  }
+  return "unknown";
+}
+
+}  // extern "C"

@@ -1,0 +1,65 @@
+// Internal declarations shared by the C-ABI layer and the kernel translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "mustdrop.h"
+
+namespace mustdrop {
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxTxt = 128;
+constexpr int kMaxVis = 4096;
+
+// Workspace layout (bytes).  The first 256 bytes hold the device status word:
+//   int32 code, int32 detail.  Everything after is kernel scratch.
+constexpr size_t kWsStatusBytes = 256;
+
+enum ScoreVariant : int32_t {
+  kScoreTwoPassMma = 0,   // row statistics pass + accumulate pass, warp-level mma
+};
+
+struct Resolved {
+  int32_t B, H, D, hidden, L, vis_start, M, txt_start, N;
+  int32_t causal, mode, criteria, budget, key_max, cap;
+  float scale, scale_log2e, gamma, alpha;
+  int64_t k_sb, k_sh, k_sl, v_sb, v_sh, v_sl, hid_sb, hid_sl;
+};
+
+}  // namespace mustdrop
+
+struct mustdrop_plan {
+  uint32_t magic;
+  mustdrop_config_t config;
+  mustdrop::Resolved r;
+  int32_t device;
+  int32_t sm_count;
+  int32_t score_variant;
+  size_t ws_bytes;
+  size_t ws_rowstats_off;   // float2 [B,H,N]: (row max in log2 units, 1 / row sum)
+};
+
+namespace mustdrop {
+
+constexpr uint32_t kPlanMagic = 0x4d445250u;  // "MDRP"
+
+// Each launcher enqueues on `stream` and returns the launch error (cudaGetLastError).
+cudaError_t launch_score_two_pass(const mustdrop_plan& p, const void* q_text, const void* k,
+                                  float* g_out, float* i_out, void* rowstats, cudaStream_t stream);
+cudaError_t launch_select(const mustdrop_plan& p, const float* g, const float* i, const int32_t* key_idx,
+                          const int32_t* key_cnt, int32_t* kept_idx, int32_t* kept_cnt, float* s_out,
+                          void* workspace, cudaStream_t stream);
+cudaError_t launch_compact(const mustdrop_plan& p, const int32_t* kept_idx, const int32_t* kept_cnt,
+                           const void* hidden, const void* k, const void* v, void* hidden_out, void* k_out,
+                           void* v_out, void* workspace, cudaStream_t stream);
+
+// Device-side helper: record the first device-detected condition (never traps).
+__device__ __forceinline__ void record_status(void* workspace, int32_t code, int32_t detail) {
+  if (workspace == nullptr) return;
+  int32_t* w = reinterpret_cast<int32_t*>(workspace);
+  if (atomicCAS(w, 0, code) == 0) w[1] = detail;
+}
+
+}  // namespace mustdrop
