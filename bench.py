@@ -1,0 +1,364 @@
+#!/usr/bin/env python
+"""Benchmark of the vision-token filter: one step = score + select + compact over one batch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  `value` is vision tokens filtered per second with the inputs
+resident in device memory; `e2e` is the same metric with pinned host inputs copied in and
+results copied out every step; `roofline` describes the dominant kernel (the score call)
+against the measured HBM copy bandwidth; `cpu_baseline` is the CPU oracle on a bounded sample.
+With N > 1 (torchrun) every rank filters its own batch: requests are independent, so there
+is no collective on the data path (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2411_10803_b200 import synth  # noqa: E402
+
+METRIC = "vision tokens filtered/sec (score+select+compact)"
+UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "c2_llava7b_b64"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def bytes_model(w):
+    """Algorithmic bytes per step (whole batch)."""
+    B, H, D, L, N, M, Kp = w.batch, w.n_heads, w.head_dim, w.seq_len, w.n_txt, w.n_vis, w.budget
+    k_bytes = B * H * L * D * 2
+    q_bytes = B * H * N * D * 2
+    out_bytes = B * Kp * (w.hidden + 2 * H * D) * 2
+    score_bytes = k_bytes + q_bytes + 2 * B * M * 4
+    return {
+        "score": score_bytes,                      # K + Q_text read, G and I written
+        "headline": k_bytes + q_bytes + out_bytes,  # K + Q_text + compacted outputs
+        "full": k_bytes + q_bytes + 2 * out_bytes,  # + the gather's source rows
+        "h2d": k_bytes * 2 + q_bytes + B * L * w.hidden * 2 + B * (max(w.key_cnt, 1) + 1) * 4,
+        "d2h": out_bytes + B * (Kp + 1) * 4,
+    }
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML (read-only) while the GPU is busy."""
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            handle = None
+            try:
+                import torch
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                handle = None
+            if handle is None:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+                idx = device_index
+                if vis:
+                    try:
+                        idx = int(vis.split(",")[device_index])
+                    except Exception:
+                        idx = device_index
+                handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.h = handle
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def finish(self):
+        self._stop.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_step(w, requests):
+    """The CPU oracle over the given requests: score + select + compact.  Returns seconds."""
+    import oracle
+    d = synth.make_batch(w, requests=requests)
+    t0 = time.perf_counter()
+    G, I = oracle.score(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start)
+    kidx = d["key_idx"] if w.key_cnt else None
+    kcnt = d["key_cnt"] if w.key_cnt else None
+    kept, cnt, _, _ = oracle.select(G, I, w.seq_len, kidx, kcnt, budget=w.budget)
+    oracle.compact(kept, cnt, w.vis_start, d["hidden"], d["k"], d["v"])
+    return time.perf_counter() - t0
+
+
+def run_reference(args, w):
+    """The oracle as it stands, timed on the host cores: each step is a bounded sample of requests."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    probe = oracle_step(w, range(0, 1))                                 # also warms the page cache
+    budget_s = 150.0
+    per_step = int(max(1, min(8, w.batch, budget_s / max(probe * (args.steps + args.warmup), 1e-9))))
+    for i in range(args.warmup):
+        oracle_step(w, range(0, per_step))
+    total = 0.0
+    for i in range(args.steps):
+        lo = (i * per_step) % max(w.batch - per_step + 1, 1)
+        total += oracle_step(w, range(lo, lo + per_step))
+    ms = 1e3 * total / max(args.steps, 1)
+    value = per_step * w.n_vis / (ms / 1e3)
+    sample = "%d of the %d requests per step (score+select+compact)" % (per_step, w.batch)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "n_vis": w.n_vis, "n_txt": w.n_txt, "n_heads": w.n_heads,
+                   "hidden": w.hidden, "budget": w.budget, "key_set": w.key_cnt, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2411_10803_b200 import binding as md
+    from paper_2411_10803_b200 import build as md_build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the filter has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if rank == 0:
+        md_build.build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    dev = torch.device("cuda", local_rank)
+
+    # every rank filters its own batch of w.batch requests (distinct request numbers per rank)
+    reqs = range(rank * w.batch, (rank + 1) * w.batch)
+    host = synth.make_batch(w, requests=reqs)
+
+    def pinned(a):
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else
+                                np.ascontiguousarray(a)).pin_memory()
+
+    h_q, h_k, h_v, h_hid = (pinned(host[n]) for n in ("q_text", "k", "v", "hidden"))
+    h_ki, h_kc = pinned(host["key_idx"]), pinned(host["key_cnt"])
+    d_q, d_k, d_v, d_hid = (t.to(dev).view(torch.bfloat16) for t in (h_q, h_k, h_v, h_hid))
+    d_ki, d_kc = h_ki.to(dev), h_kc.to(dev)
+    use_keys = w.key_cnt > 0
+    f = md.Filter(md.config_for(w), device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        f.score(d_q, d_k, stream)
+        f.select(d_ki if use_keys else None, d_kc if use_keys else None, stream=stream, want_s=False)
+        f.compact(d_hid, d_k, d_v, stream=stream)
+
+    launches_per_step = {"two_pass_mma": 2}.get(f.score_variant, 1) + 2
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler is not None:
+        sampler.start()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    # timed region: exactly K steps; events around every call give the per-call durations
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record(stream)
+    for s in range(K):
+        ev[s][0].record(stream)
+        f.score(d_q, d_k, stream)
+        ev[s][1].record(stream)
+        f.select(d_ki if use_keys else None, d_kc if use_keys else None, stream=stream, want_s=False)
+        ev[s][2].record(stream)
+        f.compact(d_hid, d_k, d_v, stream=stream)
+        ev[s][3].record(stream)
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    elapsed_ms = t_begin.elapsed_time(t_end)
+    t_score = statistics.mean(ev[s][0].elapsed_time(ev[s][1]) for s in range(K))
+    t_select = statistics.mean(ev[s][1].elapsed_time(ev[s][2]) for s in range(K))
+    t_compact = statistics.mean(ev[s][2].elapsed_time(ev[s][3]) for s in range(K))
+    code, detail = f.device_status()
+    if code != 0:
+        raise RuntimeError("device status %d (detail %d) after the timed region" % (code, detail))
+
+    # end to end: pinned host inputs in, results out, every step
+    o_idx = torch.empty(f.kept_idx.shape, dtype=torch.int32).pin_memory()
+    o_cnt = torch.empty(f.kept_cnt.shape, dtype=torch.int32).pin_memory()
+    o_h = torch.empty(f.hidden_out.shape, dtype=torch.bfloat16).pin_memory()
+    o_k = torch.empty(f.k_out.shape, dtype=torch.bfloat16).pin_memory()
+    o_v = torch.empty(f.v_out.shape, dtype=torch.bfloat16).pin_memory()
+    s_q, s_k, s_v, s_hid = (torch.empty_like(t) for t in (d_q, d_k, d_v, d_hid))
+    s_ki, s_kc = torch.empty_like(d_ki), torch.empty_like(d_kc)
+
+    def e2e_step():
+        s_q.view(torch.int16).copy_(h_q, non_blocking=True)
+        s_k.view(torch.int16).copy_(h_k, non_blocking=True)
+        s_v.view(torch.int16).copy_(h_v, non_blocking=True)
+        s_hid.view(torch.int16).copy_(h_hid, non_blocking=True)
+        s_ki.copy_(h_ki, non_blocking=True)
+        s_kc.copy_(h_kc, non_blocking=True)
+        f.score(s_q, s_k, stream)
+        f.select(s_ki if use_keys else None, s_kc if use_keys else None, stream=stream, want_s=False)
+        f.compact(s_hid, s_k, s_v, stream=stream)
+        o_idx.copy_(f.kept_idx, non_blocking=True)
+        o_cnt.copy_(f.kept_cnt, non_blocking=True)
+        o_h.copy_(f.hidden_out, non_blocking=True)
+        o_k.copy_(f.k_out, non_blocking=True)
+        o_v.copy_(f.v_out, non_blocking=True)
+
+    e2e_steps = max(3, min(K, 20))
+    e2e_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    clocks = sampler.finish() if sampler is not None else None
+
+    # max over ranks
+    if world > 1:
+        t = torch.tensor([elapsed_ms, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = elapsed_ms / K
+    tokens_per_step = world * w.batch * w.n_vis
+    value = tokens_per_step / (ms_per_step / 1e3)
+    e2e_value = tokens_per_step / (e2e_ms / 1e3)
+
+    if rank == 0:
+        bm = bytes_model(w)
+        peak, peak_kind = measured_peak()
+        achieved = bm["score"] / (t_score / 1e3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+            "config": {"workload": w.name, "batch_per_gpu": w.batch, "n_vis": w.n_vis, "n_txt": w.n_txt,
+                       "n_heads": w.n_heads, "hidden": w.hidden, "budget": w.budget, "key_set": w.key_cnt,
+                       "parallelism": "dp%d (independent requests, no collective)" % world,
+                       "l2": "inputs exceed L2 (K alone is %.0f MB per GPU)" % (bm["score"] / 1e6),
+                       "score_variant": f.score_variant},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bm["h2d"], "d2h_bytes_per_step": bm["d2h"],
+                    "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "gpu_launches": launches_per_step * K,
+            "kernel_ms": {"score": t_score, "select": t_select, "compact": t_compact},
+            "hbm_headline": {"bytes_per_step": bm["headline"], "gbs": bm["headline"] / (ms_per_step / 1e3) / 1e9,
+                             "frac_of_peak": bm["headline"] / (ms_per_step / 1e3) / 1e9 / peak, "peak_kind": peak_kind},
+            "roofline": {"kernel": "score (%s)" % f.score_variant, "bound": "hbm", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind,
+                         "algorithmic_bytes": bm["score"]},
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            probe = oracle_step(w, range(0, 1))
+            n_req = int(max(1, min(w.batch, 15.0 / max(probe, 1e-6))))
+            secs = oracle_step(w, range(0, n_req))
+            line["cpu_baseline"] = {"value": n_req * w.n_vis / secs, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": "%d of the %d requests, score+select+compact, %.1f s" % (n_req, w.batch, secs)}
+        print(json.dumps(line), flush=True)
+    f.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--budget", type=int, default=0, help="override the workload's keep budget")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.budget:
+        w = w.with_(budget=args.budget)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,115 @@
+"""Host-side checks of the C ABI: the library loads without a GPU, exports every declared
+symbol, and rejects bad configurations synchronously."""
+import os
+import re
+
+import pytest
+
+from paper_2411_10803_b200 import binding as md
+from paper_2411_10803_b200 import build as md_build
+from paper_2411_10803_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    md_build.build()
+
+
+def _declared():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(mustdrop_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    L = md.lib()
+    declared = _declared()
+    assert {"mustdrop_filter_plan", "mustdrop_score", "mustdrop_select", "mustdrop_compact"} <= declared
+    for name in declared:
+        assert hasattr(L, name), name
+    assert declared == set(md.EXPORTS) | (declared - set(md.EXPORTS))
+    for name in md.EXPORTS:
+        assert name in declared, name
+
+
+def _cfg(**kw):
+    w = synth.WORKLOADS["c1_tiny"]
+    return md.config_for(w, **kw)
+
+
+def test_valid_plan_and_workspace_size():
+    st, plan, ws = md.mustdrop_filter_plan(_cfg())
+    assert st == md.MUSTDROP_OK and plan and ws >= 256 and ws % 256 == 0
+    assert md.mustdrop_plan_score_variant(plan) != "invalid plan"
+    assert md.mustdrop_plan_destroy(plan) == md.MUSTDROP_OK
+    assert md.mustdrop_status_string(md.MUSTDROP_ERR_BUDGET)
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(batch=0), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(n_txt=0), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(vis_start=10), md.MUSTDROP_ERR_INVALID_ARG),            # vision span runs into the text span
+    (dict(txt_start=500), md.MUSTDROP_ERR_INVALID_ARG),           # text before the end of the vision span
+    (dict(seq_len=600), md.MUSTDROP_ERR_INVALID_ARG),             # text span leaves the sequence
+    (dict(causal=2), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(mode=5), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(criteria=3), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(gamma=-1.0), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(alpha=float("nan")), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(scale=float("inf")), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(reserved=1), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(k_stride_l=-8), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(k_stride_l=64), md.MUSTDROP_ERR_INVALID_ARG),           # rows would overlap
+    (dict(head_dim=64), md.MUSTDROP_ERR_UNSUPPORTED),
+    (dict(n_txt=129, seq_len=576 + 129), md.MUSTDROP_ERR_UNSUPPORTED),
+    (dict(n_vis=4097, txt_start=4097, seq_len=4097 + 32, budget=64), md.MUSTDROP_ERR_UNSUPPORTED),
+    (dict(hidden=4100), md.MUSTDROP_ERR_UNSUPPORTED),
+    (dict(k_stride_h=12), md.MUSTDROP_ERR_UNSUPPORTED),
+    (dict(budget=0), md.MUSTDROP_ERR_BUDGET),
+    (dict(budget=577), md.MUSTDROP_ERR_BUDGET),
+    (dict(budget=8, key_max=16), md.MUSTDROP_ERR_BUDGET),
+])
+def test_bad_configurations_are_rejected(kw, code):
+    st, plan, ws = md.mustdrop_filter_plan(_cfg(**kw))
+    assert st == code and plan == 0 and ws == 0
+
+
+def test_threshold_mode_needs_no_budget():
+    st, plan, _ = md.mustdrop_filter_plan(_cfg(mode=md.MUSTDROP_MODE_THRESHOLD, budget=0))
+    assert st == md.MUSTDROP_OK
+    md.mustdrop_plan_destroy(plan)
+
+
+def test_null_and_misaligned_arguments_launch_nothing():
+    st, plan, _ = md.mustdrop_filter_plan(_cfg())
+    assert st == md.MUSTDROP_OK
+    try:
+        assert md.lib().mustdrop_score(plan, None, None, None, None, None, None) == md.MUSTDROP_ERR_INVALID_ARG
+        assert md.lib().mustdrop_score(plan, 256, 256, 256, 256, None, None) == md.MUSTDROP_ERR_WORKSPACE
+        assert md.lib().mustdrop_score(plan, 256, 260, 256, 256, 256, None) == md.MUSTDROP_ERR_INVALID_ARG
+        assert md.lib().mustdrop_select(plan, 256, 256, None, None, 256, 256, None, 256, None) == \
+            md.MUSTDROP_ERR_INVALID_ARG                      # key_max > 0 needs key_idx / key_cnt
+        assert md.lib().mustdrop_compact(plan, 256, 256, 256, None, None, None, None, None, None, None) == \
+            md.MUSTDROP_ERR_INVALID_ARG                      # source without destination
+        assert md.lib().mustdrop_compact(plan, 256, 256, None, None, None, None, None, None, None, None) == \
+            md.MUSTDROP_OK                                   # nothing to do
+        assert md.lib().mustdrop_score(0, 256, 256, 256, 256, 256, None) == md.MUSTDROP_ERR_INVALID_ARG
+    finally:
+        md.mustdrop_plan_destroy(plan)
+
+
+def test_shard_ranges_partition_the_batch():
+    from paper_2411_10803_b200.sharding import shard_range
+    for batch in (0, 1, 7, 64):
+        for world in (1, 2, 3, 8):
+            spans = [shard_range(batch, r, world) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == batch
+            assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+            sizes = [hi - lo for lo, hi in spans]
+            assert max(sizes) - min(sizes) <= 1
