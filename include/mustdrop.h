@@ -45,7 +45,8 @@ typedef enum {
   MUSTDROP_ERR_WORKSPACE = 4,     /* null workspace */
   MUSTDROP_ERR_CUDA = 5,          /* a CUDA runtime call failed; see mustdrop_last_cuda_error */
   MUSTDROP_ERR_TIMEOUT = 6,       /* device status only: a bounded wait inside a kernel ran out */
-  MUSTDROP_ERR_BAD_KEY_INDEX = 7  /* device status only: an index outside [0, n_vis) was ignored */
+  MUSTDROP_ERR_BAD_KEY_INDEX = 7, /* device status only: an index outside [0, n_vis) was ignored */
+  MUSTDROP_ERR_SCRATCH_LIMIT = 8  /* mustdrop_score_static: batch * n_heads * n_txt exceeds the built-in scratch */
 } mustdrop_status_t;
 
 typedef enum { MUSTDROP_MODE_BUDGET = 0, MUSTDROP_MODE_THRESHOLD = 1 } mustdrop_mode_t;
@@ -108,6 +109,33 @@ mustdrop_status_t mustdrop_plan_destroy(mustdrop_plan_t *plan);
  */
 mustdrop_status_t mustdrop_score(const mustdrop_plan_t *plan, const void *q_text, const void *k,
                                  float *g_out, float *i_out, void *workspace, void *cuda_stream);
+
+/*
+ * mustdrop_score for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, with identical results.)
+ *
+ * Who needs it: code running where cudaMalloc is not an option - inside an engine whose pool
+ * allocator owns the whole device heap, in a plug-in that must leave the host application's
+ * allocator alone, or after a process has fixed its memory budget.  Such a caller has no
+ * workspace to pass, so this call keeps its scratch (the per-row softmax statistics) in a
+ * fixed 4 MiB array inside the library image; every GPU that loads the library holds that
+ * array until the process exits.  The call itself allocates nothing and frees nothing.
+ *
+ * Limit: batch * n_heads * n_txt <= mustdrop_score_static_max_rows() (524288); a larger plan
+ * is refused with MUSTDROP_ERR_SCRATCH_LIMIT and nothing is launched.
+ * Sharing: all calls on a device use the same array.  Nothing in it has to start at zero
+ * (each call overwrites every entry it later reads), but two calls that overlap on the GPU
+ * (different streams, or different host threads without ordering) race on it and must be
+ * serialised by the caller.  Calls on one stream are safe.
+ * First call: the first call on each device looks up the array's device address (the device
+ * must be current); make that first call outside any stream capture.
+ * Arguments and results are those of mustdrop_score, without the workspace.
+ */
+mustdrop_status_t mustdrop_score_static(const mustdrop_plan_t *plan, const void *q_text, const void *k,
+                                        float *g_out, float *i_out, void *cuda_stream);
+
+/* Largest batch * n_heads * n_txt that mustdrop_score_static accepts. */
+size_t mustdrop_score_static_max_rows(void);
 
 /*
  * Dual criteria, key set and selection (Eq. 9, Eq. 10; the key set O of Sec. 3.3 is always kept).

@@ -24,6 +24,7 @@ MUSTDROP_ERR_WORKSPACE = 4
 MUSTDROP_ERR_CUDA = 5
 MUSTDROP_ERR_TIMEOUT = 6
 MUSTDROP_ERR_BAD_KEY_INDEX = 7
+MUSTDROP_ERR_SCRATCH_LIMIT = 8
 
 MUSTDROP_MODE_BUDGET, MUSTDROP_MODE_THRESHOLD = 0, 1
 MUSTDROP_CRIT_DUAL, MUSTDROP_CRIT_GLOBAL_ONLY, MUSTDROP_CRIT_INDIVIDUAL_ONLY = 0, 1, 2
@@ -31,7 +32,8 @@ MUSTDROP_CRIT_DUAL, MUSTDROP_CRIT_GLOBAL_ONLY, MUSTDROP_CRIT_INDIVIDUAL_ONLY = 0
 EXPORTS = (
     "mustdrop_filter_plan", "mustdrop_plan_destroy", "mustdrop_score", "mustdrop_select",
     "mustdrop_compact", "mustdrop_device_status", "mustdrop_status_string",
-    "mustdrop_last_cuda_error", "mustdrop_plan_score_variant",
+    "mustdrop_last_cuda_error", "mustdrop_plan_score_variant", "mustdrop_score_static",
+    "mustdrop_score_static_max_rows",
 )
 
 
@@ -76,6 +78,9 @@ def lib() -> ctypes.CDLL:
         L.mustdrop_plan_destroy.argtypes = [vp]
         L.mustdrop_score.argtypes = [vp] * 7
         L.mustdrop_select.argtypes = [vp] * 10
+        L.mustdrop_score_static.argtypes = [vp] * 6
+        L.mustdrop_score_static.restype = ctypes.c_int
+        L.mustdrop_score_static_max_rows.restype = ctypes.c_size_t
         L.mustdrop_compact.argtypes = [vp] * 11
         L.mustdrop_device_status.argtypes = [vp, vp, vp, i32p, i32p]
         L.mustdrop_status_string.argtypes = [ctypes.c_int]
@@ -164,6 +169,16 @@ def mustdrop_plan_destroy(plan: int) -> int:
 def mustdrop_score(plan, q_text, k, g_out, i_out, workspace, stream=None) -> int:
     return lib().mustdrop_score(plan, _ptr(q_text), _ptr(k), _ptr(g_out), _ptr(i_out), _ptr(workspace),
                                 _stream(stream))
+
+
+def mustdrop_score_static(plan, q_text, k, g_out, i_out, stream=None) -> int:
+    """mustdrop_score without a workspace, for callers that may not allocate device memory: the
+    scratch lives in a fixed array inside the library.  Calls that overlap on the GPU race on it."""
+    return lib().mustdrop_score_static(plan, _ptr(q_text), _ptr(k), _ptr(g_out), _ptr(i_out), _stream(stream))
+
+
+def mustdrop_score_static_max_rows() -> int:
+    return lib().mustdrop_score_static_max_rows()
 
 
 def mustdrop_select(plan, g, i, key_idx, key_cnt, kept_idx, kept_cnt, s_out, workspace, stream=None) -> int:

@@ -23,6 +23,10 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace
 
+namespace mustdrop {
+void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int32_t>(e); }
+}  // namespace mustdrop
+
 extern "C" {
 
 mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan_t** plan_out,
@@ -188,6 +192,8 @@ const char* mustdrop_status_string(mustdrop_status_t s) {
     case MUSTDROP_ERR_CUDA: return "CUDA runtime error";
     case MUSTDROP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case MUSTDROP_ERR_BAD_KEY_INDEX: return "index outside [0, n_vis) ignored";
+    case MUSTDROP_ERR_SCRATCH_LIMIT:
+      return "batch * n_heads * n_txt exceeds the built-in scratch of mustdrop_score_static (524288 rows)";
   }
   return "unknown status";
 }

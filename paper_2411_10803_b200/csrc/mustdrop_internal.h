@@ -55,6 +55,9 @@ cudaError_t launch_compact(const mustdrop_plan& p, const int32_t* kept_idx, cons
                            const void* hidden, const void* k, const void* v, void* hidden_out, void* k_out,
                            void* v_out, void* workspace, cudaStream_t stream);
 
+// Remember the cudaError_t of a failed runtime call for mustdrop_last_cuda_error (per thread).
+void set_last_cuda_error(cudaError_t e);
+
 // Device-side helper: record the first device-detected condition (never traps).
 __device__ __forceinline__ void record_status(void* workspace, int32_t code, int32_t detail) {
   if (workspace == nullptr) return;
