@@ -1,6 +1,7 @@
 // C-ABI layer: configuration checks, plan object, argument checks, kernel dispatch.
 // The operations themselves are defined by Sec. 3.4 (Eq. 8-10) of the paper; see mustdrop.h.
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -103,7 +104,17 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   }
   (void)cudaGetLastError();
 
+  // Score kernel: the fused single-pass kernel where its geometry covers the shape, else the
+  // two-pass kernel.  MUSTDROP_SCORE_VARIANT (two_pass | fused) and MUSTDROP_CLUSTER (1..8) are
+  // debugging overrides read here, once per plan.
   p->score_variant = kScoreTwoPassMma;
+  {
+    const char* want = std::getenv("MUSTDROP_SCORE_VARIANT");
+    const char* cl = std::getenv("MUSTDROP_CLUSTER");
+    const int forced_cluster = cl ? std::atoi(cl) : 0;
+    const bool allow_fused = !(want && std::strcmp(want, "two_pass") == 0);
+    if (allow_fused && plan_score_fused(r, p->sm_count, forced_cluster, &p->fused)) p->score_variant = kScoreFusedCluster;
+  }
   size_t off = kWsStatusBytes;
   p->ws_rowstats_off = off;
   off += round_up(sizeof(float) * 2 * static_cast<size_t>(r.B) * r.H * r.N, 256);
@@ -129,8 +140,13 @@ mustdrop_status_t mustdrop_score(const mustdrop_plan_t* plan, const void* q_text
   if (!aligned16(q_text) || !aligned16(k) || !aligned16(g_out) || !aligned16(i_out) || !aligned16(workspace))
     return MUSTDROP_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  void* rowstats = static_cast<unsigned char*>(workspace) + plan->ws_rowstats_off;
-  cudaError_t e = mustdrop::launch_score_two_pass(*plan, q_text, k, g_out, i_out, rowstats, stream);
+  cudaError_t e;
+  if (plan->score_variant == mustdrop::kScoreFusedCluster) {
+    e = mustdrop::launch_score_fused(*plan, q_text, k, g_out, i_out, workspace, stream);
+  } else {
+    void* rowstats = static_cast<unsigned char*>(workspace) + plan->ws_rowstats_off;
+    e = mustdrop::launch_score_two_pass(*plan, q_text, k, g_out, i_out, rowstats, stream);
+  }
   return e == cudaSuccess ? MUSTDROP_OK : cuda_fail(e);
 }
 
@@ -204,6 +220,7 @@ const char* mustdrop_plan_score_variant(const mustdrop_plan_t* plan) {
   if (!valid_plan(plan)) return "invalid plan";
   switch (plan->score_variant) {
     case mustdrop::kScoreTwoPassMma: return "two_pass_mma";
+    case mustdrop::kScoreFusedCluster: return "fused_cluster_tcgen05";
   }
   return "unknown";
 }

@@ -19,6 +19,18 @@ constexpr size_t kWsStatusBytes = 256;
 
 enum ScoreVariant : int32_t {
   kScoreTwoPassMma = 0,   // row statistics pass + accumulate pass, warp-level mma
+  kScoreFusedCluster = 1, // one pass: tcgen05 MMA + TMA, key range split over a thread-block cluster
+};
+
+// Launch geometry of the fused score kernel.
+struct FusedGeometry {
+  int32_t halves;     // 2: two M=64 tiles per head (N <= 64); 1: one M=128 tile
+  int32_t cluster;    // CTAs per request
+  int32_t tk;         // keys per CTA
+  int32_t cpl;        // tensor-memory columns per lane and head (= tk / halves)
+  int32_t n_stage;    // shared-memory stages
+  int32_t n_buf;      // tensor-memory buffers
+  size_t smem_bytes;  // dynamic shared memory
 };
 
 struct Resolved {
@@ -39,6 +51,7 @@ struct mustdrop_plan {
   int32_t score_variant;
   size_t ws_bytes;
   size_t ws_rowstats_off;   // float2 [B,H,N]: (row max in log2 units, 1 / row sum)
+  mustdrop::FusedGeometry fused;
 };
 
 namespace mustdrop {
@@ -48,6 +61,9 @@ constexpr uint32_t kPlanMagic = 0x4d445250u;  // "MDRP"
 // Each launcher enqueues on `stream` and returns the launch error (cudaGetLastError).
 cudaError_t launch_score_two_pass(const mustdrop_plan& p, const void* q_text, const void* k,
                                   float* g_out, float* i_out, void* rowstats, cudaStream_t stream);
+bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out);
+cudaError_t launch_score_fused(const mustdrop_plan& p, const void* q_text, const void* k, float* g_out,
+                               float* i_out, void* workspace, cudaStream_t stream);
 cudaError_t launch_select(const mustdrop_plan& p, const float* g, const float* i, const int32_t* key_idx,
                           const int32_t* key_cnt, int32_t* kept_idx, int32_t* kept_cnt, float* s_out,
                           void* workspace, cudaStream_t stream);

@@ -1,0 +1,551 @@
+// Importance scores in ONE pass over the keys (Eq. 1, Eq. 8, Eq. 10), sm_100a only.
+//
+// A thread-block cluster owns one request and splits its L keys over its CTAs; each CTA loops
+// over the heads.  Per head: TMA stages the CTA's K rows and the head's text queries in shared
+// memory, one thread issues tcgen05 MMAs (bf16 in, fp32 accumulators in tensor memory), and the
+// softmax warps read the logits from tensor memory with text queries on the TMEM lanes, so each
+// thread owns one text row and a run of key columns: row maxima and row sums are in-thread.
+// The exponentials (relative to a per-thread maximum) go back to tensor memory, the per-row
+// (max, sum) pairs are exchanged between the CTAs of the cluster through distributed shared
+// memory, and the normalised probabilities are added into per-thread head sums that live in
+// registers for the whole kernel.  After the last head the head mean is reduced over the text
+// rows into G (column sum) and I (column max).  K is read once; nothing goes through global
+// scratch.
+//
+// Lane layouts.  N <= 64: two M=64 MMAs per head write the two halves of the CTA's key range
+// to the lower and upper 16 lanes of every 32-lane TMEM quadrant, so all 128 lanes carry one of
+// 64 text rows.  N > 64: one M=128 MMA, lane = text row.
+//
+// Every wait on an mbarrier is bounded; when a wait runs out the CTA records
+// MUSTDROP_ERR_TIMEOUT in the workspace status word, stops working and goes to the common exit
+// (which still frees tensor memory and joins the cluster barrier).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "mustdrop_internal.h"
+
+namespace mustdrop {
+namespace {
+
+constexpr int kSoftmaxWarps = 8;            // 4 TMEM lane quadrants x 2 column groups
+constexpr int kColGroups = 2;
+constexpr int kSoftmaxThreads = kSoftmaxWarps * 32;
+constexpr int kTmaWarp = kSoftmaxWarps;     // warp 8
+constexpr int kMmaWarp = kSoftmaxWarps + 1; // warp 9
+constexpr int kThreads = (kSoftmaxWarps + 2) * 32;
+constexpr int kChunk = 16;                  // TMEM columns per tcgen05.ld / st
+constexpr int kMaxChunks = 5;               // chunks per thread: up to 160 columns per TMEM lane
+constexpr int kMaxCluster = 8;
+constexpr int kMaxStages = 4;
+constexpr int kMaxBufs = 8;
+constexpr int kTmemCols = 512;
+constexpr long long kWaitCycles = 2000000000LL;  // ~1 s at 2 GHz
+
+struct FusedParams {
+  float* g_out;
+  float* i_out;
+  void* workspace;
+  int32_t H, N, L, M, vis_start, txt_start, causal;
+  int32_t cluster, tk, cpl, n_stage, n_buf;  // CTAs per request, keys per CTA, columns per lane
+  float scale_log2e, inv_heads;
+};
+
+// ---- small PTX wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the wait ran out or the
+// CTA has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag != 0 || clock64() - t0 > kWaitCycles) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t cta_rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(cta_rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_f32x2(uint32_t addr, float a, float b) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const float (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+      ::"r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])),
+        "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])),
+        "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15])), "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Shared-memory matrix descriptor: K-major rows of 128 bytes, 128-byte swizzle, 8-row groups
+// 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return static_cast<uint64_t>((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Merge (m, l) pairs of a softmax row: l counts exponentials relative to 2^m.  m == -inf means "empty".
+__device__ __forceinline__ void merge_stats(float& m, float& l, float om, float ol) {
+  if (om == -INFINITY) return;
+  if (m == -INFINITY) { m = om; l = ol; return; }
+  const float n = fmaxf(m, om);
+  l = l * ex2(m - n) + ol * ex2(om - n);
+  m = n;
+}
+
+struct __align__(8) Barriers {
+  uint64_t full[kMaxStages];     // TMA -> MMA: stage filled
+  uint64_t empty[kMaxStages];    // MMA -> TMA: stage consumed
+  uint64_t tfull[kMaxBufs];      // MMA -> softmax: logits of a head are in tensor memory
+  uint64_t tempty[kMaxBufs];     // softmax -> MMA: tensor-memory buffer free
+  uint64_t sfull[2];             // all CTAs' row statistics of a head have arrived
+  uint64_t pfull;                // every softmax thread has published its (m, l) of the current head
+  uint64_t fin;                  // softmax threads meet before / after staging the head sums
+};
+
+template <int HALVES>
+__global__ void __launch_bounds__(kThreads, 1)
+score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                   const FusedParams p) {
+  constexpr int NROWS = 128 / HALVES;            // text rows carried by the TMEM lanes
+  constexpr int NPART = HALVES * kColGroups;     // threads that share a text row
+
+  extern __shared__ __align__(1024) unsigned char smem_dyn[];
+  __shared__ Barriers bars;
+  __shared__ float2 part[NROWS][NPART];                       // per-thread (m, l) of the current head
+  __shared__ float2 stats[2][kMaxCluster][NROWS];             // per-CTA (m, l), written by every CTA of the cluster
+  __shared__ uint32_t tmem_base_holder;
+  __shared__ int abort_flag_s;
+
+  volatile int* abort_flag = &abort_flag_s;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_cta_rank();
+  const int b = blockIdx.x / p.cluster;
+  const uint32_t stage_bytes = static_cast<uint32_t>(NROWS + p.tk) * 256u;
+  // 1024-byte aligned base of the staging area (shared-window address)
+  const uint32_t stage_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&bars.full[s]), 1); mbar_init(smem_u32(&bars.empty[s]), 1); }
+    for (int s = 0; s < kMaxBufs; ++s) { mbar_init(smem_u32(&bars.tfull[s]), 1); mbar_init(smem_u32(&bars.tempty[s]), kSoftmaxWarps); }
+    for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&bars.sfull[s]), static_cast<uint32_t>(p.cluster) * NROWS);
+    mbar_init(smem_u32(&bars.pfull), kSoftmaxThreads);
+    mbar_init(smem_u32(&bars.fin), kSoftmaxThreads);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kMmaWarp) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // every CTA's barriers are initialised before any remote arrive
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_holder;
+
+  if (warp == kTmaWarp) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      const int key0 = static_cast<int>(rank) * p.tk;
+      int issued = 0;
+      for (int h = 0; h < p.H; ++h) {
+        const int s = h % p.n_stage;
+        const uint32_t ph = static_cast<uint32_t>(h / p.n_stage) & 1u;
+        if (!mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag)) break;
+        const uint32_t full = smem_u32(&bars.full[s]);
+        const uint32_t q_dst = stage_base + s * stage_bytes;
+        const uint32_t k_dst = q_dst + NROWS * 256u;
+        mbar_expect_tx(full, stage_bytes);
+#pragma unroll
+        for (int slab = 0; slab < 2; ++slab) {
+          tma_load_4d(q_dst + slab * (NROWS * 128u), &q_map, slab * 64, 0, h, b, full);
+#pragma unroll
+          for (int hv = 0; hv < HALVES; ++hv)
+            tma_load_4d(k_dst + slab * (p.tk * 128u) + hv * (p.cpl * 128u), &k_map, slab * 64, key0 + hv * p.cpl, h, b,
+                        full);
+        }
+        issued = h + 1;
+      }
+      // Leave only when every copy this thread started has landed (bounded).
+      for (int h = (issued > p.n_stage ? issued - p.n_stage : 0); h < issued; ++h) {
+        const uint32_t bar = smem_u32(&bars.full[h % p.n_stage]);
+        const uint32_t ph = static_cast<uint32_t>(h / p.n_stage) & 1u;
+        const long long t0 = clock64();
+        while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles) {}
+      }
+    }
+  } else if (warp == kMmaWarp) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(p.cpl >> 3) << 17) |
+                             (static_cast<uint32_t>(NROWS >> 4) << 24);
+      for (int h = 0; h < p.H; ++h) {
+        const int s = h % p.n_stage, buf = h % p.n_buf;
+        const uint32_t ph = static_cast<uint32_t>(h / p.n_stage) & 1u;
+        const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
+        if (!mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag)) break;
+        if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t q_src = stage_base + s * stage_bytes;
+        const uint32_t k_src = q_src + NROWS * 256u;
+#pragma unroll
+        for (int hv = 0; hv < HALVES; ++hv) {
+          // the second M=64 tile goes to the upper 16 lanes of every TMEM quadrant
+          const uint32_t d = tmem_base + static_cast<uint32_t>(buf * p.cpl) + (hv ? (16u << 16) : 0u);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t slab = ks >> 2, koff = (ks & 3) * 32u;
+            const uint64_t ad = smem_desc(q_src + slab * (NROWS * 128u) + koff);
+            const uint64_t bd = smem_desc(k_src + slab * (p.tk * 128u) + hv * (p.cpl * 128u) + koff);
+            tc_mma(d, ad, bd, idesc, ks > 0 ? 1u : 0u);
+          }
+        }
+        tc_commit(smem_u32(&bars.empty[s]));
+        tc_commit(smem_u32(&bars.tfull[buf]));
+      }
+    }
+  } else {
+    // ---------------- softmax warps ----------------
+    const int q = warp & 3, g = warp >> 2;
+    const int half = (HALVES == 2) ? (lane >> 4) : 0;
+    const int row = (HALVES == 2) ? (16 * q + (lane & 15)) : (32 * q + lane);
+    const uint32_t lane_addr = static_cast<uint32_t>(32 * q) << 16;
+    const int total_chunks = p.cpl / kChunk;
+    const int my_chunks = (total_chunks - g + kColGroups - 1) / kColGroups;   // chunks g, g+2, ... (uniform per warp)
+    const int key_lane0 = static_cast<int>(rank) * p.tk + half * p.cpl;        // key of this lane's column 0
+    int lim = p.causal ? (p.txt_start + row + 1) : p.L;                        // keys below lim are visible
+    lim = lim < p.L ? lim : p.L;
+    const bool writer = (g == 0) && (half == 0);
+
+    float acc[kMaxChunks][kChunk];
+#pragma unroll
+    for (int t = 0; t < kMaxChunks; ++t)
+#pragma unroll
+      for (int j = 0; j < kChunk; ++j) acc[t][j] = 0.0f;
+
+    bool alive = true;
+    for (int h = 0; h < p.H && alive; ++h) {
+      const int buf = h % p.n_buf;
+      const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
+      const int slot = h & 1;
+      const uint32_t sph = static_cast<uint32_t>(h >> 1) & 1u;
+      if (!mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag)) { alive = false; break; }
+      tc_fence_after();
+      const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
+
+      // phase 1: exponentials relative to the chunk maximum, back into tensor memory
+      float mc[kMaxChunks];
+      float m_thr = -INFINITY, l_thr = 0.0f;
+#pragma unroll
+      for (int t = 0; t < kMaxChunks; ++t) {
+        mc[t] = -INFINITY;
+        if (t < my_chunks) {
+          const int col = kChunk * (g + t * kColGroups);
+          float z[kChunk];
+          tc_ld16(tbuf + col, z);
+          tc_wait_ld();
+          const int nvis = lim - (key_lane0 + col);     // visible columns of this chunk
+          float mx = -INFINITY;
+          if (nvis >= kChunk) {
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) mx = fmaxf(mx, z[j]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) {
+              z[j] = (j < nvis) ? z[j] : -INFINITY;
+              mx = fmaxf(mx, z[j]);
+            }
+          }
+          mx *= p.scale_log2e;                            // scale > 0 keeps the order
+          const float sub = (mx == -INFINITY) ? 0.0f : mx;
+          float lsum = 0.0f;
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) {
+            z[j] = ex2(fmaf(z[j], p.scale_log2e, -sub));
+            lsum += z[j];
+          }
+          tc_st16(tbuf + col, z);
+          mc[t] = mx;
+          merge_stats(m_thr, l_thr, mx, lsum);
+        }
+      }
+      tc_wait_st();
+      part[row][half * kColGroups + g] = make_float2(m_thr, l_thr);
+      mbar_arrive(smem_u32(&bars.pfull));
+      if (writer) {
+        if (!mbar_wait(smem_u32(&bars.pfull), static_cast<uint32_t>(h) & 1u, abort_flag)) { alive = false; break; }
+        float m = -INFINITY, l = 0.0f;
+#pragma unroll
+        for (int x = 0; x < NPART; ++x) {
+          const float2 v = part[row][x];
+          merge_stats(m, l, v.x, v.y);
+        }
+        const uint32_t slot_addr = smem_u32(&stats[slot][rank][row]);
+        const uint32_t bar_addr = smem_u32(&bars.sfull[slot]);
+        for (int c = 0; c < p.cluster; ++c) {
+          st_cluster_f32x2(map_to_cta(slot_addr, c), m, l);
+          mbar_arrive_cluster(map_to_cta(bar_addr, c));
+        }
+      }
+
+      // phase 2: normalise with the row statistics of the whole key range, add into the head sum
+      if (!mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag)) { alive = false; break; }
+      float m = -INFINITY, l = 0.0f;
+      for (int c = 0; c < p.cluster; ++c) {
+        const float2 v = stats[slot][c][row];
+        merge_stats(m, l, v.x, v.y);
+      }
+      const float inv_l = 1.0f / l;
+#pragma unroll
+      for (int t = 0; t < kMaxChunks; ++t) {
+        if (t < my_chunks) {
+          const int col = kChunk * (g + t * kColGroups);
+          const float f = (mc[t] == -INFINITY) ? 0.0f : ex2(mc[t] - m) * inv_l;
+          float e[kChunk];
+          tc_ld16(tbuf + col, e);
+          tc_wait_ld();
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) acc[t][j] = fmaf(e[j], f, acc[t][j]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars.tempty[buf]));
+    }
+
+    // head mean -> column sum (Eq. 8) and column max (Eq. 10) over the text rows
+    mbar_arrive(smem_u32(&bars.fin));
+    if (mbar_wait(smem_u32(&bars.fin), 0u, abort_flag)) {
+      // all TMA copies have landed and all MMAs have read them: the staging area is free
+      float* mat = reinterpret_cast<float*>(smem_dyn + (stage_base - smem_u32(smem_dyn)));
+      const int ld = p.tk | 1;
+      if (row < p.N) {
+#pragma unroll
+        for (int t = 0; t < kMaxChunks; ++t) {
+          if (t < my_chunks) {
+            const int key_local = half * p.cpl + kChunk * (g + t * kColGroups);
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) mat[row * ld + key_local + j] = acc[t][j];
+          }
+        }
+      }
+      mbar_arrive(smem_u32(&bars.fin));
+      const bool staged = mbar_wait(smem_u32(&bars.fin), 1u, abort_flag);
+      for (int c = threadIdx.x; staged && c < p.tk; c += kSoftmaxThreads) {
+        const int j = static_cast<int>(rank) * p.tk + c - p.vis_start;   // vision-relative index
+        if (j < 0 || j >= p.M) continue;
+        float s = 0.0f, mx = -INFINITY;
+        for (int r = 0; r < p.N; ++r) {
+          const float v = mat[r * ld + c];
+          s += v;
+          mx = fmaxf(mx, v);
+        }
+        p.g_out[static_cast<size_t>(b) * p.M + j] = s * p.inv_heads;
+        p.i_out[static_cast<size_t>(b) * p.M + j] = mx * p.inv_heads;
+      }
+    }
+  }
+
+  // ---------------- common exit ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag != 0) record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
+  if (warp == kMmaWarp) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+  cluster_sync_all();   // no CTA leaves while a peer may still write into its shared memory
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+// bf16 tensor [d3][d2][d1][128] with byte strides s1, s2, s3; box = 64 x rows x 1 x 1, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, uint64_t d1, uint64_t d2, uint64_t d3, uint64_t s1, uint64_t s2,
+              uint64_t s3, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[4] = {128, d1, d2, d3};
+  const cuuint64_t strides[3] = {s1, s2, s3};
+  const cuuint32_t box[4] = {64, box_rows, 1, 1};
+  const cuuint32_t elem[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+// Geometry of the fused kernel for a problem; false when the shape is outside what it covers.
+bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out) {
+  const int halves = r.N <= 64 ? 2 : 1;
+  const int nrows = 128 / halves;
+  const int max_cpl = kMaxChunks * kChunk * kColGroups;   // 160 columns per TMEM lane
+  double best = -1.0;
+  FusedGeometry g{};
+  for (int c = 1; c <= kMaxCluster; ++c) {
+    if (forced_cluster > 0 && c != forced_cluster) continue;
+    const int per_cta = (r.L + c - 1) / c;
+    int cpl = (per_cta + halves - 1) / halves;
+    cpl = (cpl + kChunk - 1) / kChunk * kChunk;
+    if (cpl > max_cpl) continue;
+    const int tk = cpl * halves;
+    const size_t stage = static_cast<size_t>(nrows + tk) * 256;
+    int n_stage = static_cast<int>((200 * 1024) / stage);
+    if (n_stage < 2) continue;
+    if (n_stage > kMaxStages) n_stage = kMaxStages;
+    int n_buf = kTmemCols / cpl;
+    if (n_buf > kMaxBufs) n_buf = kMaxBufs;
+    if (n_buf < 2) continue;
+    const long ctas = static_cast<long>(r.B) * c;
+    const long waves = (ctas + sm_count - 1) / sm_count;
+    const double fill = static_cast<double>(ctas) / static_cast<double>(waves * sm_count);
+    const double useful = static_cast<double>(r.L) / static_cast<double>(c * tk);
+    const double score = fill * useful - 0.002 * c;   // prefer smaller clusters among equals
+    if (score > best) {
+      best = score;
+      g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_stage = n_stage; g.n_buf = n_buf;
+      // at least 116 KB, so that two CTAs (each wanting all of tensor memory) never share an SM
+      g.smem_bytes = stage * n_stage + 1024;
+      if (g.smem_bytes < 116 * 1024) g.smem_bytes = 116 * 1024;
+    }
+  }
+  if (best < 0.0) return false;
+  *out = g;
+  return true;
+}
+
+cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, const void* k, float* g_out,
+                               float* i_out, void* workspace, cudaStream_t stream) {
+  const Resolved& r = plan.r;
+  const FusedGeometry& geo = plan.fused;
+  const int nrows = 128 / geo.halves;
+  CUtensorMap q_map, k_map;
+  if (!make_map(&q_map, q_text, r.N, r.H, r.B, 256, static_cast<uint64_t>(r.N) * 256,
+                static_cast<uint64_t>(r.H) * r.N * 256, nrows) ||
+      !make_map(&k_map, k, r.L, r.H, r.B, static_cast<uint64_t>(r.k_sl) * 2, static_cast<uint64_t>(r.k_sh) * 2,
+                static_cast<uint64_t>(r.k_sb) * 2, geo.cpl))
+    return cudaErrorInvalidValue;
+  FusedParams p;
+  p.g_out = g_out; p.i_out = i_out; p.workspace = workspace;
+  p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
+  p.causal = r.causal;
+  p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_stage = geo.n_stage; p.n_buf = geo.n_buf;
+  p.scale_log2e = r.scale_log2e;
+  p.inv_heads = 1.0f / static_cast<float>(r.H);
+
+  auto kernel = geo.halves == 2 ? score_fused_kernel<2> : score_fused_kernel<1>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(geo.smem_bytes));
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(r.B * geo.cluster));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = geo.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(geo.cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, q_map, k_map, p);
+}
+
+}  // namespace mustdrop

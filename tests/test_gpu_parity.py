@@ -29,6 +29,31 @@ def small(**kw):
     return TINY.with_(**base)
 
 
+VARIANTS = ["auto", "two_pass", "fused:1", "fused:2", "fused:3", "fused:5", "fused:8"]
+
+
+@pytest.fixture
+def variant(request, monkeypatch):
+    """Force a score kernel variant / cluster size through the library's debugging overrides."""
+    v = request.param
+    monkeypatch.delenv("MUSTDROP_SCORE_VARIANT", raising=False)
+    monkeypatch.delenv("MUSTDROP_CLUSTER", raising=False)
+    if v == "two_pass":
+        monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "two_pass")
+    elif v.startswith("fused:"):
+        monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "fused")
+        monkeypatch.setenv("MUSTDROP_CLUSTER", v.split(":")[1])
+    return v
+
+
+def check_variant(f, v):
+    if v == "two_pass":
+        assert f.score_variant == "two_pass_mma"
+    elif v.startswith("fused:") and f.score_variant != "fused_cluster_tcgen05":
+        f.close()
+        pytest.skip("this shape does not fit the fused kernel at that cluster size")
+
+
 def key_args(w, d):
     if w.key_cnt == 0:
         return None, None
@@ -50,13 +75,15 @@ SCORE_CASES = [
 ]
 
 
+@pytest.mark.parametrize("variant", VARIANTS, indirect=True)
 @pytest.mark.parametrize("causal", [1, 0])
 @pytest.mark.parametrize("case", range(len(SCORE_CASES)))
-def test_score_matches_oracle(case, causal):
+def test_score_matches_oracle(case, causal, variant):
     w = small(**SCORE_CASES[case])
     d = synth.make_batch(w, with_values=False)
     G, I = oracle.score(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start, bool(causal))
     f = md.Filter(md.config_for(w, causal=causal))
+    check_variant(f, variant)
     g, i = f.score(to_dev_bf16(d["q_text"]), to_dev_bf16(d["k"]))
     torch.cuda.synchronize()
     assert_scores_close(g.cpu().numpy(), G, "G case %d" % case)
@@ -65,7 +92,8 @@ def test_score_matches_oracle(case, causal):
     f.close()
 
 
-def test_score_with_text_after_the_span_and_explicit_scale():
+@pytest.mark.parametrize("variant", ["auto", "two_pass", "fused:2"], indirect=True)
+def test_score_with_text_after_the_span_and_explicit_scale(variant):
     """Keys beyond the text span (a later turn) are visible only when the mask is off."""
     w = small(n_vis=90, n_txt=9)
     d = synth.make_batch(w, with_values=False)
@@ -82,7 +110,8 @@ def test_score_with_text_after_the_span_and_explicit_scale():
         f.close()
 
 
-def test_score_with_strided_keys():
+@pytest.mark.parametrize("variant", ["auto", "two_pass", "fused:2"], indirect=True)
+def test_score_with_strided_keys(variant):
     """K stored as [B, L, H, D] (token-major) and addressed through the plan's strides."""
     w = small(n_vis=70, n_txt=12, n_heads=4, hidden=512)
     d = synth.make_batch(w, with_values=False)
@@ -96,7 +125,8 @@ def test_score_with_strided_keys():
     f.close()
 
 
-def test_score_extreme_logits_do_not_overflow():
+@pytest.mark.parametrize("variant", ["auto", "two_pass", "fused:2"], indirect=True)
+def test_score_extreme_logits_do_not_overflow(variant):
     w = small(n_vis=40, n_txt=6, n_heads=2, hidden=256, n_salient=0)
     d = synth.make_batch(w, with_values=False)
     q = synth.bf16_bits_to_f32(d["q_text"]) * 6.0
