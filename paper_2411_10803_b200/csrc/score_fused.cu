@@ -39,7 +39,8 @@ constexpr int kMaxCluster = 8;
 constexpr int kMaxStages = 4;
 constexpr int kMaxBufs = 8;
 constexpr int kTmemCols = 512;
-constexpr long long kWaitCycles = 2000000000LL;  // ~1 s at 2 GHz
+constexpr int kStatSlots = 4;               // row-statistics slots in flight (software pipeline depth 1 needs 4)
+constexpr long long kWaitCycles = 200000000LL;   // ~0.1 s at 2 GHz; no legitimate wait comes near it
 
 struct FusedParams {
   float* g_out;
@@ -92,11 +93,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t cta
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(cta_rank));
   return r;
 }
-__device__ __forceinline__ void st_cluster_f32x2(uint32_t addr, float a, float b) {
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+// Asynchronous store of 8 bytes into (possibly another CTA's) shared memory; its arrival is
+// counted on the mbarrier of the destination CTA, so no fence or separate arrive is needed.
+__device__ __forceinline__ void st_async_f32x2(uint32_t addr, float a, float b, uint32_t bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];" ::"r"(addr),
+               "f"(a), "f"(b), "r"(bar)
+               : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -162,6 +164,20 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   return static_cast<uint64_t>((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// Optional timeline tracing (compiled out unless MUSTDROP_TRACE is defined): one global-timer
+// stamp per (CTA, head, event) into the scratch part of the workspace.
+#ifdef MUSTDROP_TRACE
+__device__ __forceinline__ void trace_stamp(void* workspace, int n_heads, int h, int ev) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(workspace) + 4096)
+      [(static_cast<size_t>(blockIdx.x) * n_heads + h) * 16 + ev] = t;
+}
+#define MD_TRACE(h, ev) trace_stamp(p.workspace, p.H, (h), (ev))
+#else
+#define MD_TRACE(h, ev) ((void)0)
+#endif
+
 // Merge (m, l) pairs of a softmax row: l counts exponentials relative to 2^m.  m == -inf means "empty".
 __device__ __forceinline__ void merge_stats(float& m, float& l, float om, float ol) {
   if (om == -INFINITY) return;
@@ -176,7 +192,7 @@ struct __align__(8) Barriers {
   uint64_t empty[kMaxStages];    // MMA -> TMA: stage consumed
   uint64_t tfull[kMaxBufs];      // MMA -> softmax: logits of a head are in tensor memory
   uint64_t tempty[kMaxBufs];     // softmax -> MMA: tensor-memory buffer free
-  uint64_t sfull[2];             // all CTAs' row statistics of a head have arrived
+  uint64_t sfull[kStatSlots];    // all CTAs' row statistics of a head have arrived
   uint64_t pfull;                // every softmax thread has published its (m, l) of the current head
   uint64_t fin;                  // softmax threads meet before / after staging the head sums
 };
@@ -187,11 +203,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                    const FusedParams p) {
   constexpr int NROWS = 128 / HALVES;            // text rows carried by the TMEM lanes
   constexpr int NPART = HALVES * kColGroups;     // threads that share a text row
+  constexpr unsigned kWriterLanes = (HALVES == 2) ? 0x0000ffffu : 0xffffffffu;
 
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
   __shared__ Barriers bars;
-  __shared__ float2 part[NROWS][NPART];                       // per-thread (m, l) of the current head
-  __shared__ float2 stats[2][kMaxCluster][NROWS];             // per-CTA (m, l), written by every CTA of the cluster
   __shared__ uint32_t tmem_base_holder;
   __shared__ int abort_flag_s;
 
@@ -200,14 +215,17 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const uint32_t rank = cluster_cta_rank();
   const int b = blockIdx.x / p.cluster;
   const uint32_t stage_bytes = static_cast<uint32_t>(NROWS + p.tk) * 256u;
-  // 1024-byte aligned base of the staging area (shared-window address)
+  // dynamic shared memory: [stages][stats: kStatSlots x cluster x NROWS float2][part: 2 x NROWS x NPART float2]
   const uint32_t stage_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* stage_ptr = smem_dyn + (stage_base - smem_u32(smem_dyn));
+  float2* stats = reinterpret_cast<float2*>(stage_ptr + static_cast<size_t>(p.n_stage) * stage_bytes);
+  float2* part = stats + kStatSlots * p.cluster * NROWS;
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&bars.full[s]), 1); mbar_init(smem_u32(&bars.empty[s]), 1); }
     for (int s = 0; s < kMaxBufs; ++s) { mbar_init(smem_u32(&bars.tfull[s]), 1); mbar_init(smem_u32(&bars.tempty[s]), kSoftmaxWarps); }
-    for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&bars.sfull[s]), static_cast<uint32_t>(p.cluster) * NROWS);
+    for (int s = 0; s < kStatSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), 1);
     mbar_init(smem_u32(&bars.pfull), kSoftmaxThreads);
     mbar_init(smem_u32(&bars.fin), kSoftmaxThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -237,6 +255,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const uint32_t q_dst = stage_base + s * stage_bytes;
         const uint32_t k_dst = q_dst + NROWS * 256u;
         mbar_expect_tx(full, stage_bytes);
+        MD_TRACE(h, 0);
 #pragma unroll
         for (int slab = 0; slab < 2; ++slab) {
           tma_load_4d(q_dst + slab * (NROWS * 128u), &q_map, slab * 64, 0, h, b, full);
@@ -265,7 +284,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const uint32_t ph = static_cast<uint32_t>(h / p.n_stage) & 1u;
         const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
         if (!mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag)) break;
+        MD_TRACE(h, 1);
         if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag)) break;
+        MD_TRACE(h, 2);
         tc_fence_after();
         const uint32_t q_src = stage_base + s * stage_bytes;
         const uint32_t k_src = q_src + NROWS * 256u;
@@ -287,6 +308,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     }
   } else {
     // ---------------- softmax warps ----------------
+    // Software pipeline over heads: exponentials of head h, then normalise-and-add of head h-1,
+    // so the exchange of row statistics between CTAs overlaps the next head's arithmetic.
     const int q = warp & 3, g = warp >> 2;
     const int half = (HALVES == 2) ? (lane >> 4) : 0;
     const int row = (HALVES == 2) ? (16 * q + (lane & 15)) : (32 * q + lane);
@@ -295,8 +318,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const int my_chunks = (total_chunks - g + kColGroups - 1) / kColGroups;   // chunks g, g+2, ... (uniform per warp)
     const int key_lane0 = static_cast<int>(rank) * p.tk + half * p.cpl;        // key of this lane's column 0
     int lim = p.causal ? (p.txt_start + row + 1) : p.L;                        // keys below lim are visible
-    lim = lim < p.L ? lim : p.L;
+    lim = (lim < p.L ? lim : p.L) - key_lane0;                                 // ... as a column count of this lane
+    const bool all_visible = lim >= p.cpl;
     const bool writer = (g == 0) && (half == 0);
+    const int part_idx = row * NPART + half * kColGroups + g;
 
     float acc[kMaxChunks][kChunk];
 #pragma unroll
@@ -304,101 +329,147 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 #pragma unroll
       for (int j = 0; j < kChunk; ++j) acc[t][j] = 0.0f;
 
-    bool alive = true;
-    for (int h = 0; h < p.H && alive; ++h) {
-      const int buf = h % p.n_buf;
-      const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
-      const int slot = h & 1;
-      const uint32_t sph = static_cast<uint32_t>(h >> 1) & 1u;
-      if (!mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag)) { alive = false; break; }
-      tc_fence_after();
-      const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
-
-      // phase 1: exponentials relative to the chunk maximum, back into tensor memory
-      float mc[kMaxChunks];
-      float m_thr = -INFINITY, l_thr = 0.0f;
+    // The thread's chunks are worked in two batches (chunks 0-2 and 3-4), each with its own
+    // stabiliser, to bound the registers that hold logits in flight.
+#define MD_BATCH_LO(bt) ((bt) * 3)
+#define MD_BATCH_HI(bt) ((bt) == 0 ? 3 : kMaxChunks)
+    float m_prev[2] = {-INFINITY, -INFINITY};   // stabilisers of head h-1, per batch
+    // Every decision to give up is taken by the whole warp (votes), so no lane is ever left
+    // alone at a warp-level synchronisation.
+    for (int h = 0; h <= p.H; ++h) {
+      float m_cur[2] = {-INFINITY, -INFINITY};
+      bool bad = false;
+      if (h < p.H) {
+        // ---- exponentials of head h, relative to the batch maximum, back into tensor memory
+        const int buf = h % p.n_buf;
+        const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag))) break;
+        if (threadIdx.x == 0) MD_TRACE(h, 3);
+        tc_fence_after();
+        const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
+        float m_thr = -INFINITY, l_thr = 0.0f;
 #pragma unroll
-      for (int t = 0; t < kMaxChunks; ++t) {
-        mc[t] = -INFINITY;
-        if (t < my_chunks) {
-          const int col = kChunk * (g + t * kColGroups);
-          float z[kChunk];
-          tc_ld16(tbuf + col, z);
-          tc_wait_ld();
-          const int nvis = lim - (key_lane0 + col);     // visible columns of this chunk
-          float mx = -INFINITY;
-          if (nvis >= kChunk) {
+        for (int bt = 0; bt < 2; ++bt) {
+          if (MD_BATCH_LO(bt) < my_chunks) {
+            float z[3][kChunk];
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) mx = fmaxf(mx, z[j]);
-          } else {
+            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
+              if (t < my_chunks) tc_ld16(tbuf + kChunk * (g + t * kColGroups), z[t - MD_BATCH_LO(bt)]);
+            tc_wait_ld();
+            if (threadIdx.x == 0) MD_TRACE(h, 8 + bt);
+            if (!all_visible) {
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) {
-              z[j] = (j < nvis) ? z[j] : -INFINITY;
-              mx = fmaxf(mx, z[j]);
+              for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t) {
+                const int nvis = lim - kChunk * (g + t * kColGroups);
+#pragma unroll
+                for (int j = 0; j < kChunk; ++j) z[t - MD_BATCH_LO(bt)][j] = (j < nvis) ? z[t - MD_BATCH_LO(bt)][j] : -INFINITY;
+              }
             }
-          }
-          mx *= p.scale_log2e;                            // scale > 0 keeps the order
-          const float sub = (mx == -INFINITY) ? 0.0f : mx;
-          float lsum = 0.0f;
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-          for (int j = 0; j < kChunk; ++j) {
-            z[j] = ex2(fmaf(z[j], p.scale_log2e, -sub));
-            lsum += z[j];
+            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
+              if (t < my_chunks) {
+#pragma unroll
+                for (int j = 0; j < kChunk; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], z[t - MD_BATCH_LO(bt)][j]);
+              }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;  // scale > 0 keeps the order
+            const float sub = (mx == -INFINITY) ? 0.0f : mx;
+            float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
+              if (t < my_chunks) {
+#pragma unroll
+                for (int j = 0; j < kChunk; ++j) {
+                  const float e = ex2(fmaf(z[t - MD_BATCH_LO(bt)][j], p.scale_log2e, -sub));
+                  z[t - MD_BATCH_LO(bt)][j] = e;
+                  ls4[j & 3] += e;
+                }
+                tc_st16(tbuf + kChunk * (g + t * kColGroups), z[t - MD_BATCH_LO(bt)]);
+              }
+            m_cur[bt] = mx;
+            merge_stats(m_thr, l_thr, mx, (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
+            if (threadIdx.x == 0) MD_TRACE(h, 10 + bt);
           }
-          tc_st16(tbuf + col, z);
-          mc[t] = mx;
-          merge_stats(m_thr, l_thr, mx, lsum);
+        }
+        // one thread arms this head's statistics barrier with the bytes all CTAs will send
+        if (threadIdx.x == 0)
+          mbar_expect_tx(smem_u32(&bars.sfull[h % kStatSlots]), static_cast<uint32_t>(p.cluster) * NROWS * 8u);
+        part[(h & 1) * NROWS * NPART + part_idx] = make_float2(m_thr, l_thr);
+        if (threadIdx.x == 0) MD_TRACE(h, 4);
+        mbar_arrive(smem_u32(&bars.pfull));
+        if (writer) {
+          bad = !__all_sync(kWriterLanes, mbar_wait(smem_u32(&bars.pfull), static_cast<uint32_t>(h) & 1u, abort_flag));
+        }
+        if (threadIdx.x == 0) MD_TRACE(h, 12);
+        if (writer && !bad) {
+          float m = -INFINITY, l = 0.0f;
+#pragma unroll
+          for (int x = 0; x < NPART; ++x) {
+            const float2 v = part[(h & 1) * NROWS * NPART + row * NPART + x];
+            merge_stats(m, l, v.x, v.y);
+          }
+          const int slot = h % kStatSlots;
+          const uint32_t slot_addr = smem_u32(&stats[(slot * p.cluster + rank) * NROWS + row]);
+          const uint32_t bar_addr = smem_u32(&bars.sfull[slot]);
+          for (int c = 0; c < p.cluster; ++c) st_async_f32x2(map_to_cta(slot_addr, c), m, l, map_to_cta(bar_addr, c));
         }
       }
-      tc_wait_st();
-      part[row][half * kColGroups + g] = make_float2(m_thr, l_thr);
-      mbar_arrive(smem_u32(&bars.pfull));
-      if (writer) {
-        if (!mbar_wait(smem_u32(&bars.pfull), static_cast<uint32_t>(h) & 1u, abort_flag)) { alive = false; break; }
+      if (h >= 1) {
+        // ---- head h-1: normalise with the row statistics of the whole key range, add into the head sum
+        const int hp = h - 1;
+        const int buf = hp % p.n_buf;
+        const int slot = hp % kStatSlots;
+        const uint32_t sph = static_cast<uint32_t>(hp / kStatSlots) & 1u;
+        if (threadIdx.x == 0) MD_TRACE(hp, 5);
+        if (!__all_sync(0xffffffffu, !bad && mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag))) break;
+        if (threadIdx.x == 0) MD_TRACE(hp, 6);
         float m = -INFINITY, l = 0.0f;
-#pragma unroll
-        for (int x = 0; x < NPART; ++x) {
-          const float2 v = part[row][x];
+        for (int c = 0; c < p.cluster; ++c) {
+          const float2 v = stats[(slot * p.cluster + c) * NROWS + row];
           merge_stats(m, l, v.x, v.y);
         }
-        const uint32_t slot_addr = smem_u32(&stats[slot][rank][row]);
-        const uint32_t bar_addr = smem_u32(&bars.sfull[slot]);
-        for (int c = 0; c < p.cluster; ++c) {
-          st_cluster_f32x2(map_to_cta(slot_addr, c), m, l);
-          mbar_arrive_cluster(map_to_cta(bar_addr, c));
-        }
-      }
-
-      // phase 2: normalise with the row statistics of the whole key range, add into the head sum
-      if (!mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag)) { alive = false; break; }
-      float m = -INFINITY, l = 0.0f;
-      for (int c = 0; c < p.cluster; ++c) {
-        const float2 v = stats[slot][c][row];
-        merge_stats(m, l, v.x, v.y);
-      }
-      const float inv_l = 1.0f / l;
+        const float inv_l = 1.0f / l;
+        const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
+        if (threadIdx.x == 0) MD_TRACE(hp, 13);
+        tc_wait_st();
+        if (threadIdx.x == 0) MD_TRACE(hp, 14);
 #pragma unroll
-      for (int t = 0; t < kMaxChunks; ++t) {
-        if (t < my_chunks) {
-          const int col = kChunk * (g + t * kColGroups);
-          const float f = (mc[t] == -INFINITY) ? 0.0f : ex2(mc[t] - m) * inv_l;
-          float e[kChunk];
-          tc_ld16(tbuf + col, e);
-          tc_wait_ld();
+        for (int bt = 0; bt < 2; ++bt) {
+          if (MD_BATCH_LO(bt) < my_chunks) {
+            const float f = (m_prev[bt] == -INFINITY) ? 0.0f : ex2(m_prev[bt] - m) * inv_l;
+            float e[3][kChunk];
 #pragma unroll
-          for (int j = 0; j < kChunk; ++j) acc[t][j] = fmaf(e[j], f, acc[t][j]);
+            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
+              if (t < my_chunks) tc_ld16(tbuf + kChunk * (g + t * kColGroups), e[t - MD_BATCH_LO(bt)]);
+            tc_wait_ld();
+            if (threadIdx.x == 0 && bt == 0) MD_TRACE(hp, 15);
+#pragma unroll
+            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
+              if (t < my_chunks) {
+#pragma unroll
+                for (int j = 0; j < kChunk; ++j) acc[t][j] = fmaf(e[t - MD_BATCH_LO(bt)][j], f, acc[t][j]);
+              }
+          }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars.tempty[buf]));
+        if (threadIdx.x == 0) MD_TRACE(hp, 7);
+      } else if (__any_sync(0xffffffffu, bad)) {
+        break;
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars.tempty[buf]));
+      m_prev[0] = m_cur[0];
+      m_prev[1] = m_cur[1];
     }
+
+#undef MD_BATCH_LO
+#undef MD_BATCH_HI
 
     // head mean -> column sum (Eq. 8) and column max (Eq. 10) over the text rows
     mbar_arrive(smem_u32(&bars.fin));
     if (mbar_wait(smem_u32(&bars.fin), 0u, abort_flag)) {
       // all TMA copies have landed and all MMAs have read them: the staging area is free
-      float* mat = reinterpret_cast<float*>(smem_dyn + (stage_base - smem_u32(smem_dyn)));
+      float* mat = reinterpret_cast<float*>(stage_ptr);
       const int ld = p.tk | 1;
       if (row < p.N) {
 #pragma unroll
@@ -486,12 +557,15 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     if (cpl > max_cpl) continue;
     const int tk = cpl * halves;
     const size_t stage = static_cast<size_t>(nrows + tk) * 256;
-    int n_stage = static_cast<int>((200 * 1024) / stage);
+    // row statistics (kStatSlots x cluster x rows) and per-thread partials (2 x rows x threads per row), 8 bytes each
+    const size_t extra = static_cast<size_t>(kStatSlots) * c * nrows * 8 + 2 * static_cast<size_t>(nrows) * halves * kColGroups * 8;
+    const size_t budget = 227 * 1024 - 2048 /* static */ - 1024 /* alignment */ - extra;
+    int n_stage = static_cast<int>(budget / stage);
     if (n_stage < 2) continue;
     if (n_stage > kMaxStages) n_stage = kMaxStages;
     int n_buf = kTmemCols / cpl;
     if (n_buf > kMaxBufs) n_buf = kMaxBufs;
-    if (n_buf < 2) continue;
+    if (n_buf < 3) continue;   // logits of head h+1, exponentials of heads h and h-1
     const long ctas = static_cast<long>(r.B) * c;
     const long waves = (ctas + sm_count - 1) / sm_count;
     const double fill = static_cast<double>(ctas) / static_cast<double>(waves * sm_count);
@@ -501,7 +575,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
       best = score;
       g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_stage = n_stage; g.n_buf = n_buf;
       // at least 116 KB, so that two CTAs (each wanting all of tensor memory) never share an SM
-      g.smem_bytes = stage * n_stage + 1024;
+      g.smem_bytes = stage * n_stage + 1024 + extra;
       if (g.smem_bytes < 116 * 1024) g.smem_bytes = 116 * 1024;
     }
   }
