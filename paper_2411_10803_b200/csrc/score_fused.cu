@@ -1,16 +1,19 @@
 // Importance scores in ONE pass over the keys (Eq. 1, Eq. 8, Eq. 10), sm_100a only.
 //
 // A thread-block cluster owns one request and splits its L keys over its CTAs; each CTA loops
-// over the heads.  Per head: TMA stages the CTA's K rows and the head's text queries in shared
-// memory, one thread issues tcgen05 MMAs (bf16 in, fp32 accumulators in tensor memory), and the
-// softmax warps read the logits from tensor memory with text queries on the TMEM lanes, so each
-// thread owns one text row and a run of key columns: row maxima and row sums are in-thread.
-// The exponentials (relative to a per-thread maximum) go back to tensor memory, the per-row
-// (max, sum) pairs are exchanged between the CTAs of the cluster through distributed shared
-// memory, and the normalised probabilities are added into per-thread head sums that live in
-// registers for the whole kernel.  After the last head the head mean is reduced over the text
-// rows into G (column sum) and I (column max).  K is read once; nothing goes through global
-// scratch.
+// over the heads.  Warp roles inside a CTA (16 warps):
+//   TMA warp      stages the CTA's K rows and the head's text queries in shared memory;
+//   MMA warp      one thread issues tcgen05 MMAs (bf16 in, fp32 logits in tensor memory);
+//   8 exp warps   read the logits with text queries on the TMEM lanes (a thread owns one text row
+//                 and a run of key columns, so row maxima and sums are in-thread), write the
+//                 exponentials back to tensor memory and send their (max, sum) pairs to every
+//                 CTA of the cluster with asynchronous distributed-shared-memory stores that
+//                 count on the receiver's mbarrier;
+//   4 add warps   once all pairs of a head have arrived, normalise the exponentials and add them
+//                 into per-thread head sums that live in registers for the whole kernel.
+// Three tensor-memory buffers keep the MMA, exp and add stages of consecutive heads in flight.
+// After the last head the head mean is reduced over the text rows into G (column sum) and
+// I (column max).  K is read once; nothing goes through global scratch.
 //
 // Lane layouts.  N <= 64: two M=64 MMAs per head write the two halves of the CTA's key range
 // to the lower and upper 16 lanes of every 32-lane TMEM quadrant, so all 128 lanes carry one of
@@ -27,19 +30,21 @@
 namespace mustdrop {
 namespace {
 
-constexpr int kSoftmaxWarps = 8;            // 4 TMEM lane quadrants x 2 column groups
+constexpr int kExpWarps = 8;                // warps 0-7: 4 TMEM lane quadrants x 2 column groups
 constexpr int kColGroups = 2;
-constexpr int kSoftmaxThreads = kSoftmaxWarps * 32;
-constexpr int kTmaWarp = kSoftmaxWarps;     // warp 8
-constexpr int kMmaWarp = kSoftmaxWarps + 1; // warp 9
-constexpr int kThreads = (kSoftmaxWarps + 2) * 32;
+constexpr int kAddWarps = 4;                // warps 8-11: one per lane quadrant, all columns
+constexpr int kExpThreads = kExpWarps * 32;
+constexpr int kAddThreads = kAddWarps * 32;
+constexpr int kTmaWarp = kExpWarps + kAddWarps;   // warp 12
+constexpr int kMmaWarp = kTmaWarp + 1;            // warp 13; warps 14-15 only fill the last warpgroup
+constexpr int kThreads = 16 * 32;
 constexpr int kChunk = 16;                  // TMEM columns per tcgen05.ld / st
-constexpr int kMaxChunks = 5;               // chunks per thread: up to 160 columns per TMEM lane
+constexpr int kBatch0 = 3;                  // an exp thread works its chunks in two batches: 3 + 2
 constexpr int kMaxCluster = 8;
 constexpr int kMaxStages = 4;
-constexpr int kMaxBufs = 8;
+constexpr int kNumBufs = 3;                 // tensor-memory buffers (MMA, exp, add stages in flight)
+constexpr int kStatSlots = 2 * kNumBufs;    // a peer's exp warps run at most 2*kNumBufs heads ahead of our add warps
 constexpr int kTmemCols = 512;
-constexpr int kStatSlots = 4;               // row-statistics slots in flight (software pipeline depth 1 needs 4)
 constexpr long long kWaitCycles = 200000000LL;   // ~0.1 s at 2 GHz; no legitimate wait comes near it
 
 struct FusedParams {
@@ -47,7 +52,7 @@ struct FusedParams {
   float* i_out;
   void* workspace;
   int32_t H, N, L, M, vis_start, txt_start, causal;
-  int32_t cluster, tk, cpl, n_stage, n_buf;  // CTAs per request, keys per CTA, columns per lane
+  int32_t cluster, tk, cpl, n_stage;  // CTAs per request, keys per CTA, columns per TMEM lane
   float scale_log2e, inv_heads;
 };
 
@@ -178,32 +183,27 @@ __device__ __forceinline__ void trace_stamp(void* workspace, int n_heads, int h,
 #define MD_TRACE(h, ev) ((void)0)
 #endif
 
-// Merge (m, l) pairs of a softmax row: l counts exponentials relative to 2^m.  m == -inf means "empty".
-__device__ __forceinline__ void merge_stats(float& m, float& l, float om, float ol) {
-  if (om == -INFINITY) return;
-  if (m == -INFINITY) { m = om; l = ol; return; }
-  const float n = fmaxf(m, om);
-  l = l * ex2(m - n) + ol * ex2(om - n);
-  m = n;
-}
-
 struct __align__(8) Barriers {
   uint64_t full[kMaxStages];     // TMA -> MMA: stage filled
   uint64_t empty[kMaxStages];    // MMA -> TMA: stage consumed
-  uint64_t tfull[kMaxBufs];      // MMA -> softmax: logits of a head are in tensor memory
-  uint64_t tempty[kMaxBufs];     // softmax -> MMA: tensor-memory buffer free
-  uint64_t sfull[kStatSlots];    // all CTAs' row statistics of a head have arrived
-  uint64_t pfull;                // every softmax thread has published its (m, l) of the current head
-  uint64_t fin;                  // softmax threads meet before / after staging the head sums
+  uint64_t tfull[kNumBufs];      // MMA -> exp warps: logits of a head are in tensor memory
+  uint64_t eready[kNumBufs];     // exp -> add warps: exponentials of a head are in tensor memory
+  uint64_t tempty[kNumBufs];     // add warps -> MMA: tensor-memory buffer free
+  uint64_t sfull[kStatSlots];    // all CTAs' (max, sum) pairs of a head have arrived
+  uint64_t fin;                  // add warps meet before / after staging the head sums
 };
 
-template <int HALVES>
+// HALVES: 2 = two M=64 tiles per head (N <= 64), 1 = one M=128 tile.
+// ACH: chunks (of 16 columns) an add thread may own; an exp thread owns up to (ACH+1)/2.
+template <int HALVES, int ACH>
 __global__ void __launch_bounds__(kThreads, 1)
 score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const FusedParams p) {
   constexpr int NROWS = 128 / HALVES;            // text rows carried by the TMEM lanes
-  constexpr int NPART = HALVES * kColGroups;     // threads that share a text row
-  constexpr unsigned kWriterLanes = (HALVES == 2) ? 0x0000ffffu : 0xffffffffu;
+  constexpr int ECH = (ACH + 1) / 2;             // chunks per exp thread
+  constexpr int NBT = (ECH > kBatch0) ? 2 : 1;   // batches (= stabilisers) per exp thread
+  constexpr int EPR = kColGroups * NBT;          // (max, sum) pairs per text row and CTA
+  constexpr bool kRealloc = ACH > 5;             // move registers from the other warpgroups to the add warps
 
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
   __shared__ Barriers bars;
@@ -215,19 +215,22 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const uint32_t rank = cluster_cta_rank();
   const int b = blockIdx.x / p.cluster;
   const uint32_t stage_bytes = static_cast<uint32_t>(NROWS + p.tk) * 256u;
-  // dynamic shared memory: [stages][stats: kStatSlots x cluster x NROWS float2][part: 2 x NROWS x NPART float2]
+  // dynamic shared memory: [stages][stats: kStatSlots x cluster x NROWS x EPR float2]
   const uint32_t stage_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* stage_ptr = smem_dyn + (stage_base - smem_u32(smem_dyn));
   float2* stats = reinterpret_cast<float2*>(stage_ptr + static_cast<size_t>(p.n_stage) * stage_bytes);
-  float2* part = stats + kStatSlots * p.cluster * NROWS;
+  const uint32_t slot_pairs = static_cast<uint32_t>(p.cluster) * NROWS * EPR;   // pairs per slot
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&bars.full[s]), 1); mbar_init(smem_u32(&bars.empty[s]), 1); }
-    for (int s = 0; s < kMaxBufs; ++s) { mbar_init(smem_u32(&bars.tfull[s]), 1); mbar_init(smem_u32(&bars.tempty[s]), kSoftmaxWarps); }
+    for (int s = 0; s < kNumBufs; ++s) {
+      mbar_init(smem_u32(&bars.tfull[s]), 1);
+      mbar_init(smem_u32(&bars.eready[s]), kExpWarps);
+      mbar_init(smem_u32(&bars.tempty[s]), kAddWarps);
+    }
     for (int s = 0; s < kStatSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), 1);
-    mbar_init(smem_u32(&bars.pfull), kSoftmaxThreads);
-    mbar_init(smem_u32(&bars.fin), kSoftmaxThreads);
+    mbar_init(smem_u32(&bars.fin), kAddThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kMmaWarp) {
@@ -238,13 +241,14 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   }
   tc_fence_before();
   __syncthreads();
-  cluster_sync_all();   // every CTA's barriers are initialised before any remote arrive
+  cluster_sync_all();   // every CTA's barriers are initialised before any remote store counts on them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_holder;
 
-  if (warp == kTmaWarp) {
-    // ---------------- TMA producer ----------------
-    if (lane == 0) {
+  if (warp >= kTmaWarp) {
+    if (kRealloc) asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    if (warp == kTmaWarp && lane == 0) {
+      // ---------------- TMA producer ----------------
       const int key0 = static_cast<int>(rank) * p.tk;
       int issued = 0;
       for (int h = 0; h < p.H; ++h) {
@@ -273,16 +277,14 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const long long t0 = clock64();
         while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles) {}
       }
-    }
-  } else if (warp == kMmaWarp) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    } else if (warp == kMmaWarp && lane == 0) {
+      // ---------------- MMA issuer ----------------
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(p.cpl >> 3) << 17) |
                              (static_cast<uint32_t>(NROWS >> 4) << 24);
       for (int h = 0; h < p.H; ++h) {
-        const int s = h % p.n_stage, buf = h % p.n_buf;
+        const int s = h % p.n_stage, buf = h % kNumBufs;
         const uint32_t ph = static_cast<uint32_t>(h / p.n_stage) & 1u;
-        const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
+        const uint32_t bph = static_cast<uint32_t>(h / kNumBufs) & 1u;
         if (!mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag)) break;
         MD_TRACE(h, 1);
         if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag)) break;
@@ -306,10 +308,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         tc_commit(smem_u32(&bars.tfull[buf]));
       }
     }
-  } else {
-    // ---------------- softmax warps ----------------
-    // Software pipeline over heads: exponentials of head h, then normalise-and-add of head h-1,
-    // so the exchange of row statistics between CTAs overlaps the next head's arithmetic.
+  } else if (warp < kExpWarps) {
+    // ---------------- exp warps ----------------
+    if (kRealloc) asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
     const int q = warp & 3, g = warp >> 2;
     const int half = (HALVES == 2) ? (lane >> 4) : 0;
     const int row = (HALVES == 2) ? (16 * q + (lane & 15)) : (32 * q + lane);
@@ -320,170 +321,163 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     int lim = p.causal ? (p.txt_start + row + 1) : p.L;                        // keys below lim are visible
     lim = (lim < p.L ? lim : p.L) - key_lane0;                                 // ... as a column count of this lane
     const bool all_visible = lim >= p.cpl;
-    const bool writer = (g == 0) && (half == 0);
-    const int part_idx = row * NPART + half * kColGroups + g;
+    const bool sender = (half == 0);           // with two halves, lanes s and s+16 share a row: the lower one sends
+    const uint32_t pair_idx = (rank * NROWS + row) * EPR + g * NBT;            // this thread's first pair in a slot
 
-    float acc[kMaxChunks][kChunk];
+    for (int h = 0; h < p.H; ++h) {
+      const int buf = h % kNumBufs;
+      const uint32_t bph = static_cast<uint32_t>(h / kNumBufs) & 1u;
+      const int slot = h % kStatSlots;
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag))) break;
+      if (threadIdx.x == 0) {
+        MD_TRACE(h, 3);
+        // arm this head's statistics barrier with the bytes all CTAs will send
+        mbar_expect_tx(smem_u32(&bars.sfull[slot]), slot_pairs * 8u);
+      }
+      tc_fence_after();
+      const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
+      const uint32_t slot_addr = smem_u32(&stats[slot * slot_pairs + pair_idx]);
+      const uint32_t bar_addr = smem_u32(&bars.sfull[slot]);
 #pragma unroll
-    for (int t = 0; t < kMaxChunks; ++t)
+      for (int bt = 0; bt < NBT; ++bt) {
+        const int lo = bt == 0 ? 0 : kBatch0;
+        const int hi = bt == 0 ? (ECH < kBatch0 ? ECH : kBatch0) : ECH;
+        float z[kBatch0][kChunk];
 #pragma unroll
-      for (int j = 0; j < kChunk; ++j) acc[t][j] = 0.0f;
-
-    // The thread's chunks are worked in two batches (chunks 0-2 and 3-4), each with its own
-    // stabiliser, to bound the registers that hold logits in flight.
-#define MD_BATCH_LO(bt) ((bt) * 3)
-#define MD_BATCH_HI(bt) ((bt) == 0 ? 3 : kMaxChunks)
-    float m_prev[2] = {-INFINITY, -INFINITY};   // stabilisers of head h-1, per batch
-    // Every decision to give up is taken by the whole warp (votes), so no lane is ever left
-    // alone at a warp-level synchronisation.
-    for (int h = 0; h <= p.H; ++h) {
-      float m_cur[2] = {-INFINITY, -INFINITY};
-      bool bad = false;
-      if (h < p.H) {
-        // ---- exponentials of head h, relative to the batch maximum, back into tensor memory
-        const int buf = h % p.n_buf;
-        const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
-        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag))) break;
-        if (threadIdx.x == 0) MD_TRACE(h, 3);
-        tc_fence_after();
-        const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
-        float m_thr = -INFINITY, l_thr = 0.0f;
+        for (int t = lo; t < hi; ++t)
+          if (t < my_chunks) tc_ld16(tbuf + kChunk * (g + t * kColGroups), z[t - lo]);
+        tc_wait_ld();
+        if (!all_visible) {
 #pragma unroll
-        for (int bt = 0; bt < 2; ++bt) {
-          if (MD_BATCH_LO(bt) < my_chunks) {
-            float z[3][kChunk];
+          for (int t = lo; t < hi; ++t) {
+            const int nvis = lim - kChunk * (g + t * kColGroups);
 #pragma unroll
-            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
-              if (t < my_chunks) tc_ld16(tbuf + kChunk * (g + t * kColGroups), z[t - MD_BATCH_LO(bt)]);
-            tc_wait_ld();
-            if (threadIdx.x == 0) MD_TRACE(h, 8 + bt);
-            if (!all_visible) {
+            for (int j = 0; j < kChunk; ++j) z[t - lo][j] = (j < nvis) ? z[t - lo][j] : -INFINITY;
+          }
+        }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-              for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t) {
-                const int nvis = lim - kChunk * (g + t * kColGroups);
+        for (int t = lo; t < hi; ++t)
+          if (t < my_chunks) {
 #pragma unroll
-                for (int j = 0; j < kChunk; ++j) z[t - MD_BATCH_LO(bt)][j] = (j < nvis) ? z[t - MD_BATCH_LO(bt)][j] : -INFINITY;
-              }
+            for (int j = 0; j < kChunk; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], z[t - lo][j]);
+          }
+        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;   // scale > 0 keeps the order
+        if (HALVES == 2) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));            // one stabiliser per row
+        const float sub = (mx == -INFINITY) ? 0.0f : mx;
+        float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int t = lo; t < hi; ++t)
+          if (t < my_chunks) {
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) {
+              const float e = ex2(fmaf(z[t - lo][j], p.scale_log2e, -sub));
+              z[t - lo][j] = e;
+              ls4[j & 3] += e;
             }
-            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
-              if (t < my_chunks) {
-#pragma unroll
-                for (int j = 0; j < kChunk; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], z[t - MD_BATCH_LO(bt)][j]);
-              }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;  // scale > 0 keeps the order
-            const float sub = (mx == -INFINITY) ? 0.0f : mx;
-            float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
-              if (t < my_chunks) {
-#pragma unroll
-                for (int j = 0; j < kChunk; ++j) {
-                  const float e = ex2(fmaf(z[t - MD_BATCH_LO(bt)][j], p.scale_log2e, -sub));
-                  z[t - MD_BATCH_LO(bt)][j] = e;
-                  ls4[j & 3] += e;
-                }
-                tc_st16(tbuf + kChunk * (g + t * kColGroups), z[t - MD_BATCH_LO(bt)]);
-              }
-            m_cur[bt] = mx;
-            merge_stats(m_thr, l_thr, mx, (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
-            if (threadIdx.x == 0) MD_TRACE(h, 10 + bt);
+            tc_st16(tbuf + kChunk * (g + t * kColGroups), z[t - lo]);
           }
-        }
-        // one thread arms this head's statistics barrier with the bytes all CTAs will send
-        if (threadIdx.x == 0)
-          mbar_expect_tx(smem_u32(&bars.sfull[h % kStatSlots]), static_cast<uint32_t>(p.cluster) * NROWS * 8u);
-        part[(h & 1) * NROWS * NPART + part_idx] = make_float2(m_thr, l_thr);
-        if (threadIdx.x == 0) MD_TRACE(h, 4);
-        mbar_arrive(smem_u32(&bars.pfull));
-        if (writer) {
-          bad = !__all_sync(kWriterLanes, mbar_wait(smem_u32(&bars.pfull), static_cast<uint32_t>(h) & 1u, abort_flag));
-        }
-        if (threadIdx.x == 0) MD_TRACE(h, 12);
-        if (writer && !bad) {
-          float m = -INFINITY, l = 0.0f;
-#pragma unroll
-          for (int x = 0; x < NPART; ++x) {
-            const float2 v = part[(h & 1) * NROWS * NPART + row * NPART + x];
-            merge_stats(m, l, v.x, v.y);
-          }
-          const int slot = h % kStatSlots;
-          const uint32_t slot_addr = smem_u32(&stats[(slot * p.cluster + rank) * NROWS + row]);
-          const uint32_t bar_addr = smem_u32(&bars.sfull[slot]);
-          for (int c = 0; c < p.cluster; ++c) st_async_f32x2(map_to_cta(slot_addr, c), m, l, map_to_cta(bar_addr, c));
+        float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+        if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
+        if (sender) {
+          for (int c = 0; c < p.cluster; ++c)
+            st_async_f32x2(map_to_cta(slot_addr + bt * 8u, c), mx, lsum, map_to_cta(bar_addr, c));
         }
       }
-      if (h >= 1) {
-        // ---- head h-1: normalise with the row statistics of the whole key range, add into the head sum
-        const int hp = h - 1;
-        const int buf = hp % p.n_buf;
-        const int slot = hp % kStatSlots;
-        const uint32_t sph = static_cast<uint32_t>(hp / kStatSlots) & 1u;
-        if (threadIdx.x == 0) MD_TRACE(hp, 5);
-        if (!__all_sync(0xffffffffu, !bad && mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag))) break;
-        if (threadIdx.x == 0) MD_TRACE(hp, 6);
-        float m = -INFINITY, l = 0.0f;
-        for (int c = 0; c < p.cluster; ++c) {
-          const float2 v = stats[(slot * p.cluster + c) * NROWS + row];
-          merge_stats(m, l, v.x, v.y);
-        }
-        const float inv_l = 1.0f / l;
-        const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
-        if (threadIdx.x == 0) MD_TRACE(hp, 13);
-        tc_wait_st();
-        if (threadIdx.x == 0) MD_TRACE(hp, 14);
-#pragma unroll
-        for (int bt = 0; bt < 2; ++bt) {
-          if (MD_BATCH_LO(bt) < my_chunks) {
-            const float f = (m_prev[bt] == -INFINITY) ? 0.0f : ex2(m_prev[bt] - m) * inv_l;
-            float e[3][kChunk];
-#pragma unroll
-            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
-              if (t < my_chunks) tc_ld16(tbuf + kChunk * (g + t * kColGroups), e[t - MD_BATCH_LO(bt)]);
-            tc_wait_ld();
-            if (threadIdx.x == 0 && bt == 0) MD_TRACE(hp, 15);
-#pragma unroll
-            for (int t = MD_BATCH_LO(bt); t < MD_BATCH_HI(bt); ++t)
-              if (t < my_chunks) {
-#pragma unroll
-                for (int j = 0; j < kChunk; ++j) acc[t][j] = fmaf(e[t - MD_BATCH_LO(bt)][j], f, acc[t][j]);
-              }
-          }
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars.tempty[buf]));
-        if (threadIdx.x == 0) MD_TRACE(hp, 7);
-      } else if (__any_sync(0xffffffffu, bad)) {
-        break;
-      }
-      m_prev[0] = m_cur[0];
-      m_prev[1] = m_cur[1];
+      tc_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars.eready[buf]));
+      if (threadIdx.x == 0) MD_TRACE(h, 4);
     }
+  } else {
+    // ---------------- add warps ----------------
+    if (kRealloc) asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+    const int q = warp & 3;
+    const int half = (HALVES == 2) ? (lane >> 4) : 0;
+    const int row = (HALVES == 2) ? (16 * q + (lane & 15)) : (32 * q + lane);
+    const uint32_t lane_addr = static_cast<uint32_t>(32 * q) << 16;
+    const int total_chunks = p.cpl / kChunk;
+    const int tid_a = threadIdx.x - kExpThreads;
 
-#undef MD_BATCH_LO
-#undef MD_BATCH_HI
+    float acc[ACH][kChunk];
+#pragma unroll
+    for (int c = 0; c < ACH; ++c)
+#pragma unroll
+      for (int j = 0; j < kChunk; ++j) acc[c][j] = 0.0f;
+
+    int h = 0;
+    for (; h < p.H; ++h) {
+      const int buf = h % kNumBufs;
+      const uint32_t bph = static_cast<uint32_t>(h / kNumBufs) & 1u;
+      const int slot = h % kStatSlots;
+      const uint32_t sph = static_cast<uint32_t>(h / kStatSlots) & 1u;
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag))) break;
+      if (tid_a == 0) MD_TRACE(h, 5);
+      // statistics of this row over the whole key range: every CTA's pairs
+      const float2* srow = stats + slot * slot_pairs + row * EPR;
+      float m = -INFINITY;
+      for (int c = 0; c < p.cluster; ++c)
+#pragma unroll
+        for (int x = 0; x < EPR; ++x) m = fmaxf(m, srow[c * NROWS * EPR + x].x);
+      float l = 0.0f;
+      for (int c = 0; c < p.cluster; ++c)
+#pragma unroll
+        for (int x = 0; x < EPR; ++x) {
+          const float2 v = srow[c * NROWS * EPR + x];
+          l = fmaf(v.y, ex2(v.x - m), l);     // an empty pair is (-inf, 0): contributes 0
+        }
+      const float inv_l = 1.0f / l;
+      float f[EPR];                            // factor of each of this CTA's pairs
+#pragma unroll
+      for (int x = 0; x < EPR; ++x) f[x] = ex2(srow[rank * NROWS * EPR + x].x - m) * inv_l;
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.eready[buf]), bph, abort_flag))) break;
+      if (tid_a == 0) MD_TRACE(h, 6);
+      tc_fence_after();
+      const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
+#pragma unroll
+      for (int c0 = 0; c0 < ACH; c0 += 2) {
+        if (c0 < total_chunks) {
+          float e[2][kChunk];
+          tc_ld16(tbuf + kChunk * c0, e[0]);
+          if (c0 + 1 < ACH && c0 + 1 < total_chunks) tc_ld16(tbuf + kChunk * (c0 + 1), e[1]);
+          tc_wait_ld();
+          // chunk c belongs to column group c & 1, local index c >> 1, batch (c >> 1) >= kBatch0
+          const float f0 = f[0 * NBT + ((c0 >> 1) >= kBatch0 ? NBT - 1 : 0)];
+          const float f1 = f[1 * NBT + ((c0 >> 1) >= kBatch0 ? NBT - 1 : 0)];
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) acc[c0][j] = fmaf(e[0][j], f0, acc[c0][j]);
+          if (c0 + 1 < ACH && c0 + 1 < total_chunks) {
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) acc[c0 + 1][j] = fmaf(e[1][j], f1, acc[c0 + 1][j]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars.tempty[buf]));
+      if (tid_a == 0) MD_TRACE(h, 7);
+    }
 
     // head mean -> column sum (Eq. 8) and column max (Eq. 10) over the text rows
     mbar_arrive(smem_u32(&bars.fin));
-    if (mbar_wait(smem_u32(&bars.fin), 0u, abort_flag)) {
+    if (__all_sync(0xffffffffu, h == p.H && mbar_wait(smem_u32(&bars.fin), 0u, abort_flag))) {
       // all TMA copies have landed and all MMAs have read them: the staging area is free
       float* mat = reinterpret_cast<float*>(stage_ptr);
       const int ld = p.tk | 1;
       if (row < p.N) {
 #pragma unroll
-        for (int t = 0; t < kMaxChunks; ++t) {
-          if (t < my_chunks) {
-            const int key_local = half * p.cpl + kChunk * (g + t * kColGroups);
+        for (int c = 0; c < ACH; ++c) {
+          if (c < total_chunks) {
+            const int key_local = half * p.cpl + kChunk * c;
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) mat[row * ld + key_local + j] = acc[t][j];
+            for (int j = 0; j < kChunk; ++j) mat[row * ld + key_local + j] = acc[c][j];
           }
         }
       }
       mbar_arrive(smem_u32(&bars.fin));
       const bool staged = mbar_wait(smem_u32(&bars.fin), 1u, abort_flag);
-      for (int c = threadIdx.x; staged && c < p.tk; c += kSoftmaxThreads) {
+      for (int c = tid_a; staged && c < p.tk; c += kAddThreads) {
         const int j = static_cast<int>(rank) * p.tk + c - p.vis_start;   // vision-relative index
         if (j < 0 || j >= p.M) continue;
         float s = 0.0f, mx = -INFINITY;
@@ -546,7 +540,7 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t d1, uint64_t d2, uint
 bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out) {
   const int halves = r.N <= 64 ? 2 : 1;
   const int nrows = 128 / halves;
-  const int max_cpl = kMaxChunks * kChunk * kColGroups;   // 160 columns per TMEM lane
+  const int max_cpl = 10 * kChunk;   // 160 columns per TMEM lane (add threads with 10 chunks)
   double best = -1.0;
   FusedGeometry g{};
   for (int c = 1; c <= kMaxCluster; ++c) {
@@ -557,15 +551,15 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     if (cpl > max_cpl) continue;
     const int tk = cpl * halves;
     const size_t stage = static_cast<size_t>(nrows + tk) * 256;
-    // row statistics (kStatSlots x cluster x rows) and per-thread partials (2 x rows x threads per row), 8 bytes each
-    const size_t extra = static_cast<size_t>(kStatSlots) * c * nrows * 8 + 2 * static_cast<size_t>(nrows) * halves * kColGroups * 8;
-    const size_t budget = 227 * 1024 - 2048 /* static */ - 1024 /* alignment */ - extra;
+    const int ach = cpl <= 5 * kChunk ? 5 : 10;             // chunks per add thread (kernel variant)
+    const int epr = kColGroups * (ach > 5 ? 2 : 1);         // (max, sum) pairs per row and CTA
+    // statistics slots: kStatSlots x cluster x rows x pairs, 8 bytes each
+    const size_t extra = static_cast<size_t>(kStatSlots) * c * nrows * epr * 8;
+    const size_t budget = 227 * 1024 - 1024 /* static */ - 1024 /* alignment */ - extra;
     int n_stage = static_cast<int>(budget / stage);
     if (n_stage < 2) continue;
     if (n_stage > kMaxStages) n_stage = kMaxStages;
-    int n_buf = kTmemCols / cpl;
-    if (n_buf > kMaxBufs) n_buf = kMaxBufs;
-    if (n_buf < 3) continue;   // logits of head h+1, exponentials of heads h and h-1
+    if (kNumBufs * cpl > kTmemCols) continue;
     const long ctas = static_cast<long>(r.B) * c;
     const long waves = (ctas + sm_count - 1) / sm_count;
     const double fill = static_cast<double>(ctas) / static_cast<double>(waves * sm_count);
@@ -573,7 +567,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     const double score = fill * useful - 0.002 * c;   // prefer smaller clusters among equals
     if (score > best) {
       best = score;
-      g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_stage = n_stage; g.n_buf = n_buf;
+      g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_stage = n_stage; g.n_buf = kNumBufs; g.ach = ach;
       // at least 116 KB, so that two CTAs (each wanting all of tensor memory) never share an SM
       g.smem_bytes = stage * n_stage + 1024 + extra;
       if (g.smem_bytes < 116 * 1024) g.smem_bytes = 116 * 1024;
@@ -599,11 +593,12 @@ cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, co
   p.g_out = g_out; p.i_out = i_out; p.workspace = workspace;
   p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
   p.causal = r.causal;
-  p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_stage = geo.n_stage; p.n_buf = geo.n_buf;
+  p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_stage = geo.n_stage;
   p.scale_log2e = r.scale_log2e;
   p.inv_heads = 1.0f / static_cast<float>(r.H);
 
-  auto kernel = geo.halves == 2 ? score_fused_kernel<2> : score_fused_kernel<1>;
+  auto kernel = geo.halves == 2 ? (geo.ach > 5 ? score_fused_kernel<2, 10> : score_fused_kernel<2, 5>)
+                                : (geo.ach > 5 ? score_fused_kernel<1, 10> : score_fused_kernel<1, 5>);
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(geo.smem_bytes));
   if (e != cudaSuccess) return e;
