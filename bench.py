@@ -224,15 +224,26 @@ def run_ours(args, w):
         step()
     torch.cuda.synchronize()
 
-    # timed region: exactly K steps; events around every call give the per-call durations
+    # timed region: exactly K steps between two events on the launching stream.  No events are
+    # recorded inside it, so the kernels' programmatic dependent launches overlap as in real use.
     K = args.steps
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     t_begin.record(stream)
+    for s in range(K):
+        step()
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    elapsed_ms = t_begin.elapsed_time(t_end)
+
+    # per-call durations for the roofline: a second pass over the same K steps with an event
+    # around every call (the events serialise the calls, so these add up to more than a step)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
     for s in range(K):
         ev[s][0].record(stream)
         f.score(d_q, d_k, stream)
@@ -241,11 +252,7 @@ def run_ours(args, w):
         ev[s][2].record(stream)
         f.compact(d_hid, d_k, d_v, stream=stream)
         ev[s][3].record(stream)
-    t_end.record(stream)
     torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    elapsed_ms = t_begin.elapsed_time(t_end)
     t_score = statistics.mean(ev[s][0].elapsed_time(ev[s][1]) for s in range(K))
     t_select = statistics.mean(ev[s][1].elapsed_time(ev[s][2]) for s in range(K))
     t_compact = statistics.mean(ev[s][2].elapsed_time(ev[s][3]) for s in range(K))
@@ -318,7 +325,8 @@ def run_ours(args, w):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bm["h2d"], "d2h_bytes_per_step": bm["d2h"],
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": launches_per_step * K,
-            "kernel_ms": {"score": t_score, "select": t_select, "compact": t_compact},
+            "kernel_ms": {"score": t_score, "select": t_select, "compact": t_compact,
+                          "how": "second pass over the same steps with an event around every call"},
             "hbm_headline": {"bytes_per_step": bm["headline"], "gbs": bm["headline"] / (ms_per_step / 1e3) / 1e9,
                              "frac_of_peak": bm["headline"] / (ms_per_step / 1e3) / 1e9 / peak, "peak_kind": peak_kind},
             "roofline": {"kernel": "score (%s)" % f.score_variant, "bound": "hbm", "achieved": achieved, "peak": peak,

@@ -39,6 +39,8 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
 
 __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams p) {
   const int r = blockIdx.x, b = blockIdx.y, which = blockIdx.z;
+  pdl_launch_dependents();
+  pdl_wait();   // kept_idx / kept_cnt come from the previous kernel in the stream
   if (p.src[which] == nullptr) return;
   if (r >= p.kept_cnt[b]) return;
   const int j = p.kept_idx[static_cast<size_t>(b) * p.cap + r];
@@ -104,8 +106,7 @@ cudaError_t launch_compact(const mustdrop_plan& plan, const int32_t* kept_idx, c
   p.k_sb = r.k_sb / 8; p.k_sh = r.k_sh / 8; p.k_sl = r.k_sl / 8;
   p.v_sb = r.v_sb / 8; p.v_sh = r.v_sh / 8; p.v_sl = r.v_sl / 8;
   dim3 grid(r.cap, r.B, 3);
-  compact_kernel<<<grid, kCompactThreads, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(compact_kernel, grid, dim3(kCompactThreads), 0, stream, p);
 }
 
 }  // namespace mustdrop

@@ -75,6 +75,28 @@ cudaError_t launch_compact(const mustdrop_plan& p, const int32_t* kept_idx, cons
 // Remember the cudaError_t of a failed runtime call for mustdrop_last_cuda_error (per thread).
 void set_last_cuda_error(cudaError_t e);
 
+// Programmatic dependent launch.  Every kernel of the library is launched with the
+// programmatic-stream-serialization attribute: it may start while its predecessor in the stream
+// is still running, does work that touches no global data, and then calls pdl_wait(), which
+// returns once the predecessor grids have completed and their writes are visible.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename Kernel, typename... Args>
+inline cudaError_t launch_pdl(Kernel kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // Device-side helper: record the first device-detected condition (never traps).
 __device__ __forceinline__ void record_status(void* workspace, int32_t code, int32_t detail) {
   if (workspace == nullptr) return;

@@ -243,6 +243,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   __syncthreads();
   cluster_sync_all();   // every CTA's barriers are initialised before any remote store counts on them
   tc_fence_after();
+  // Up to here nothing touched global memory.  Let the next kernel in the stream begin its own
+  // prologue, then wait for the previous kernels (which may still read g_out / i_out).
+  pdl_launch_dependents();
+  pdl_wait();
   const uint32_t tmem_base = tmem_base_holder;
 
   if (warp >= kTmaWarp) {
@@ -607,13 +611,15 @@ cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, co
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = geo.smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = static_cast<unsigned>(geo.cluster);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, q_map, k_map, p);
 }
 

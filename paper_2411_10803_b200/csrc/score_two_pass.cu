@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(256) rowstats_kernel(ScoreParams p) {
   const int h = blockIdx.x, b = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int n_threads = blockDim.x;
+  pdl_wait();   // the row-statistics scratch may still be read by an earlier launch
   const __nv_bfloat16* qg = p.q + (static_cast<int64_t>(b) * p.H + h) * p.N * kHeadDim;
   const __nv_bfloat16* kg = p.k + b * p.k_sb + h * p.k_sh;
   const int n_tiles = (p.L + kTileKeys - 1) / kTileKeys;
@@ -186,6 +187,7 @@ __global__ void __launch_bounds__(256) accumulate_kernel(ScoreParams p) {
   const int vt = blockIdx.x, b = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int n_threads = blockDim.x;
+  pdl_wait();
   const int j_base = vt * kTileKeys;            // first vision token of this tile
   const int valid_keys = p.M - j_base;          // rows of the tile that exist
   const __nv_bfloat16* qg = p.q + static_cast<int64_t>(b) * p.H * p.N * kHeadDim;

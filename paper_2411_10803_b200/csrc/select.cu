@@ -64,10 +64,16 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
   __shared__ double s_dsum[kSelWarps];
   __shared__ int s_warp[kSelWarps];
   __shared__ int s_pick[2];
+  __shared__ int s_wsuf[kSelWarps];
+  static_assert(kSelThreads == 256, "one thread per radix bin");
 
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int M = p.M;
+  // Programmatic dependent launch: let the next kernel start its prologue, then wait until the
+  // kernel that produced g / i has finished and its writes are visible.
+  pdl_launch_dependents();
+  pdl_wait();
   const float* g = p.g + static_cast<size_t>(b) * M;
   const float* in = p.i + static_cast<size_t>(b) * M;
 
@@ -141,11 +147,22 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
           if (!(s_flag[j] & 1) && (u & mask) == prefix) atomicAdd(&s_hist[(u >> shift) & 255u], 1);
         }
         __syncthreads();
-        // digit d is the cut iff (#candidates with a larger digit) < remaining <= that + hist[d]
-        if (tid < 256) {
-          int above = 0;
-          for (int e = tid + 1; e < 256; ++e) above += s_hist[e];
+        // digit d is the cut iff (#candidates with a larger digit) < remaining <= that + hist[d];
+        // thread d owns bin d: suffix sums by warp shuffles, then across the eight warps
+        {
           const int here = s_hist[tid];
+          int suf = here;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_down_sync(0xffffffffu, suf, d);
+            if (lane + d < 32) suf += t;
+          }
+          if (lane == 0) s_wsuf[warp] = suf;
+          __syncthreads();
+          int above = suf - here;
+#pragma unroll
+          for (int w = 0; w < kSelWarps; ++w)
+            if (w > warp) above += s_wsuf[w];
           if (above < remaining && remaining <= above + here) {
             s_pick[0] = tid;
             s_pick[1] = remaining - above;
@@ -214,8 +231,7 @@ cudaError_t launch_select(const mustdrop_plan& plan, const float* g, const float
   p.s_out = s_out; p.workspace = workspace;
   p.M = r.M; p.key_max = r.key_max; p.mode = r.mode; p.criteria = r.criteria; p.budget = r.budget; p.cap = r.cap;
   p.gamma = r.gamma; p.alpha = r.alpha;
-  select_kernel<<<r.B, kSelThreads, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(select_kernel, dim3(r.B), dim3(kSelThreads), 0, stream, p);
 }
 
 }  // namespace mustdrop
