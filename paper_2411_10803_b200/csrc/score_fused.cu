@@ -243,10 +243,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   __syncthreads();
   cluster_sync_all();   // every CTA's barriers are initialised before any remote store counts on them
   tc_fence_after();
-  // Up to here nothing touched global memory.  Let the next kernel in the stream begin its own
-  // prologue, then wait for the previous kernels (which may still read g_out / i_out).
+  // Let the next kernel in the stream begin its prologue.  This kernel only reads q_text and k,
+  // which no kernel of the library writes, so it does not wait for its predecessors here; the add
+  // warps wait just before they store g_out / i_out, which an earlier select may still be reading.
   pdl_launch_dependents();
-  pdl_wait();
   const uint32_t tmem_base = tmem_base_holder;
 
   if (warp >= kTmaWarp) {
@@ -481,6 +481,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       }
       mbar_arrive(smem_u32(&bars.fin));
       const bool staged = mbar_wait(smem_u32(&bars.fin), 1u, abort_flag);
+      pdl_wait();
       for (int c = tid_a; staged && c < p.tk; c += kAddThreads) {
         const int j = static_cast<int>(rank) * p.tk + c - p.vis_start;   // vision-relative index
         if (j < 0 || j >= p.M) continue;

@@ -5,6 +5,9 @@
 // radix select over the order-preserving integer image of the score, followed by an
 // index-ordered emit, so kept indices come out ascending and equal scores resolve to the
 // lower index.
+//
+// Every thread owns a run of consecutive tokens and keeps their scores in registers; shared
+// memory only holds the key-set bitmap, one 256-bin histogram and a few per-warp partials.
 #include "mustdrop_internal.h"
 
 namespace mustdrop {
@@ -12,7 +15,7 @@ namespace {
 
 constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kChunk = kMaxVis / kSelThreads;  // 16 consecutive tokens per thread in the ordered passes
+constexpr int kOwn = kMaxVis / kSelThreads;  // at most 16 consecutive tokens per thread
 
 // Larger float <=> larger unsigned image (handles negative values and -0 as well).
 __device__ __forceinline__ uint32_t ordered_bits(float f) {
@@ -21,7 +24,7 @@ __device__ __forceinline__ uint32_t ordered_bits(float f) {
 }
 
 // Exclusive prefix sum of one int per thread over the block; also returns the block total.
-// Fixed order, so results never depend on scheduling.
+// Fixed order, so results never depend on scheduling.  Uses two barriers.
 __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums /*[kSelWarps]*/, int* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int inc = v;
@@ -58,162 +61,183 @@ struct SelectParams {
 };
 
 __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
-  __shared__ uint32_t s_bits[kMaxVis];      // ordered image of the score
-  __shared__ uint8_t s_flag[kMaxVis];       // bit0: in key set, bit1: keep
+  __shared__ uint32_t s_key[kMaxVis / 32];  // key-set bitmap
   __shared__ int s_hist[256];
   __shared__ double s_dsum[kSelWarps];
   __shared__ int s_warp[kSelWarps];
-  __shared__ int s_pick[2];
   __shared__ int s_wsuf[kSelWarps];
+  __shared__ int s_pick[2];
   static_assert(kSelThreads == 256, "one thread per radix bin");
 
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int M = p.M;
-  // Programmatic dependent launch: let the next kernel start its prologue, then wait until the
-  // kernel that produced g / i has finished and its writes are visible.
+  const int own = (M + kSelThreads - 1) / kSelThreads;   // tokens per thread (<= kOwn)
+  const int j0 = tid * own;                              // this thread's first token
+
+  // Work that touches no global data, then let the next kernel start its prologue and wait for
+  // the kernel that produced g / i.
+  for (int w = tid; w < kMaxVis / 32; w += kSelThreads) s_key[w] = 0u;
+  s_hist[tid] = 0;
   pdl_launch_dependents();
   pdl_wait();
+
   const float* g = p.g + static_cast<size_t>(b) * M;
   const float* in = p.i + static_cast<size_t>(b) * M;
-
-  // T = sum_j g[j] in double; thread-strided partial sums, then a fixed shuffle tree.
+  float gv[kOwn], iv[kOwn];
   double part = 0.0;
-  for (int j = tid; j < M; j += kSelThreads) part += static_cast<double>(g[j]);
+#pragma unroll
+  for (int e = 0; e < kOwn; ++e) {
+    const int j = j0 + e;
+    const bool ok = e < own && j < M;
+    gv[e] = ok ? g[j] : 0.0f;
+    iv[e] = ok ? in[j] : 0.0f;
+    part += static_cast<double>(gv[e]);
+  }
+  // T = sum_j g[j] in double: per-thread runs, then a fixed shuffle tree, then the eight warps in order
 #pragma unroll
   for (int d = 16; d >= 1; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
   if (lane == 0) s_dsum[warp] = part;
-  for (int j = tid; j < M; j += kSelThreads) s_flag[j] = 0;
-  __syncthreads();
+  __syncthreads();   // also orders the bitmap clear before the key marks below
+  // key set: mark distinct in-range indices
+  if (p.key_max > 0) {
+    int c = p.key_cnt[b];
+    c = c < p.key_max ? c : p.key_max;
+    for (int t = tid; t < c; t += kSelThreads) {
+      const int j = p.key_idx[static_cast<size_t>(b) * p.key_max + t];
+      if (j >= 0 && j < M) atomicOr(&s_key[j >> 5], 1u << (j & 31));
+      else record_status(p.workspace, MUSTDROP_ERR_BAD_KEY_INDEX, b * 65536 + t);
+    }
+  }
   double tsum = 0.0;
 #pragma unroll
   for (int w = 0; w < kSelWarps; ++w) tsum += s_dsum[w];
   const float T = static_cast<float>(tsum);
   const float gt = __fmul_rn(p.gamma, T);
 
-  // key set: mark distinct in-range indices
-  if (p.key_max > 0) {
-    int c = p.key_cnt[b];
-    c = c < p.key_max ? c : p.key_max;
-    for (int t = tid; t < c; t += kSelThreads) {
-      int j = p.key_idx[static_cast<size_t>(b) * p.key_max + t];
-      if (j >= 0 && j < M) s_flag[j] = 1;
-      else record_status(p.workspace, MUSTDROP_ERR_BAD_KEY_INDEX, b * 65536 + t);
+  // scores of the thread's tokens, as ordered integers
+  uint32_t u[kOwn];
+#pragma unroll
+  for (int e = 0; e < kOwn; ++e) {
+    const int j = j0 + e;
+    u[e] = 0u;
+    if (e < own && j < M) {
+      const float gj = __fdiv_rn(gv[e], gt);
+      const float rj = __fdiv_rn(iv[e], p.alpha);
+      float s;
+      if (p.criteria == MUSTDROP_CRIT_GLOBAL_ONLY) s = gj;
+      else if (p.criteria == MUSTDROP_CRIT_INDIVIDUAL_ONLY) s = rj;
+      else s = (gj > rj) ? gj : rj;
+      u[e] = ordered_bits(s);
+      if (p.s_out != nullptr) p.s_out[static_cast<size_t>(b) * M + j] = s;
     }
   }
-  // scores
-  for (int j = tid; j < M; j += kSelThreads) {
-    const float gj = __fdiv_rn(g[j], gt);
-    const float rj = __fdiv_rn(in[j], p.alpha);
-    float s;
-    if (p.criteria == MUSTDROP_CRIT_GLOBAL_ONLY) s = gj;
-    else if (p.criteria == MUSTDROP_CRIT_INDIVIDUAL_ONLY) s = rj;
-    else s = (gj > rj) ? gj : rj;
-    s_bits[j] = ordered_bits(s);
-    if (p.s_out != nullptr) p.s_out[static_cast<size_t>(b) * M + j] = s;
-  }
-  __syncthreads();
+  __syncthreads();   // key marks complete
 
-  const int j0 = tid * kChunk;  // this thread's run of consecutive tokens in the ordered passes
+  // per-token bits: bit e of `valid` = token exists, of `key` = in the key set, of `keep` = retained
+  uint32_t valid = 0u, key = 0u, keep = 0u;
+#pragma unroll
+  for (int e = 0; e < kOwn; ++e) {
+    const int j = j0 + e;
+    if (e < own && j < M) {
+      valid |= 1u << e;
+      if ((s_key[j >> 5] >> (j & 31)) & 1u) key |= 1u << e;
+    }
+  }
+  const uint32_t cand = valid & ~key;
 
   if (p.mode == MUSTDROP_MODE_THRESHOLD) {
-    for (int j = tid; j < M; j += kSelThreads) {
-      const bool in_d = g[j] <= gt;            // Eq. 9
-      const bool small = in[j] < p.alpha;      // Eq. 10
-      bool drop;
-      if (p.criteria == MUSTDROP_CRIT_GLOBAL_ONLY) drop = in_d;
-      else if (p.criteria == MUSTDROP_CRIT_INDIVIDUAL_ONLY) drop = small;
-      else drop = in_d && small;
-      if ((s_flag[j] & 1) || !drop) s_flag[j] |= 2;
+#pragma unroll
+    for (int e = 0; e < kOwn; ++e) {
+      if ((valid >> e) & 1u) {
+        const bool in_d = gv[e] <= gt;            // Eq. 9
+        const bool small = iv[e] < p.alpha;       // Eq. 10
+        bool drop;
+        if (p.criteria == MUSTDROP_CRIT_GLOBAL_ONLY) drop = in_d;
+        else if (p.criteria == MUSTDROP_CRIT_INDIVIDUAL_ONLY) drop = small;
+        else drop = in_d && small;
+        if (!drop) keep |= 1u << e;
+      }
     }
+    keep |= key;
   } else {
-    // number of distinct keys
-    int nk = 0;
-    for (int j = tid; j < M; j += kSelThreads) nk += (s_flag[j] & 1);
     int n_key;
-    (void)block_exclusive_scan(nk, s_warp, &n_key);
+    (void)block_exclusive_scan(__popc(key), s_warp, &n_key);
     int want = p.budget - n_key;
     const int n_cand = M - n_key;
     want = want < n_cand ? want : n_cand;
+    keep = key;
     if (want > 0) {
       // radix select of the want-th largest candidate: four 8-bit digits from the top
       uint32_t prefix = 0, mask = 0;
       int remaining = want;
       for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int t = tid; t < 256; t += kSelThreads) s_hist[t] = 0;
-        __syncthreads();
-        for (int j = tid; j < M; j += kSelThreads) {
-          const uint32_t u = s_bits[j];
-          if (!(s_flag[j] & 1) && (u & mask) == prefix) atomicAdd(&s_hist[(u >> shift) & 255u], 1);
+        // Scores crowd into a few bins (same exponent), so lanes with the same digit elect one
+        // leader that adds their count: one shared-memory atomic per distinct digit and warp.
+#pragma unroll
+        for (int e = 0; e < kOwn; ++e) {
+          if (e < own) {   // uniform over the block
+            const bool act = ((cand >> e) & 1u) && (u[e] & mask) == prefix;
+            const uint32_t digit = (u[e] >> shift) & 255u;
+            const uint32_t peers = __match_any_sync(0xffffffffu, act ? digit : 256u + lane);
+            if (act && lane == __ffs(peers) - 1) atomicAdd(&s_hist[digit], __popc(peers));
+          }
         }
         __syncthreads();
         // digit d is the cut iff (#candidates with a larger digit) < remaining <= that + hist[d];
         // thread d owns bin d: suffix sums by warp shuffles, then across the eight warps
-        {
-          const int here = s_hist[tid];
-          int suf = here;
+        const int here = s_hist[tid];
+        s_hist[tid] = 0;   // ready for the next digit
+        int suf = here;
 #pragma unroll
-          for (int d = 1; d < 32; d <<= 1) {
-            const int t = __shfl_down_sync(0xffffffffu, suf, d);
-            if (lane + d < 32) suf += t;
-          }
-          if (lane == 0) s_wsuf[warp] = suf;
-          __syncthreads();
-          int above = suf - here;
+        for (int d = 1; d < 32; d <<= 1) {
+          const int t = __shfl_down_sync(0xffffffffu, suf, d);
+          if (lane + d < 32) suf += t;
+        }
+        if (lane == 0) s_wsuf[warp] = suf;
+        __syncthreads();
+        int above = suf - here;
 #pragma unroll
-          for (int w = 0; w < kSelWarps; ++w)
-            if (w > warp) above += s_wsuf[w];
-          if (above < remaining && remaining <= above + here) {
-            s_pick[0] = tid;
-            s_pick[1] = remaining - above;
-          }
+        for (int w = 0; w < kSelWarps; ++w)
+          if (w > warp) above += s_wsuf[w];
+        if (above < remaining && remaining <= above + here) {
+          s_pick[0] = tid;
+          s_pick[1] = remaining - above;
         }
         __syncthreads();
         prefix |= static_cast<uint32_t>(s_pick[0]) << shift;
         mask |= 255u << shift;
         remaining = s_pick[1];
-        __syncthreads();
       }
       // prefix is now the cut value; `remaining` tokens equal to it are taken, lowest index first
-      int eq = 0;
-      for (int t = 0; t < kChunk; ++t) {
-        const int j = j0 + t;
-        if (j < M && !(s_flag[j] & 1) && s_bits[j] == prefix) ++eq;
+      uint32_t eq = 0u;
+#pragma unroll
+      for (int e = 0; e < kOwn; ++e) {
+        if ((cand >> e) & 1u) {
+          if (u[e] > prefix) keep |= 1u << e;
+          else if (u[e] == prefix) eq |= 1u << e;
+        }
       }
       int eq_total;
-      int eq_rank = block_exclusive_scan(eq, s_warp, &eq_total);
-      for (int t = 0; t < kChunk; ++t) {
-        const int j = j0 + t;
-        if (j >= M) break;
-        const uint8_t f = s_flag[j];
-        if (f & 1) continue;
-        const uint32_t u = s_bits[j];
-        if (u > prefix) s_flag[j] = f | 2;
-        else if (u == prefix) {
-          if (eq_rank < remaining) s_flag[j] = f | 2;
+      int eq_rank = block_exclusive_scan(__popc(eq), s_warp, &eq_total);
+#pragma unroll
+      for (int e = 0; e < kOwn; ++e) {
+        if ((eq >> e) & 1u) {
+          if (eq_rank < remaining) keep |= 1u << e;
           ++eq_rank;
         }
       }
     }
-    __syncthreads();
-    for (int j = tid; j < M; j += kSelThreads)
-      if (s_flag[j] & 1) s_flag[j] |= 2;
   }
-  __syncthreads();
 
   // index-ordered emit
-  int cnt = 0;
-  for (int t = 0; t < kChunk; ++t) {
-    const int j = j0 + t;
-    if (j < M && (s_flag[j] & 2)) ++cnt;
-  }
   int total;
-  int pos = block_exclusive_scan(cnt, s_warp, &total);
+  int pos = block_exclusive_scan(__popc(keep), s_warp, &total);
   int32_t* out = p.kept_idx + static_cast<size_t>(b) * p.cap;
-  for (int t = 0; t < kChunk; ++t) {
-    const int j = j0 + t;
-    if (j < M && (s_flag[j] & 2)) {
-      if (pos < p.cap) out[pos] = j;
+#pragma unroll
+  for (int e = 0; e < kOwn; ++e) {
+    if ((keep >> e) & 1u) {
+      if (pos < p.cap) out[pos] = j0 + e;
       ++pos;
     }
   }
