@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kOwn = kMaxVis / kSelThreads;  // at most 16 consecutive tokens per thread
+constexpr int kMaxOwn = kMaxVis / kSelThreads;  // at most 16 consecutive tokens per thread
 
 // Larger float <=> larger unsigned image (handles negative values and -0 as well).
 __device__ __forceinline__ uint32_t ordered_bits(float f) {
@@ -25,7 +25,7 @@ __device__ __forceinline__ uint32_t ordered_bits(float f) {
 
 // Exclusive prefix sum of one int per thread over the block; also returns the block total.
 // Fixed order, so results never depend on scheduling.  Uses two barriers.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums /*[kSelWarps]*/, int* total) {
+__device__ __noinline__ int block_exclusive_scan(int v, int* warp_sums /*[kSelWarps]*/, int* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int inc = v;
 #pragma unroll
@@ -60,7 +60,10 @@ struct SelectParams {
   float gamma, alpha;
 };
 
+// OWN: consecutive tokens per thread (1, 2, 4, 8 or 16; OWN * 256 >= M).
+template <int OWN>
 __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
+  constexpr int kOwn = OWN;
   __shared__ uint32_t s_key[kMaxVis / 32];  // key-set bitmap
   __shared__ int s_hist[256];
   __shared__ double s_dsum[kSelWarps];
@@ -72,7 +75,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int M = p.M;
-  const int own = (M + kSelThreads - 1) / kSelThreads;   // tokens per thread (<= kOwn)
+  constexpr int own = OWN;
   const int j0 = tid * own;                              // this thread's first token
 
   // Work that touches no global data, then let the next kernel start its prologue and wait for
@@ -171,6 +174,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
       // radix select of the want-th largest candidate: four 8-bit digits from the top
       uint32_t prefix = 0, mask = 0;
       int remaining = want;
+      // (kept as a real loop: the kernel runs once per launch from a cold instruction cache, so
+      // code size, not instruction count, sets its latency)
+#pragma unroll 1
       for (int shift = 24; shift >= 0; shift -= 8) {
         // Scores crowd into a few bins (same exponent), so lanes with the same digit elect one
         // leader that adds their count: one shared-memory atomic per distinct digit and warp.
@@ -255,7 +261,13 @@ cudaError_t launch_select(const mustdrop_plan& plan, const float* g, const float
   p.s_out = s_out; p.workspace = workspace;
   p.M = r.M; p.key_max = r.key_max; p.mode = r.mode; p.criteria = r.criteria; p.budget = r.budget; p.cap = r.cap;
   p.gamma = r.gamma; p.alpha = r.alpha;
-  return launch_pdl(select_kernel, dim3(r.B), dim3(kSelThreads), 0, stream, p);
+  const int own = (r.M + kSelThreads - 1) / kSelThreads;
+  static_assert(kMaxOwn == 16, "dispatch below covers up to 16 tokens per thread");
+  if (own <= 1) return launch_pdl(select_kernel<1>, dim3(r.B), dim3(kSelThreads), 0, stream, p);
+  if (own <= 2) return launch_pdl(select_kernel<2>, dim3(r.B), dim3(kSelThreads), 0, stream, p);
+  if (own <= 4) return launch_pdl(select_kernel<4>, dim3(r.B), dim3(kSelThreads), 0, stream, p);
+  if (own <= 8) return launch_pdl(select_kernel<8>, dim3(r.B), dim3(kSelThreads), 0, stream, p);
+  return launch_pdl(select_kernel<16>, dim3(r.B), dim3(kSelThreads), 0, stream, p);
 }
 
 }  // namespace mustdrop
