@@ -47,6 +47,13 @@ __device__ __noinline__ int block_exclusive_scan(int v, int* warp_sums /*[kSelWa
   return base + inc - v;
 }
 
+#ifdef MUSTDROP_TRACE
+#define SEL_STAMP(ev) do { if (threadIdx.x == 0 && blockIdx.x == 0 && p.workspace) { \
+  reinterpret_cast<long long*>(static_cast<unsigned char*>(p.workspace) + 2048)[ev] = clock64(); } } while (0)
+#else
+#define SEL_STAMP(ev) ((void)0)
+#endif
+
 struct SelectParams {
   const float* g;
   const float* i;
@@ -69,7 +76,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
   __shared__ double s_dsum[kSelWarps];
   __shared__ int s_warp[kSelWarps];
   __shared__ int s_wsuf[kSelWarps];
-  __shared__ int s_pick[2];
+  __shared__ int s_pick[3];
+  __shared__ int s_nkey;
   static_assert(kSelThreads == 256, "one thread per radix bin");
 
   const int b = blockIdx.x;
@@ -80,13 +88,22 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
 
   // Work that touches no global data, then let the next kernel start its prologue and wait for
   // the kernel that produced g / i.
+  SEL_STAMP(0);
   for (int w = tid; w < kMaxVis / 32; w += kSelThreads) s_key[w] = 0u;
   s_hist[tid] = 0;
+  if (tid == 0) s_nkey = 0;
   pdl_launch_dependents();
   pdl_wait();
+  SEL_STAMP(1);
 
   const float* g = p.g + static_cast<size_t>(b) * M;
   const float* in = p.i + static_cast<size_t>(b) * M;
+  // the key-set loads are issued first so that their latency overlaps the score loads
+  int key_c = 0, key_j = -1;
+  if (p.key_max > 0) {
+    key_c = p.key_cnt[b];
+    if (tid < p.key_max) key_j = p.key_idx[static_cast<size_t>(b) * p.key_max + tid];
+  }
   float gv[kOwn], iv[kOwn];
   double part = 0.0;
 #pragma unroll
@@ -101,15 +118,20 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
 #pragma unroll
   for (int d = 16; d >= 1; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
   if (lane == 0) s_dsum[warp] = part;
+  SEL_STAMP(2);
   __syncthreads();   // also orders the bitmap clear before the key marks below
+  SEL_STAMP(3);
   // key set: mark distinct in-range indices
   if (p.key_max > 0) {
-    int c = p.key_cnt[b];
-    c = c < p.key_max ? c : p.key_max;
+    const int c = key_c < p.key_max ? key_c : p.key_max;
     for (int t = tid; t < c; t += kSelThreads) {
-      const int j = p.key_idx[static_cast<size_t>(b) * p.key_max + t];
-      if (j >= 0 && j < M) atomicOr(&s_key[j >> 5], 1u << (j & 31));
-      else record_status(p.workspace, MUSTDROP_ERR_BAD_KEY_INDEX, b * 65536 + t);
+      const int j = t == tid ? key_j : p.key_idx[static_cast<size_t>(b) * p.key_max + t];
+      if (j >= 0 && j < M) {
+        const uint32_t bit = 1u << (j & 31);
+        if (!(atomicOr(&s_key[j >> 5], bit) & bit)) atomicAdd(&s_nkey, 1);   // count distinct keys
+      } else {
+        record_status(p.workspace, MUSTDROP_ERR_BAD_KEY_INDEX, b * 65536 + t);
+      }
     }
   }
   double tsum = 0.0;
@@ -135,7 +157,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
       if (p.s_out != nullptr) p.s_out[static_cast<size_t>(b) * M + j] = s;
     }
   }
+  SEL_STAMP(4);
   __syncthreads();   // key marks complete
+  SEL_STAMP(5);
 
   // per-token bits: bit e of `valid` = token exists, of `key` = in the key set, of `keep` = retained
   uint32_t valid = 0u, key = 0u, keep = 0u;
@@ -164,8 +188,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
     }
     keep |= key;
   } else {
-    int n_key;
-    (void)block_exclusive_scan(__popc(key), s_warp, &n_key);
+    const int n_key = s_nkey;
+    SEL_STAMP(6);
     int want = p.budget - n_key;
     const int n_cand = M - n_key;
     want = want < n_cand ? want : n_cand;
@@ -178,18 +202,14 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
       // code size, not instruction count, sets its latency)
 #pragma unroll 1
       for (int shift = 24; shift >= 0; shift -= 8) {
-        // Scores crowd into a few bins (same exponent), so lanes with the same digit elect one
-        // leader that adds their count: one shared-memory atomic per distinct digit and warp.
 #pragma unroll
         for (int e = 0; e < kOwn; ++e) {
-          if (e < own) {   // uniform over the block
-            const bool act = ((cand >> e) & 1u) && (u[e] & mask) == prefix;
-            const uint32_t digit = (u[e] >> shift) & 255u;
-            const uint32_t peers = __match_any_sync(0xffffffffu, act ? digit : 256u + lane);
-            if (act && lane == __ffs(peers) - 1) atomicAdd(&s_hist[digit], __popc(peers));
-          }
+          const bool act = ((cand >> e) & 1u) && (u[e] & mask) == prefix;
+          if (act) atomicAdd(&s_hist[(u[e] >> shift) & 255u], 1);
         }
+        if (shift == 16) SEL_STAMP(13);
         __syncthreads();
+        if (shift == 16) SEL_STAMP(14);
         // digit d is the cut iff (#candidates with a larger digit) < remaining <= that + hist[d];
         // thread d owns bin d: suffix sums by warp shuffles, then across the eight warps
         const int here = s_hist[tid];
@@ -201,7 +221,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
           if (lane + d < 32) suf += t;
         }
         if (lane == 0) s_wsuf[warp] = suf;
+        if (shift == 16) SEL_STAMP(15);
         __syncthreads();
+        if (shift == 16) SEL_STAMP(16);
         int above = suf - here;
 #pragma unroll
         for (int w = 0; w < kSelWarps; ++w)
@@ -209,33 +231,42 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
         if (above < remaining && remaining <= above + here) {
           s_pick[0] = tid;
           s_pick[1] = remaining - above;
+          s_pick[2] = here;
         }
         __syncthreads();
+        SEL_STAMP(7 + (24 - shift) / 8);
         prefix |= static_cast<uint32_t>(s_pick[0]) << shift;
         mask |= 255u << shift;
         remaining = s_pick[1];
+        if (remaining == s_pick[2]) break;   // the whole bin is taken: lower digits cannot matter
       }
-      // prefix is now the cut value; `remaining` tokens equal to it are taken, lowest index first
+      // Over the resolved digits, prefix is the cut: larger tokens are kept, and `remaining` of
+      // the tokens equal to it, lowest index first (all of them after an early exit).
+      const bool all_equal_kept = remaining == s_pick[2];
       uint32_t eq = 0u;
 #pragma unroll
       for (int e = 0; e < kOwn; ++e) {
         if ((cand >> e) & 1u) {
-          if (u[e] > prefix) keep |= 1u << e;
-          else if (u[e] == prefix) eq |= 1u << e;
+          const uint32_t v = u[e] & mask;
+          if (v > prefix || (all_equal_kept && v == prefix)) keep |= 1u << e;
+          else if (v == prefix) eq |= 1u << e;
         }
       }
-      int eq_total;
-      int eq_rank = block_exclusive_scan(__popc(eq), s_warp, &eq_total);
+      if (!all_equal_kept) {   // uniform over the block
+        int eq_total;
+        int eq_rank = block_exclusive_scan(__popc(eq), s_warp, &eq_total);
 #pragma unroll
-      for (int e = 0; e < kOwn; ++e) {
-        if ((eq >> e) & 1u) {
-          if (eq_rank < remaining) keep |= 1u << e;
-          ++eq_rank;
+        for (int e = 0; e < kOwn; ++e) {
+          if ((eq >> e) & 1u) {
+            if (eq_rank < remaining) keep |= 1u << e;
+            ++eq_rank;
+          }
         }
       }
     }
   }
 
+  SEL_STAMP(11);
   // index-ordered emit
   int total;
   int pos = block_exclusive_scan(__popc(keep), s_warp, &total);
@@ -248,6 +279,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
     }
   }
   if (tid == 0) p.kept_cnt[b] = total;
+  SEL_STAMP(12);
 }
 
 }  // namespace
