@@ -201,7 +201,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                    const FusedParams p) {
   constexpr int NROWS = 128 / HALVES;            // text rows carried by the TMEM lanes
   constexpr int ECH = (ACH + 1) / 2;             // chunks per exp thread
-  constexpr int NBT = (ECH > kBatch0) ? 2 : 1;   // batches (= stabilisers) per exp thread
+  constexpr int NBT = 1;                         // stabilisers per exp thread
   constexpr int EPR = kColGroups * NBT;          // (max, sum) pairs per text row and CTA
   constexpr bool kRealloc = ACH > 5;             // move registers from the other warpgroups to the add warps
 
@@ -314,7 +314,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     }
   } else if (warp < kExpWarps) {
     // ---------------- exp warps ----------------
-    if (kRealloc) asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
+    if (kRealloc) asm volatile("setmaxnreg.dec.sync.aligned.u32 112;");
     const int q = warp & 3, g = warp >> 2;
     const int half = (HALVES == 2) ? (lane >> 4) : 0;
     const int row = (HALVES == 2) ? (16 * q + (lane & 15)) : (32 * q + lane);
@@ -328,6 +328,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const bool sender = (half == 0);           // with two halves, lanes s and s+16 share a row: the lower one sends
     const uint32_t pair_idx = (rank * NROWS + row) * EPR + g * NBT;            // this thread's first pair in a slot
 
+    int last_buf = -1;
     for (int h = 0; h < p.H; ++h) {
       const int buf = h % kNumBufs;
       const uint32_t bph = static_cast<uint32_t>(h / kNumBufs) & 1u;
@@ -342,61 +343,67 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
       const uint32_t slot_addr = smem_u32(&stats[slot * slot_pairs + pair_idx]);
       const uint32_t bar_addr = smem_u32(&bars.sfull[slot]);
+      // All of this thread's logits of the head are loaded at once; while they are in flight the
+      // previous head is handed to the add warps (its exponentials have been stored by now).
+      float z[ECH][kChunk];
 #pragma unroll
-      for (int bt = 0; bt < NBT; ++bt) {
-        const int lo = bt == 0 ? 0 : kBatch0;
-        const int hi = bt == 0 ? (ECH < kBatch0 ? ECH : kBatch0) : ECH;
-        float z[kBatch0][kChunk];
+      for (int t = 0; t < ECH; ++t)
+        if (t < my_chunks) tc_ld16(tbuf + kChunk * (g + t * kColGroups), z[t]);
+      if (h > 0) {
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[(h - 1) % kNumBufs]));
+      }
+      tc_wait_ld();
+      if (!all_visible) {
 #pragma unroll
-        for (int t = lo; t < hi; ++t)
-          if (t < my_chunks) tc_ld16(tbuf + kChunk * (g + t * kColGroups), z[t - lo]);
-        tc_wait_ld();
-        if (!all_visible) {
+        for (int t = 0; t < ECH; ++t) {
+          const int nvis = lim - kChunk * (g + t * kColGroups);
 #pragma unroll
-          for (int t = lo; t < hi; ++t) {
-            const int nvis = lim - kChunk * (g + t * kColGroups);
-#pragma unroll
-            for (int j = 0; j < kChunk; ++j) z[t - lo][j] = (j < nvis) ? z[t - lo][j] : -INFINITY;
-          }
-        }
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int t = lo; t < hi; ++t)
-          if (t < my_chunks) {
-#pragma unroll
-            for (int j = 0; j < kChunk; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], z[t - lo][j]);
-          }
-        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;   // scale > 0 keeps the order
-        if (HALVES == 2) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));            // one stabiliser per row
-        const float sub = (mx == -INFINITY) ? 0.0f : mx;
-        float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-        for (int t = lo; t < hi; ++t)
-          if (t < my_chunks) {
-#pragma unroll
-            for (int j = 0; j < kChunk; ++j) {
-              const float e = ex2(fmaf(z[t - lo][j], p.scale_log2e, -sub));
-              z[t - lo][j] = e;
-              ls4[j & 3] += e;
-            }
-            tc_st16(tbuf + kChunk * (g + t * kColGroups), z[t - lo]);
-          }
-        float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-        if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
-        if (sender) {
-          for (int c = 0; c < p.cluster; ++c)
-            st_async_f32x2(map_to_cta(slot_addr + bt * 8u, c), mx, lsum, map_to_cta(bar_addr, c));
+          for (int j = 0; j < kChunk; ++j) z[t][j] = (j < nvis) ? z[t][j] : -INFINITY;
         }
       }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int t = 0; t < ECH; ++t)
+        if (t < my_chunks) {
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], z[t][j]);
+        }
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;   // scale > 0 keeps the order
+      if (HALVES == 2) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));            // one stabiliser per row
+      const float sub = (mx == -INFINITY) ? 0.0f : mx;
+      float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+      for (int t = 0; t < ECH; ++t)
+        if (t < my_chunks) {
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) {
+            const float e = ex2(fmaf(z[t][j], p.scale_log2e, -sub));
+            z[t][j] = e;
+            ls4[j & 3] += e;
+          }
+          tc_st16(tbuf + kChunk * (g + t * kColGroups), z[t]);
+        }
+      float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+      if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
+      if (sender) {
+        for (int c = 0; c < p.cluster; ++c)
+          st_async_f32x2(map_to_cta(slot_addr, c), mx, lsum, map_to_cta(bar_addr, c));
+      }
+      last_buf = buf;
+      if (threadIdx.x == 0) MD_TRACE(h, 4);
+    }
+    if (last_buf >= 0) {   // hand over the last head that was worked on
       tc_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars.eready[buf]));
-      if (threadIdx.x == 0) MD_TRACE(h, 4);
+      if (lane == 0) mbar_arrive(smem_u32(&bars.eready[last_buf]));
     }
   } else {
     // ---------------- add warps ----------------
-    if (kRealloc) asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+    if (kRealloc) asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
     const int q = warp & 3;
     const int half = (HALVES == 2) ? (lane >> 4) : 0;
     const int row = (HALVES == 2) ? (16 * q + (lane & 15)) : (32 * q + lane);
@@ -557,7 +564,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     const int tk = cpl * halves;
     const size_t stage = static_cast<size_t>(nrows + tk) * 256;
     const int ach = cpl <= 5 * kChunk ? 5 : 10;             // chunks per add thread (kernel variant)
-    const int epr = kColGroups * (ach > 5 ? 2 : 1);         // (max, sum) pairs per row and CTA
+    const int epr = kColGroups;                             // (max, sum) pairs per row and CTA
     // statistics slots: kStatSlots x cluster x rows x pairs, 8 bytes each
     const size_t extra = static_cast<size_t>(kStatSlots) * c * nrows * epr * 8;
     const size_t budget = 227 * 1024 - 1024 /* static */ - 1024 /* alignment */ - extra;
