@@ -359,9 +359,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       if (!all_visible) {
 #pragma unroll
         for (int t = 0; t < ECH; ++t) {
-          const int nvis = lim - kChunk * (g + t * kColGroups);
+          const int nvis = lim - kChunk * (g + t * kColGroups);   // visible columns of this chunk
+          if (nvis < kChunk) {
 #pragma unroll
-          for (int j = 0; j < kChunk; ++j) z[t][j] = (j < nvis) ? z[t][j] : -INFINITY;
+            for (int j = 0; j < kChunk; ++j) z[t][j] = (j < nvis) ? z[t][j] : -INFINITY;
+          }
         }
       }
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
