@@ -33,6 +33,12 @@ DEFAULT_WORKLOAD = "c2_llava7b_b64"
 FALLBACK_HBM_GBS = 6650.0
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu
+# capture summarised in profiles/score_fused_kernel_c2_llava7b_b64.md.  Keyed by workload and
+# kernel variant; anything else (or a kernel changed since the capture) reports null.
+NCU_TRAFFIC_BYTES = {("c2_llava7b_b64", 64, "fused_cluster_tcgen05"): 369150208 + 3738368}
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -330,7 +336,8 @@ def run_ours(args, w):
             "hbm_headline": {"bytes_per_step": bm["headline"], "gbs": bm["headline"] / (ms_per_step / 1e3) / 1e9,
                              "frac_of_peak": bm["headline"] / (ms_per_step / 1e3) / 1e9 / peak, "peak_kind": peak_kind},
             "roofline": {"kernel": "score (%s)" % f.score_variant, "bound": "hbm", "achieved": achieved, "peak": peak,
-                         "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind,
+                         "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_BYTES.get((w.name, w.budget, f.score_variant)), "peak_kind": peak_kind,
                          "algorithmic_bytes": bm["score"]},
             "clocks": clocks,
         }
