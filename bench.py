@@ -239,8 +239,10 @@ def run_ours(args, w):
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     t_begin.record(stream)
+    host_t0 = time.perf_counter()
     for s in range(K):
         step()
+    host_enqueue_ms = 1e3 * (time.perf_counter() - host_t0) / K   # host time to enqueue one step
     t_end.record(stream)
     torch.cuda.synchronize()
     if world > 1:
@@ -331,6 +333,7 @@ def run_ours(args, w):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bm["h2d"], "d2h_bytes_per_step": bm["d2h"],
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": launches_per_step * K,
+            "host_enqueue_ms_per_step": host_enqueue_ms,
             "kernel_ms": {"score": t_score, "select": t_select, "compact": t_compact,
                           "how": "second pass over the same steps with an event around every call"},
             "hbm_headline": {"bytes_per_step": bm["headline"], "gbs": bm["headline"] / (ms_per_step / 1e3) / 1e9,

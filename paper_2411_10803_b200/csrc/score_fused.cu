@@ -42,8 +42,9 @@ constexpr int kChunk = 16;                  // TMEM columns per tcgen05.ld / st
 constexpr int kBatch0 = 3;                  // an exp thread works its chunks in two batches: 3 + 2
 constexpr int kMaxCluster = 8;
 constexpr int kMaxStages = 4;
-constexpr int kNumBufs = 3;                 // tensor-memory buffers (MMA, exp, add stages in flight)
-constexpr int kStatSlots = 2 * kNumBufs;    // a peer's exp warps run at most 2*kNumBufs heads ahead of our add warps
+constexpr int kMinBufs = 3;                 // tensor-memory buffers: MMA, exp and add stages in flight ...
+constexpr int kMaxBufs = 8;                 // ... more when the columns per head allow, to hide the per-head latency chain
+constexpr int kMaxSlots = 2 * kMaxBufs;     // statistics slots = 2 x buffers: a peer's exp warps run at most that far ahead of our add warps
 constexpr int kTmemCols = 512;
 constexpr long long kWaitCycles = 200000000LL;   // ~0.1 s at 2 GHz; no legitimate wait comes near it
 
@@ -53,6 +54,7 @@ struct FusedParams {
   void* workspace;
   int32_t H, N, L, M, vis_start, txt_start, causal;
   int32_t cluster, tk, cpl, n_stage;  // CTAs per request, keys per CTA, columns per TMEM lane
+  int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (= 2 * n_buf)
   float scale_log2e, inv_heads;
 };
 
@@ -186,10 +188,10 @@ __device__ __forceinline__ void trace_stamp(void* workspace, int n_heads, int h,
 struct __align__(8) Barriers {
   uint64_t full[kMaxStages];     // TMA -> MMA: stage filled
   uint64_t empty[kMaxStages];    // MMA -> TMA: stage consumed
-  uint64_t tfull[kNumBufs];      // MMA -> exp warps: logits of a head are in tensor memory
-  uint64_t eready[kNumBufs];     // exp -> add warps: exponentials of a head are in tensor memory
-  uint64_t tempty[kNumBufs];     // add warps -> MMA: tensor-memory buffer free
-  uint64_t sfull[kStatSlots];    // all CTAs' (max, sum) pairs of a head have arrived
+  uint64_t tfull[kMaxBufs];      // MMA -> exp warps: logits of a head are in tensor memory
+  uint64_t eready[kMaxBufs];     // exp -> add warps: exponentials of a head are in tensor memory
+  uint64_t tempty[kMaxBufs];     // add warps -> MMA: tensor-memory buffer free
+  uint64_t sfull[kMaxSlots];    // all CTAs' (max, sum) pairs of a head have arrived
   uint64_t fin;                  // add warps meet before / after staging the head sums
 };
 
@@ -215,7 +217,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const uint32_t rank = cluster_cta_rank();
   const int b = blockIdx.x / p.cluster;
   const uint32_t stage_bytes = static_cast<uint32_t>(NROWS + p.tk) * 256u;
-  // dynamic shared memory: [stages][stats: kStatSlots x cluster x NROWS x EPR float2]
+  // dynamic shared memory: [stages][stats: n_slot x cluster x NROWS x EPR float2]
   const uint32_t stage_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* stage_ptr = smem_dyn + (stage_base - smem_u32(smem_dyn));
   float2* stats = reinterpret_cast<float2*>(stage_ptr + static_cast<size_t>(p.n_stage) * stage_bytes);
@@ -224,12 +226,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&bars.full[s]), 1); mbar_init(smem_u32(&bars.empty[s]), 1); }
-    for (int s = 0; s < kNumBufs; ++s) {
+    for (int s = 0; s < kMaxBufs; ++s) {
       mbar_init(smem_u32(&bars.tfull[s]), 1);
       mbar_init(smem_u32(&bars.eready[s]), kExpWarps);
       mbar_init(smem_u32(&bars.tempty[s]), kAddWarps);
     }
-    for (int s = 0; s < kStatSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), 1);
+    for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), 1);
     mbar_init(smem_u32(&bars.fin), kAddThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -286,9 +288,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(p.cpl >> 3) << 17) |
                              (static_cast<uint32_t>(NROWS >> 4) << 24);
       for (int h = 0; h < p.H; ++h) {
-        const int s = h % p.n_stage, buf = h % kNumBufs;
+        const int s = h % p.n_stage, buf = h % p.n_buf;
         const uint32_t ph = static_cast<uint32_t>(h / p.n_stage) & 1u;
-        const uint32_t bph = static_cast<uint32_t>(h / kNumBufs) & 1u;
+        const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
         if (!mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag)) break;
         MD_TRACE(h, 1);
         if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag)) break;
@@ -330,9 +332,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 
     int last_buf = -1;
     for (int h = 0; h < p.H; ++h) {
-      const int buf = h % kNumBufs;
-      const uint32_t bph = static_cast<uint32_t>(h / kNumBufs) & 1u;
-      const int slot = h % kStatSlots;
+      const int buf = h % p.n_buf;
+      const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
+      const int slot = h % p.n_slot;
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag))) break;
       if (threadIdx.x == 0) {
         MD_TRACE(h, 3);
@@ -353,7 +355,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[(h - 1) % kNumBufs]));
+        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[(h - 1) % p.n_buf]));
       }
       tc_wait_ld();
       if (!all_visible) {
@@ -421,10 +423,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 
     int h = 0;
     for (; h < p.H; ++h) {
-      const int buf = h % kNumBufs;
-      const uint32_t bph = static_cast<uint32_t>(h / kNumBufs) & 1u;
-      const int slot = h % kStatSlots;
-      const uint32_t sph = static_cast<uint32_t>(h / kStatSlots) & 1u;
+      const int buf = h % p.n_buf;
+      const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
+      const int slot = h % p.n_slot;
+      const uint32_t sph = static_cast<uint32_t>(h / p.n_slot) & 1u;
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag))) break;
       if (tid_a == 0) MD_TRACE(h, 5);
       // statistics of this row over the whole key range: every CTA's pairs
@@ -548,6 +550,41 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t d1, uint64_t d2, uint
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+using FusedKernel = void (*)(const CUtensorMap, const CUtensorMap, const FusedParams);
+
+FusedKernel pick_kernel(int halves, int ach) {
+  return halves == 2 ? (ach > 5 ? score_fused_kernel<2, 10> : score_fused_kernel<2, 5>)
+                     : (ach > 5 ? score_fused_kernel<1, 10> : score_fused_kernel<1, 5>);
+}
+
+// Clusters of `cluster` CTAs that can be resident at once (GPC boundaries make this less than
+// SMs / cluster); 0 when it cannot be asked (no device) or the shape cannot launch.
+int max_resident_clusters(int halves, int ach, int cluster, size_t smem_bytes) {
+  FusedKernel kernel = pick_kernel(halves, ach);
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) !=
+      cudaSuccess) {
+    (void)cudaGetLastError();
+    return 0;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(cluster));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 0;
+  }
+  return n;
+}
+
 }  // namespace
 
 // Geometry of the fused kernel for a problem; false when the shape is outside what it covers.
@@ -567,24 +604,41 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     const size_t stage = static_cast<size_t>(nrows + tk) * 256;
     const int ach = cpl <= 5 * kChunk ? 5 : 10;             // chunks per add thread (kernel variant)
     const int epr = kColGroups;                             // (max, sum) pairs per row and CTA
-    // statistics slots: kStatSlots x cluster x rows x pairs, 8 bytes each
-    const size_t extra = static_cast<size_t>(kStatSlots) * c * nrows * epr * 8;
-    const size_t budget = 227 * 1024 - 1024 /* static */ - 1024 /* alignment */ - extra;
-    int n_stage = static_cast<int>(budget / stage);
+    // As many tensor-memory buffers as the columns allow (3..8), fewer if their statistics
+    // slots (2 x buffers x cluster x rows x pairs x 8 bytes) would leave no room for 2 stages.
+    int n_buf = kTmemCols / cpl;
+    if (n_buf > kMaxBufs) n_buf = kMaxBufs;
+    if (n_buf < kMinBufs) continue;
+    size_t extra = 0;
+    int n_stage = 0;
+    for (; n_buf >= kMinBufs; --n_buf) {
+      extra = static_cast<size_t>(2 * n_buf) * c * nrows * epr * 8;
+      const size_t reserved = 1024 /* static */ + 1024 /* alignment */ + extra;
+      if (reserved + 2 * stage > 227 * 1024) continue;
+      n_stage = static_cast<int>((227 * 1024 - reserved) / stage);
+      // a stage is held for a load latency plus an MMA (~2.3 us): prefer four stages over more buffers
+      if (n_stage >= kMaxStages || n_buf == kMinBufs) break;
+    }
     if (n_stage < 2) continue;
     if (n_stage > kMaxStages) n_stage = kMaxStages;
-    if (kNumBufs * cpl > kTmemCols) continue;
-    const long ctas = static_cast<long>(r.B) * c;
-    const long waves = (ctas + sm_count - 1) / sm_count;
-    const double fill = static_cast<double>(ctas) / static_cast<double>(waves * sm_count);
-    const double useful = static_cast<double>(r.L) / static_cast<double>(c * tk);
-    const double score = fill * useful - 0.002 * c;   // prefer smaller clusters among equals
+    // Cost model (microseconds per head and CTA): streaming the stage at ~45 GB/s per SM, or the
+    // MMA -> exp -> exchange -> add chain (~4.5 us) spread over the buffers, whichever is longer;
+    // times the number of waves of CTAs.
+    size_t smem_bytes = stage * n_stage + 1024 + extra;
+    // at least 116 KB, so that two CTAs (each wanting all of tensor memory) never share an SM
+    if (smem_bytes < 116 * 1024) smem_bytes = 116 * 1024;
+    int resident = max_resident_clusters(halves, ach, c, smem_bytes);
+    if (resident <= 0) resident = sm_count / c;    // no device to ask: ignore GPC boundaries
+    if (resident <= 0) continue;
+    const long waves = (r.B + resident - 1) / resident;
+    const double t_stream = static_cast<double>(stage) / 45.0e3;
+    const double t_chain = 4.5 / n_buf;
+    const double t_head = t_stream > t_chain ? t_stream : t_chain;
+    const double score = 1.0 / (static_cast<double>(waves) * t_head) - 1e-4 * c;   // prefer smaller clusters among equals
     if (score > best) {
       best = score;
-      g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_stage = n_stage; g.n_buf = kNumBufs; g.ach = ach;
-      // at least 116 KB, so that two CTAs (each wanting all of tensor memory) never share an SM
-      g.smem_bytes = stage * n_stage + 1024 + extra;
-      if (g.smem_bytes < 116 * 1024) g.smem_bytes = 116 * 1024;
+      g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_stage = n_stage; g.n_buf = n_buf; g.ach = ach;
+      g.smem_bytes = smem_bytes;
     }
   }
   if (best < 0.0) return false;
@@ -608,11 +662,11 @@ cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, co
   p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
   p.causal = r.causal;
   p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_stage = geo.n_stage;
+  p.n_buf = geo.n_buf; p.n_slot = 2 * geo.n_buf;
   p.scale_log2e = r.scale_log2e;
   p.inv_heads = 1.0f / static_cast<float>(r.H);
 
-  auto kernel = geo.halves == 2 ? (geo.ach > 5 ? score_fused_kernel<2, 10> : score_fused_kernel<2, 5>)
-                                : (geo.ach > 5 ? score_fused_kernel<1, 10> : score_fused_kernel<1, 5>);
+  FusedKernel kernel = pick_kernel(geo.halves, geo.ach);
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(geo.smem_bytes));
   if (e != cudaSuccess) return e;
