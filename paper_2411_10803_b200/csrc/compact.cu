@@ -24,11 +24,12 @@ struct CompactParams {
   int64_t hid_sb, hid_sl, k_sb, k_sh, k_sl, v_sb, v_sh, v_sl;
 };
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+// Source rows are read once: no L1 allocation, first in line for L2 eviction.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p, uint64_t policy) {
   uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
+               : "l"(p), "l"(policy));
   return v;
 }
 
@@ -39,6 +40,7 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
 
 __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams p) {
   const int r = blockIdx.x, b = blockIdx.y, which = blockIdx.z;
+  MD_PIPE(p.workspace, 2, false, false);
   pdl_launch_dependents();
   pdl_wait();   // kept_idx / kept_cnt come from the previous kernel in the stream
   if (p.src[which] == nullptr) return;
@@ -49,6 +51,8 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
     return;
   }
   const int64_t row = p.vis_start + j;
+  uint64_t once;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(once));
   if (which == 0) {
     const uint4* src = p.src[0] + b * p.hid_sb + row * p.hid_sl;
     uint4* dst = p.dst[0] + (static_cast<int64_t>(b) * p.cap + r) * p.hidden_vecs;
@@ -58,7 +62,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         const int x = base + u * kCompactThreads + threadIdx.x;
-        if (x < n) v[u] = ld_stream(src + x);
+        if (x < n) v[u] = ld_stream(src + x, once);
       }
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
@@ -77,7 +81,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         const int x = base + u * kCompactThreads + threadIdx.x;
-        if (x < n) v[u] = ld_stream(src + (x >> 4) * sh + (x & 15));
+        if (x < n) v[u] = ld_stream(src + (x >> 4) * sh + (x & 15), once);
       }
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
@@ -86,6 +90,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
       }
     }
   }
+  MD_PIPE(p.workspace, 2, true, false);
 }
 
 }  // namespace

@@ -97,6 +97,30 @@ inline cudaError_t launch_pdl(Kernel kernel, dim3 grid, dim3 block, size_t smem,
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+// Optional pipeline tracing (compiled in only with -DMUSTDROP_TRACE): first CTA start and last
+// CTA end of every kernel, per step, as global-timer values in the workspace (bytes 3072..4095:
+// [counter][step % 20][kernel 0..2][start, end]).
+#ifdef MUSTDROP_TRACE
+__device__ __forceinline__ unsigned long long md_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void md_pipe_stamp(void* workspace, int kernel, bool is_end, bool new_step) {
+  if (workspace == nullptr || threadIdx.x != 0) return;
+  unsigned long long* base = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(workspace) + 3072);
+  unsigned long long step = *reinterpret_cast<volatile unsigned long long*>(base);
+  if (new_step && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) step = atomicAdd(base, 1ull) + 1ull;
+  else if (new_step) return;   // only one CTA opens a step; the others stamp at their end
+  unsigned long long* slot = base + 1 + ((step % 20ull) * 3ull + kernel) * 2ull;
+  if (is_end) atomicMax(slot + 1, md_now());
+  else atomicMin(slot, md_now());
+}
+#define MD_PIPE(ws, kernel, is_end, new_step) md_pipe_stamp((ws), (kernel), (is_end), (new_step))
+#else
+#define MD_PIPE(ws, kernel, is_end, new_step) ((void)0)
+#endif
+
 // Device-side helper: record the first device-detected condition (never traps).
 __device__ __forceinline__ void record_status(void* workspace, int32_t code, int32_t detail) {
   if (workspace == nullptr) return;

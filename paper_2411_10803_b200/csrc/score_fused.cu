@@ -122,6 +122,20 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
       : "memory");
 }
+// The same copy with an L2 eviction-priority hint (keys are read exactly once: evict them first,
+// so that they do not push out data other kernels left in L2).
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                                 uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+  return policy;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -216,6 +230,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_cta_rank();
   const int b = blockIdx.x / p.cluster;
+  MD_PIPE(p.workspace, 0, false, true);
   const uint32_t stage_bytes = static_cast<uint32_t>(NROWS + p.tk) * 256u;
   // dynamic shared memory: [stages][stats: n_slot x cluster x NROWS x EPR float2]
   const uint32_t stage_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -256,6 +271,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     if (warp == kTmaWarp && lane == 0) {
       // ---------------- TMA producer ----------------
       const int key0 = static_cast<int>(rank) * p.tk;
+      const uint64_t stream_once = l2_evict_first_policy();
       int issued = 0;
       for (int h = 0; h < p.H; ++h) {
         const int s = h % p.n_stage;
@@ -271,8 +287,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           tma_load_4d(q_dst + slab * (NROWS * 128u), &q_map, slab * 64, 0, h, b, full);
 #pragma unroll
           for (int hv = 0; hv < HALVES; ++hv)
-            tma_load_4d(k_dst + slab * (p.tk * 128u) + hv * (p.cpl * 128u), &k_map, slab * 64, key0 + hv * p.cpl, h, b,
-                        full);
+            tma_load_4d_hint(k_dst + slab * (p.tk * 128u) + hv * (p.cpl * 128u), &k_map, slab * 64, key0 + hv * p.cpl,
+                             h, b, full, stream_once);
         }
         issued = h + 1;
       }
@@ -517,6 +533,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
   cluster_sync_all();   // no CTA leaves while a peer may still write into its shared memory
+  MD_PIPE(p.workspace, 0, true, false);
 }
 
 // ---- host side ------------------------------------------------------------------------------------

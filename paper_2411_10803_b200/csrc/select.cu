@@ -89,6 +89,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
   // Work that touches no global data, then let the next kernel start its prologue and wait for
   // the kernel that produced g / i.
   SEL_STAMP(0);
+  MD_PIPE(p.workspace, 1, false, false);
   for (int w = tid; w < kMaxVis / 32; w += kSelThreads) s_key[w] = 0u;
   s_hist[tid] = 0;
   if (tid == 0) s_nkey = 0;
@@ -279,6 +280,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
     }
   }
   if (tid == 0) p.kept_cnt[b] = total;
+  MD_PIPE(p.workspace, 1, true, false);
   SEL_STAMP(12);
 }
 
