@@ -34,9 +34,9 @@ FALLBACK_HBM_GBS = 6650.0
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel, from the ncu
-# capture summarised in profiles/score_fused_kernel_c2_llava7b_b64.md.  Keyed by workload and
-# kernel variant; anything else (or a kernel changed since the capture) reports null.
-NCU_TRAFFIC_BYTES = {("c2_llava7b_b64", 64, "fused_cluster_tcgen05"): 369150208 + 3738368}
+# captures summarised under profiles/.  Keyed by (workload, budget, "filter" | "score", kernel
+# variant); anything else (or a kernel changed since its capture) reports null.
+NCU_TRAFFIC_BYTES = {}
 
 
 def measured_peak():
@@ -215,12 +215,19 @@ def run_ours(args, w):
     f = md.Filter(md.config_for(w), device=dev)
     stream = torch.cuda.current_stream()
 
-    def step():
-        f.score(d_q, d_k, stream)
-        f.select(d_ki if use_keys else None, d_kc if use_keys else None, stream=stream, want_s=False)
-        f.compact(d_hid, d_k, d_v, stream=stream)
+    ki, kc = (d_ki, d_kc) if use_keys else (None, None)
+    single_call = args.path != "staged"     # the one-call entry point (one launch where the plan allows)
 
-    launches_per_step = {"two_pass_mma": 2}.get(f.score_variant, 1) + 2
+    def step():
+        if single_call:
+            f.filter(d_q, d_k, d_v, d_hid, ki, kc, stream=stream)
+        else:
+            f.score(d_q, d_k, stream)
+            f.select(ki, kc, stream=stream, want_s=False)
+            f.compact(d_hid, d_k, d_v, stream=stream)
+
+    launches_per_step = f.filter_launches if single_call else {"two_pass_mma": 2}.get(f.score_variant, 1) + 2
+    one_kernel = single_call and launches_per_step == 1
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if sampler is not None:
@@ -251,19 +258,22 @@ def run_ours(args, w):
 
     # per-call durations for the roofline: a second pass over the same K steps with an event
     # around every call (the events serialise the calls, so these add up to more than a step)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(K)]
     for s in range(K):
         ev[s][0].record(stream)
         f.score(d_q, d_k, stream)
         ev[s][1].record(stream)
-        f.select(d_ki if use_keys else None, d_kc if use_keys else None, stream=stream, want_s=False)
+        f.select(ki, kc, stream=stream, want_s=False)
         ev[s][2].record(stream)
         f.compact(d_hid, d_k, d_v, stream=stream)
         ev[s][3].record(stream)
+        f.filter(d_q, d_k, d_v, d_hid, ki, kc, stream=stream)
+        ev[s][4].record(stream)
     torch.cuda.synchronize()
     t_score = statistics.mean(ev[s][0].elapsed_time(ev[s][1]) for s in range(K))
     t_select = statistics.mean(ev[s][1].elapsed_time(ev[s][2]) for s in range(K))
     t_compact = statistics.mean(ev[s][2].elapsed_time(ev[s][3]) for s in range(K))
+    t_filter = statistics.mean(ev[s][3].elapsed_time(ev[s][4]) for s in range(K))
     code, detail = f.device_status()
     if code != 0:
         raise RuntimeError("device status %d (detail %d) after the timed region" % (code, detail))
@@ -284,9 +294,12 @@ def run_ours(args, w):
         s_hid.view(torch.int16).copy_(h_hid, non_blocking=True)
         s_ki.copy_(h_ki, non_blocking=True)
         s_kc.copy_(h_kc, non_blocking=True)
-        f.score(s_q, s_k, stream)
-        f.select(s_ki if use_keys else None, s_kc if use_keys else None, stream=stream, want_s=False)
-        f.compact(s_hid, s_k, s_v, stream=stream)
+        if single_call:
+            f.filter(s_q, s_k, s_v, s_hid, s_ki if use_keys else None, s_kc if use_keys else None, stream=stream)
+        else:
+            f.score(s_q, s_k, stream)
+            f.select(s_ki if use_keys else None, s_kc if use_keys else None, stream=stream, want_s=False)
+            f.compact(s_hid, s_k, s_v, stream=stream)
         o_idx.copy_(f.kept_idx, non_blocking=True)
         o_cnt.copy_(f.kept_cnt, non_blocking=True)
         o_h.copy_(f.hidden_out, non_blocking=True)
@@ -320,7 +333,13 @@ def run_ours(args, w):
     if rank == 0:
         bm = bytes_model(w)
         peak, peak_kind = measured_peak()
-        achieved = bm["score"] / (t_score / 1e3) / 1e9
+        # dominant kernel: the single-launch filter kernel (score + selection + gather: K, Q_text,
+        # gathered rows read, compacted rows written), else the score kernel (K, Q_text read)
+        if one_kernel:
+            dom_name, dom_bytes, dom_ms = "filter (%s + select + gather tail)" % f.score_variant, bm["full"], t_filter
+        else:
+            dom_name, dom_bytes, dom_ms = "score (%s)" % f.score_variant, bm["score"], t_score
+        achieved = dom_bytes / (dom_ms / 1e3) / 1e9
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -329,19 +348,22 @@ def run_ours(args, w):
                        "n_heads": w.n_heads, "hidden": w.hidden, "budget": w.budget, "key_set": w.key_cnt,
                        "parallelism": "dp%d (independent requests, no collective)" % world,
                        "l2": "inputs exceed L2 (K alone is %.0f MB per GPU)" % (bm["score"] / 1e6),
-                       "score_variant": f.score_variant},
+                       "score_variant": f.score_variant,
+                       "path": ("mustdrop_filter, %d launch(es) per step" % launches_per_step) if single_call
+                       else "mustdrop_score + mustdrop_select + mustdrop_compact"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bm["h2d"], "d2h_bytes_per_step": bm["d2h"],
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": launches_per_step * K,
             "host_enqueue_ms_per_step": host_enqueue_ms,
-            "kernel_ms": {"score": t_score, "select": t_select, "compact": t_compact,
-                          "how": "second pass over the same steps with an event around every call"},
+            "kernel_ms": {"score": t_score, "select": t_select, "compact": t_compact, "filter_call": t_filter,
+                          "how": "second pass over the same steps with an event around every call "
+                                 "(the three separate calls, then the one-call filter)"},
             "hbm_headline": {"bytes_per_step": bm["headline"], "gbs": bm["headline"] / (ms_per_step / 1e3) / 1e9,
                              "frac_of_peak": bm["headline"] / (ms_per_step / 1e3) / 1e9 / peak, "peak_kind": peak_kind},
-            "roofline": {"kernel": "score (%s)" % f.score_variant, "bound": "hbm", "achieved": achieved, "peak": peak,
+            "roofline": {"kernel": dom_name, "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES.get((w.name, w.budget, f.score_variant)), "peak_kind": peak_kind,
-                         "algorithmic_bytes": bm["score"]},
+                         "traffic": NCU_TRAFFIC_BYTES.get((w.name, w.budget, dom_name.split(" ")[0], f.score_variant)),
+                         "peak_kind": peak_kind, "algorithmic_bytes": dom_bytes, "ms": dom_ms},
             "clocks": clocks,
         }
         if world == 1 and not args.no_cpu_baseline:
@@ -367,6 +389,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--budget", type=int, default=0, help="override the workload's keep budget")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--path", default="filter", choices=["filter", "staged"],
+                    help="filter: the one-call entry point; staged: score, select and compact as three calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]

@@ -173,6 +173,33 @@ mustdrop_status_t mustdrop_compact(const mustdrop_plan_t *plan, const int32_t *k
                                    void *workspace, void *cuda_stream);
 
 /*
+ * The whole filtering step of one pruning layer in one call (Sec. 3.4: Eq. 8-10 on the text-to-
+ * vision attention, the key set of Sec. 3.3 kept, pruned tokens removed from the sequence and
+ * the KV cache): mustdrop_score, then mustdrop_select on its outputs, then mustdrop_compact with
+ * the selected indices.  Results are those of the three calls made in that order on one stream;
+ * g_out, i_out, (s_out), kept_idx and kept_cnt are all written.
+ *
+ * Where the plan's score kernel is the fused one and a kept row (hidden row + K + V pieces of all
+ * heads) fits its shared-memory ring, this is ONE kernel launch: the thread-block cluster that
+ * scored a request also selects its tokens and gathers them, so a request's copy starts while
+ * other requests are still being scored.  Otherwise it enqueues the separate kernels.
+ * mustdrop_plan_filter_launches tells which (1, or the number of separate launches).
+ *
+ * Arguments as in the three calls (all device pointers, 16-byte aligned): q_text, k required;
+ * (hidden, hidden_out) and (v, v_out) may each be NULL together; k_out may be NULL to leave K
+ * uncopied; s_out may be NULL; key_idx / key_cnt may be NULL when key_max == 0.
+ * Errors as in the three calls; nothing is launched when an argument is refused.
+ */
+mustdrop_status_t mustdrop_filter(const mustdrop_plan_t *plan, const void *q_text, const void *k,
+                                  const void *v, const void *hidden, const int32_t *key_idx,
+                                  const int32_t *key_cnt, float *g_out, float *i_out, float *s_out,
+                                  int32_t *kept_idx, int32_t *kept_cnt, void *hidden_out, void *k_out,
+                                  void *v_out, void *workspace, void *cuda_stream);
+
+/* Kernel launches one mustdrop_filter call enqueues for this plan (-1: invalid plan). */
+int32_t mustdrop_plan_filter_launches(const mustdrop_plan_t *plan);
+
+/*
  * Read the device status word of a workspace (synchronises `cuda_stream`).
  * code_out (host) receives MUSTDROP_OK or the first device-detected condition, detail_out
  * (host, may be NULL) an operation-specific detail (BAD_KEY_INDEX: request * 65536 + slot).

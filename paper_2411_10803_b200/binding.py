@@ -33,7 +33,7 @@ EXPORTS = (
     "mustdrop_filter_plan", "mustdrop_plan_destroy", "mustdrop_score", "mustdrop_select",
     "mustdrop_compact", "mustdrop_device_status", "mustdrop_status_string",
     "mustdrop_last_cuda_error", "mustdrop_plan_score_variant", "mustdrop_score_static",
-    "mustdrop_score_static_max_rows",
+    "mustdrop_score_static_max_rows", "mustdrop_filter", "mustdrop_plan_filter_launches",
 )
 
 
@@ -82,6 +82,9 @@ def lib() -> ctypes.CDLL:
         L.mustdrop_score_static.restype = ctypes.c_int
         L.mustdrop_score_static_max_rows.restype = ctypes.c_size_t
         L.mustdrop_compact.argtypes = [vp] * 11
+        L.mustdrop_filter.argtypes = [vp] * 17
+        L.mustdrop_plan_filter_launches.argtypes = [vp]
+        L.mustdrop_plan_filter_launches.restype = ctypes.c_int32
         L.mustdrop_device_status.argtypes = [vp, vp, vp, i32p, i32p]
         L.mustdrop_status_string.argtypes = [ctypes.c_int]
         L.mustdrop_status_string.restype = ctypes.c_char_p
@@ -89,7 +92,7 @@ def lib() -> ctypes.CDLL:
         L.mustdrop_plan_score_variant.argtypes = [vp]
         L.mustdrop_plan_score_variant.restype = ctypes.c_char_p
         for n in ("mustdrop_filter_plan", "mustdrop_plan_destroy", "mustdrop_score", "mustdrop_select",
-                  "mustdrop_compact", "mustdrop_device_status"):
+                  "mustdrop_compact", "mustdrop_filter", "mustdrop_device_status"):
             getattr(L, n).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -192,6 +195,17 @@ def mustdrop_compact(plan, kept_idx, kept_cnt, hidden, k, v, hidden_out, k_out, 
                                   _ptr(hidden_out), _ptr(k_out), _ptr(v_out), _ptr(workspace), _stream(stream))
 
 
+def mustdrop_filter(plan, q_text, k, v, hidden, key_idx, key_cnt, g_out, i_out, s_out, kept_idx, kept_cnt,
+                    hidden_out, k_out, v_out, workspace, stream=None) -> int:
+    return lib().mustdrop_filter(plan, _ptr(q_text), _ptr(k), _ptr(v), _ptr(hidden), _ptr(key_idx), _ptr(key_cnt),
+                                 _ptr(g_out), _ptr(i_out), _ptr(s_out), _ptr(kept_idx), _ptr(kept_cnt),
+                                 _ptr(hidden_out), _ptr(k_out), _ptr(v_out), _ptr(workspace), _stream(stream))
+
+
+def mustdrop_plan_filter_launches(plan) -> int:
+    return lib().mustdrop_plan_filter_launches(plan)
+
+
 def mustdrop_device_status(plan, workspace, stream=None) -> Tuple[int, int, int]:
     """-> (status of the call, device code, detail)."""
     code, detail = ctypes.c_int32(0), ctypes.c_int32(0)
@@ -272,6 +286,19 @@ class Filter:
         self.score(q_text, k, stream)
         self.select(key_idx, key_cnt, stream=stream, want_s=want_s)
         return self.compact(hidden, k, v, stream=stream)
+
+    def filter(self, q_text, k, v, hidden, key_idx=None, key_cnt=None, stream=None, want_s=False):
+        """The whole step through the single entry point (one launch where the plan allows it)."""
+        self._check(mustdrop_filter(self.plan, q_text, k, v, hidden, key_idx, key_cnt, self.g, self.i,
+                                    self.s if want_s else None, self.kept_idx, self.kept_cnt,
+                                    self.hidden_out if hidden is not None else None, self.k_out,
+                                    self.v_out if v is not None else None, self.workspace, stream),
+                    "mustdrop_filter")
+        return self.hidden_out, self.k_out, self.v_out
+
+    @property
+    def filter_launches(self) -> int:
+        return mustdrop_plan_filter_launches(self.plan)
 
     def device_status(self, stream=None):
         st, code, detail = mustdrop_device_status(self.plan, self.workspace, stream)

@@ -114,6 +114,13 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
     const int forced_cluster = cl ? std::atoi(cl) : 0;
     const bool allow_fused = !(want && std::strcmp(want, "two_pass") == 0);
     if (allow_fused && plan_score_fused(r, p->sm_count, forced_cluster, &p->fused)) p->score_variant = kScoreFusedCluster;
+    // mustdrop_filter: one launch where the fused kernel covers the shape and a kept row fits its
+    // shared-memory ring; MUSTDROP_FILTER=staged forces the three launches (debugging override).
+    const char* fw = std::getenv("MUSTDROP_FILTER");
+    p->filter_single = 0;
+    if (p->score_variant == kScoreFusedCluster && !(fw && std::strcmp(fw, "staged") == 0) &&
+        plan_filter_single(r, p->fused, &p->filter))
+      p->filter_single = 1;
   }
   size_t off = kWsStatusBytes;
   p->ws_rowstats_off = off;
@@ -181,6 +188,41 @@ mustdrop_status_t mustdrop_compact(const mustdrop_plan_t* plan, const int32_t* k
   cudaError_t e = mustdrop::launch_compact(*plan, kept_idx, kept_cnt, hidden, k, v, hidden_out, k_out, v_out,
                                            workspace, stream);
   return e == cudaSuccess ? MUSTDROP_OK : cuda_fail(e);
+}
+
+mustdrop_status_t mustdrop_filter(const mustdrop_plan_t* plan, const void* q_text, const void* k, const void* v,
+                                  const void* hidden, const int32_t* key_idx, const int32_t* key_cnt, float* g_out,
+                                  float* i_out, float* s_out, int32_t* kept_idx, int32_t* kept_cnt,
+                                  void* hidden_out, void* k_out, void* v_out, void* workspace, void* cuda_stream) {
+  if (!valid_plan(plan) || q_text == nullptr || k == nullptr || g_out == nullptr || i_out == nullptr ||
+      kept_idx == nullptr || kept_cnt == nullptr)
+    return MUSTDROP_ERR_INVALID_ARG;
+  if (plan->r.key_max > 0 && (key_idx == nullptr || key_cnt == nullptr)) return MUSTDROP_ERR_INVALID_ARG;
+  if ((hidden == nullptr) != (hidden_out == nullptr) || (v == nullptr) != (v_out == nullptr))
+    return MUSTDROP_ERR_INVALID_ARG;
+  if (workspace == nullptr) return MUSTDROP_ERR_WORKSPACE;
+  const void* ptrs[] = {q_text, k, v, hidden, key_idx, key_cnt, g_out, i_out, s_out, kept_idx, kept_cnt,
+                        hidden_out, k_out, v_out, workspace};
+  for (const void* q : ptrs)
+    if (q != nullptr && !aligned16(q)) return MUSTDROP_ERR_INVALID_ARG;
+  if (plan->filter_single) {
+    cudaError_t e = mustdrop::launch_filter_fused(*plan, q_text, k, v, hidden, key_idx, key_cnt, g_out, i_out, s_out,
+                                                  kept_idx, kept_cnt, hidden_out, k_out, v_out, workspace,
+                                                  static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? MUSTDROP_OK : cuda_fail(e);
+  }
+  mustdrop_status_t st = mustdrop_score(plan, q_text, k, g_out, i_out, workspace, cuda_stream);
+  if (st != MUSTDROP_OK) return st;
+  st = mustdrop_select(plan, g_out, i_out, key_idx, key_cnt, kept_idx, kept_cnt, s_out, workspace, cuda_stream);
+  if (st != MUSTDROP_OK) return st;
+  return mustdrop_compact(plan, kept_idx, kept_cnt, hidden, k_out != nullptr ? k : nullptr, v, hidden_out, k_out,
+                          v_out, workspace, cuda_stream);
+}
+
+int32_t mustdrop_plan_filter_launches(const mustdrop_plan_t* plan) {
+  if (!valid_plan(plan)) return -1;
+  if (plan->filter_single) return 1;
+  return plan->score_variant == mustdrop::kScoreTwoPassMma ? 4 : 3;
 }
 
 mustdrop_status_t mustdrop_device_status(const mustdrop_plan_t* plan, const void* workspace, void* cuda_stream,

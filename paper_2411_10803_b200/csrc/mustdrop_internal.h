@@ -34,6 +34,13 @@ struct FusedGeometry {
   size_t smem_bytes;  // dynamic shared memory
 };
 
+// Shared-memory plan of the selection / gather tail of the single-launch filter kernel.
+struct FilterGeometry {
+  size_t smem_bytes;   // dynamic shared memory of the launch (>= the score geometry's)
+  int32_t slot_bytes;  // one kept row: hidden row + K pieces + V pieces of all heads
+  int32_t n_slot;      // rows in flight per CTA
+};
+
 struct Resolved {
   int32_t B, H, D, hidden, L, vis_start, M, txt_start, N;
   int32_t causal, mode, criteria, budget, key_max, cap;
@@ -53,6 +60,8 @@ struct mustdrop_plan {
   size_t ws_bytes;
   size_t ws_rowstats_off;   // float2 [B,H,N]: (row max in log2 units, 1 / row sum)
   mustdrop::FusedGeometry fused;
+  int32_t filter_single;    // 1: mustdrop_filter is one launch of the fused kernel with its tail
+  mustdrop::FilterGeometry filter;
 };
 
 namespace mustdrop {
@@ -65,6 +74,11 @@ cudaError_t launch_score_two_pass(const mustdrop_plan& p, const void* q_text, co
 bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out);
 cudaError_t launch_score_fused(const mustdrop_plan& p, const void* q_text, const void* k, float* g_out,
                                float* i_out, void* workspace, cudaStream_t stream);
+bool plan_filter_single(const Resolved& r, const FusedGeometry& geo, FilterGeometry* out);
+cudaError_t launch_filter_fused(const mustdrop_plan& p, const void* q_text, const void* k, const void* v,
+                                const void* hidden, const int32_t* key_idx, const int32_t* key_cnt, float* g_out,
+                                float* i_out, float* s_out, int32_t* kept_idx, int32_t* kept_cnt, void* hidden_out,
+                                void* k_out, void* v_out, void* workspace, cudaStream_t stream);
 cudaError_t launch_select(const mustdrop_plan& p, const float* g, const float* i, const int32_t* key_idx,
                           const int32_t* key_cnt, int32_t* kept_idx, int32_t* kept_cnt, float* s_out,
                           void* workspace, cudaStream_t stream);

@@ -11,7 +11,8 @@
 //                 count on the receiver's mbarrier;
 //   4 add warps   once all pairs of a head have arrived, normalise the exponentials and add them
 //                 into per-thread head sums that live in registers for the whole kernel.
-// Three tensor-memory buffers keep the MMA, exp and add stages of consecutive heads in flight.
+// Three to eight tensor-memory buffers (as many as the columns per head allow) keep the MMA, exp
+// and add stages of consecutive heads in flight.
 // After the last head the head mean is reduced over the text rows into G (column sum) and
 // I (column max).  K is read once; nothing goes through global scratch.
 //
@@ -26,6 +27,7 @@
 #include <cuda_bf16.h>
 
 #include "mustdrop_internal.h"
+#include "select_body.cuh"
 
 namespace mustdrop {
 namespace {
@@ -39,13 +41,14 @@ constexpr int kTmaWarp = kExpWarps + kAddWarps;   // warp 12
 constexpr int kMmaWarp = kTmaWarp + 1;            // warp 13; warps 14-15 only fill the last warpgroup
 constexpr int kThreads = 16 * 32;
 constexpr int kChunk = 16;                  // TMEM columns per tcgen05.ld / st
-constexpr int kBatch0 = 3;                  // an exp thread works its chunks in two batches: 3 + 2
 constexpr int kMaxCluster = 8;
 constexpr int kMaxStages = 4;
 constexpr int kMinBufs = 3;                 // tensor-memory buffers: MMA, exp and add stages in flight ...
 constexpr int kMaxBufs = 8;                 // ... more when the columns per head allow, to hide the per-head latency chain
 constexpr int kMaxSlots = 2 * kMaxBufs;     // statistics slots = 2 x buffers: a peer's exp warps run at most that far ahead of our add warps
 constexpr int kTmemCols = 512;
+constexpr int kMaxGatherSlots = 8;         // rows in flight per CTA in the gather tail of the filter kernel
+constexpr int kKeptListBytes = kMaxVis * 4; // the request's kept indices, at the start of dynamic shared memory
 constexpr long long kWaitCycles = 200000000LL;   // ~0.1 s at 2 GHz; no legitimate wait comes near it
 
 struct FusedParams {
@@ -56,6 +59,21 @@ struct FusedParams {
   int32_t cluster, tk, cpl, n_stage;  // CTAs per request, keys per CTA, columns per TMEM lane
   int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (= 2 * n_buf)
   float scale_log2e, inv_heads;
+};
+
+// Tail of the single-launch filter kernel: selection and gather-compaction of the request by
+// the cluster that scored it.
+struct FilterTail {
+  SelectParams sel;              // g / i are the score outputs of this launch
+  const unsigned char* hidden;   // null: tensor not copied
+  unsigned char* hidden_out;
+  int64_t hid_sb, hid_sl;        // bytes
+  int32_t hidden_bytes;          // bytes of a hidden row (0 when not copied)
+  int32_t hidden_pad;            // the same rounded up to 128 (alignment of the tensor copies behind it)
+  int32_t kv_bytes;              // bytes of a K (or V) row over all heads = H * 256
+  int32_t has_k, has_v;
+  int32_t slot_bytes, n_slot;    // gather ring in dynamic shared memory
+  int32_t vis_start;
 };
 
 // ---- small PTX wrappers ------------------------------------------------------------------------
@@ -131,6 +149,26 @@ __device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar), "l"(policy)
       : "memory");
 }
+// Bulk copies of the gather tail: a contiguous row (1-D) or one token's pieces over all heads
+// (4-D box 128 x 1 x H x 1) from global to shared memory, and back out to the dense outputs.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_store_1d(void* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::"l"(map),
+               "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {
   uint64_t policy;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
@@ -207,18 +245,24 @@ struct __align__(8) Barriers {
   uint64_t tempty[kMaxBufs];     // add warps -> MMA: tensor-memory buffer free
   uint64_t sfull[kMaxSlots];    // all CTAs' (max, sum) pairs of a head have arrived
   uint64_t fin;                  // add warps meet before / after staging the head sums
+  uint64_t gfull[kMaxGatherSlots];   // filter tail: a gathered row has landed in its slot
+};
+
+// Tensor maps of the gather tail (used only by the FILTER instantiations).
+struct GatherMaps {
+  CUtensorMap k_src, v_src, k_dst, v_dst;
 };
 
 // HALVES: 2 = two M=64 tiles per head (N <= 64), 1 = one M=128 tile.
 // ACH: chunks (of 16 columns) an add thread may own; an exp thread owns up to (ACH+1)/2.
-template <int HALVES, int ACH>
+// FILTER: after the scores, the cluster also selects the request's tokens and gathers them.
+template <int HALVES, int ACH, bool FILTER>
 __global__ void __launch_bounds__(kThreads, 1)
 score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
-                   const FusedParams p) {
+                   const FusedParams p, const __grid_constant__ GatherMaps gm, const FilterTail ft) {
   constexpr int NROWS = 128 / HALVES;            // text rows carried by the TMEM lanes
   constexpr int ECH = (ACH + 1) / 2;             // chunks per exp thread
-  constexpr int NBT = 1;                         // stabilisers per exp thread
-  constexpr int EPR = kColGroups * NBT;          // (max, sum) pairs per text row and CTA
+  constexpr int EPR = kColGroups;                // (max, sum) pairs per text row and CTA: one per column group
   constexpr bool kRealloc = ACH > 5;             // move registers from the other warpgroups to the add warps
 
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
@@ -248,6 +292,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     }
     for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), 1);
     mbar_init(smem_u32(&bars.fin), kAddThreads);
+    for (int s = 0; s < kMaxGatherSlots; ++s) mbar_init(smem_u32(&bars.gfull[s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kMmaWarp) {
@@ -344,7 +389,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     lim = (lim < p.L ? lim : p.L) - key_lane0;                                 // ... as a column count of this lane
     const bool all_visible = lim >= p.cpl;
     const bool sender = (half == 0);           // with two halves, lanes s and s+16 share a row: the lower one sends
-    const uint32_t pair_idx = (rank * NROWS + row) * EPR + g * NBT;            // this thread's first pair in a slot
+    const uint32_t pair_idx = (rank * NROWS + row) * EPR + g;                  // this thread's pair in a slot
 
     int last_buf = -1;
     for (int h = 0; h < p.H; ++h) {
@@ -473,9 +518,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           tc_ld16(tbuf + kChunk * c0, e[0]);
           if (c0 + 1 < ACH && c0 + 1 < total_chunks) tc_ld16(tbuf + kChunk * (c0 + 1), e[1]);
           tc_wait_ld();
-          // chunk c belongs to column group c & 1, local index c >> 1, batch (c >> 1) >= kBatch0
-          const float f0 = f[0 * NBT + ((c0 >> 1) >= kBatch0 ? NBT - 1 : 0)];
-          const float f1 = f[1 * NBT + ((c0 >> 1) >= kBatch0 ? NBT - 1 : 0)];
+          // chunk c was exponentiated by column group c & 1 (c0 is even)
+          const float f0 = f[0], f1 = f[1];
 #pragma unroll
           for (int j = 0; j < kChunk; ++j) acc[c0][j] = fmaf(e[0][j], f0, acc[c0][j]);
           if (c0 + 1 < ACH && c0 + 1 < total_chunks) {
@@ -525,6 +569,15 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   }
 
   // ---------------- common exit ----------------
+  if (kRealloc && FILTER) {
+    // The tail below runs on every warp: back to the 128 registers per thread the kernel was
+    // compiled for (8 x 112 + 4 x 224 + 4 x 40 warps' worth become 16 x 128, the whole file).
+    // The add warps release theirs when they get here; the others wait for that inside inc.
+    __syncwarp();
+    if (warp >= kTmaWarp) asm volatile("setmaxnreg.inc.sync.aligned.u32 128;");
+    else if (warp >= kExpWarps) asm volatile("setmaxnreg.dec.sync.aligned.u32 128;");
+    else asm volatile("setmaxnreg.inc.sync.aligned.u32 128;");
+  }
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag != 0) record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
@@ -534,6 +587,95 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   }
   cluster_sync_all();   // no CTA leaves while a peer may still write into its shared memory
   MD_PIPE(p.workspace, 0, true, false);
+
+  if constexpr (FILTER) {
+    // ---------------- selection and gather of this request ----------------
+    // The cluster barrier above also ordered every CTA's g_out / i_out stores before the loads
+    // below.  Dynamic shared memory is free: all copies have landed, all MMAs have read them and
+    // every statistics pair sent to this CTA has been consumed.  Each CTA of the cluster runs the
+    // same selection on its own (identical inputs, fixed order: identical lists); rank 0 stores
+    // the list.  Row r of the compacted outputs is then copied by CTA r mod cluster.
+    __shared__ SelectShared sel_sh;
+    __shared__ int32_t kept_total_s;
+    int32_t* kept_list = reinterpret_cast<int32_t*>(stage_ptr);
+    pdl_wait();   // the outputs written below may still be read by an earlier kernel in the stream
+    if (*abort_flag != 0) return;
+    if (warp < kSelWarps) {
+      const int tid = threadIdx.x;
+      select_clear(sel_sh, tid);
+      const bool writer = rank == 0;
+      const int own = (ft.sel.M + kSelThreads - 1) / kSelThreads;
+      if (own <= 1) select_request<1, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      else if (own <= 2) select_request<2, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      else if (own <= 4) select_request<4, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      else if (own <= 8) select_request<8, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      else select_request<16, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+    }
+    __syncthreads();
+    if (warp == kExpWarps && lane == 0) {
+      // One thread drives the copies: rows are loaded into a ring of shared-memory slots by bulk
+      // copies that count on the slot's mbarrier, and stored from there by bulk copies tracked in
+      // bulk groups.  Loads run n_slot - 2 rows ahead of the stores.
+      fence_proxy_async();   // earlier generic-proxy accesses to the slots precede the async-proxy writes
+      const int total = kept_total_s < ft.sel.cap ? kept_total_s : ft.sel.cap;
+      const int C = p.cluster;
+      const int n_mine = total > static_cast<int>(rank) ? (total - static_cast<int>(rank) + C - 1) / C : 0;
+      const int S = ft.n_slot, ahead = S - 2;
+      const uint32_t ring = stage_base + kKeptListBytes;
+      const uint32_t payload = static_cast<uint32_t>(ft.hidden_bytes) + static_cast<uint32_t>(ft.has_k + ft.has_v) * ft.kv_bytes;
+      const uint64_t once = l2_evict_first_policy();
+      bool ok = true;
+      int loaded = 0;
+      for (int i = 0; i < n_mine + ahead && ok; ++i) {
+        if (i < n_mine) {
+          const int slot = i % S;
+          if (i >= S) bulk_wait_read_1();   // the stores of row i - S have finished reading the slot
+          const int r = static_cast<int>(rank) + i * C;
+          const int row = ft.vis_start + kept_list[r];
+          const uint32_t bar = smem_u32(&bars.gfull[slot]);
+          uint32_t dst = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
+          mbar_expect_tx(bar, payload);
+          if (ft.hidden_bytes > 0) {
+            bulk_load_1d(dst, ft.hidden + b * ft.hid_sb + row * ft.hid_sl, ft.hidden_bytes, bar, once);
+            dst += ft.hidden_pad;
+          }
+          if (ft.has_k) {
+            tma_load_4d_hint(dst, &gm.k_src, 0, row, 0, b, bar, once);
+            dst += ft.kv_bytes;
+          }
+          if (ft.has_v) tma_load_4d_hint(dst, &gm.v_src, 0, row, 0, b, bar, once);
+          loaded = i + 1;
+        }
+        const int c = i - ahead;
+        if (c >= 0) {
+          const int slot = c % S;
+          if (!mbar_wait(smem_u32(&bars.gfull[slot]), static_cast<uint32_t>(c / S) & 1u, abort_flag)) { ok = false; break; }
+          const int r = static_cast<int>(rank) + c * C;
+          uint32_t src = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
+          if (ft.hidden_bytes > 0) {
+            bulk_store_1d(ft.hidden_out + (static_cast<int64_t>(b) * ft.sel.cap + r) * ft.hidden_bytes, src, ft.hidden_bytes);
+            src += ft.hidden_pad;
+          }
+          if (ft.has_k) {
+            tma_store_4d(&gm.k_dst, 0, r, 0, b, src);
+            src += ft.kv_bytes;
+          }
+          if (ft.has_v) tma_store_4d(&gm.v_dst, 0, r, 0, b, src);
+          bulk_commit();
+        }
+      }
+      if (!ok) {
+        // gave up: still leave only when every load this thread started has landed (bounded)
+        record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
+        for (int i = (loaded > S ? loaded - S : 0); i < loaded; ++i) {
+          const uint32_t bar = smem_u32(&bars.gfull[i % S]);
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar, static_cast<uint32_t>(i / S) & 1u) && clock64() - t0 < kWaitCycles) {}
+        }
+      }
+      bulk_wait_all();   // the stores have been written before the CTA (and its shared memory) goes away
+    }
+  }
 }
 
 // ---- host side ------------------------------------------------------------------------------------
@@ -567,11 +709,29 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t d1, uint64_t d2, uint
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-using FusedKernel = void (*)(const CUtensorMap, const CUtensorMap, const FusedParams);
+// bf16 tensor [d3][d2][d1][128] with byte strides s1, s2, s3, no swizzle; box = 128 x 1 x d2 x 1:
+// one token's 256-byte pieces over all heads.
+bool make_gather_map(CUtensorMap* map, const void* base, uint64_t d1, uint64_t d2, uint64_t d3, uint64_t s1,
+                     uint64_t s2, uint64_t s3) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[4] = {128, d1, d2, d3};
+  const cuuint64_t strides[3] = {s1, s2, s3};
+  const cuuint32_t box[4] = {128, 1, static_cast<cuuint32_t>(d2), 1};
+  const cuuint32_t elem[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
-FusedKernel pick_kernel(int halves, int ach) {
-  return halves == 2 ? (ach > 5 ? score_fused_kernel<2, 10> : score_fused_kernel<2, 5>)
-                     : (ach > 5 ? score_fused_kernel<1, 10> : score_fused_kernel<1, 5>);
+using FusedKernel = void (*)(const CUtensorMap, const CUtensorMap, const FusedParams, const GatherMaps, const FilterTail);
+
+FusedKernel pick_kernel(int halves, int ach, bool filter = false) {
+  if (filter)
+    return halves == 2 ? (ach > 5 ? score_fused_kernel<2, 10, true> : score_fused_kernel<2, 5, true>)
+                       : (ach > 5 ? score_fused_kernel<1, 10, true> : score_fused_kernel<1, 5, true>);
+  return halves == 2 ? (ach > 5 ? score_fused_kernel<2, 10, false> : score_fused_kernel<2, 5, false>)
+                     : (ach > 5 ? score_fused_kernel<1, 10, false> : score_fused_kernel<1, 5, false>);
 }
 
 // Clusters of `cluster` CTAs that can be resident at once (GPC boundaries make this less than
@@ -630,7 +790,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     int n_stage = 0;
     for (; n_buf >= kMinBufs; --n_buf) {
       extra = static_cast<size_t>(2 * n_buf) * c * nrows * epr * 8;
-      const size_t reserved = 1024 /* static */ + 1024 /* alignment */ + extra;
+      const size_t reserved = 4096 /* static */ + 1024 /* alignment */ + extra;
       if (reserved + 2 * stage > 227 * 1024) continue;
       n_stage = static_cast<int>((227 * 1024 - reserved) / stage);
       // a stage is held for a load latency plus an MMA (~2.3 us): prefer four stages over more buffers
@@ -663,8 +823,12 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
   return true;
 }
 
-cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, const void* k, float* g_out,
-                               float* i_out, void* workspace, cudaStream_t stream) {
+namespace {
+
+// Common launch of the score kernel, with (tail != nullptr) or without the selection / gather tail.
+cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, const void* k, float* g_out,
+                                float* i_out, void* workspace, const GatherMaps* maps, const FilterTail* tail,
+                                size_t smem_bytes, cudaStream_t stream) {
   const Resolved& r = plan.r;
   const FusedGeometry& geo = plan.fused;
   const int nrows = 128 / geo.halves;
@@ -683,14 +847,14 @@ cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, co
   p.scale_log2e = r.scale_log2e;
   p.inv_heads = 1.0f / static_cast<float>(r.H);
 
-  FusedKernel kernel = pick_kernel(geo.halves, geo.ach);
+  FusedKernel kernel = pick_kernel(geo.halves, geo.ach, tail != nullptr);
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(geo.smem_bytes));
+                                       static_cast<int>(smem_bytes));
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(r.B * geo.cluster));
   cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = geo.smem_bytes;
+  cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -701,7 +865,70 @@ cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, co
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, kernel, q_map, k_map, p);
+  static const GatherMaps no_maps = {};
+  static const FilterTail no_tail = {};
+  return cudaLaunchKernelEx(&cfg, kernel, q_map, k_map, p, maps ? *maps : no_maps, tail ? *tail : no_tail);
+}
+
+}  // namespace
+
+cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, const void* k, float* g_out,
+                               float* i_out, void* workspace, cudaStream_t stream) {
+  return launch_fused_common(plan, q_text, k, g_out, i_out, workspace, nullptr, nullptr, plan.fused.smem_bytes, stream);
+}
+
+// Shared-memory plan of the gather tail; false when a row does not fit the ring at least three times.
+bool plan_filter_single(const Resolved& r, const FusedGeometry& geo, FilterGeometry* out) {
+  if (r.H > 256) return false;                                     // box of the per-token K / V copy
+  const size_t hidden_pad = (static_cast<size_t>(r.hidden) * 2 + 127) / 128 * 128;
+  const size_t slot = hidden_pad + 2 * static_cast<size_t>(r.H) * 256;
+  const size_t limit = 227 * 1024 - 4096;                          // dynamic shared memory a CTA may ask for
+  const size_t fixed = 1024 + kKeptListBytes;
+  size_t want = fixed + kMaxGatherSlots * slot;
+  if (want < geo.smem_bytes) want = geo.smem_bytes;
+  if (want > limit) want = limit;
+  if (want < geo.smem_bytes) return false;
+  int n_slot = static_cast<int>((want - fixed) / slot);
+  if (n_slot > kMaxGatherSlots) n_slot = kMaxGatherSlots;
+  if (n_slot < 3) return false;
+  out->smem_bytes = want;
+  out->slot_bytes = static_cast<int32_t>(slot);
+  out->n_slot = n_slot;
+  return true;
+}
+
+cudaError_t launch_filter_fused(const mustdrop_plan& plan, const void* q_text, const void* k, const void* v,
+                                const void* hidden, const int32_t* key_idx, const int32_t* key_cnt, float* g_out,
+                                float* i_out, float* s_out, int32_t* kept_idx, int32_t* kept_cnt, void* hidden_out,
+                                void* k_out, void* v_out, void* workspace, cudaStream_t stream) {
+  const Resolved& r = plan.r;
+  GatherMaps maps = {};
+  const uint64_t out_s1 = 256, out_s2 = static_cast<uint64_t>(r.cap) * 256, out_s3 = static_cast<uint64_t>(r.H) * out_s2;
+  if (k_out != nullptr &&
+      (!make_gather_map(&maps.k_src, k, r.L, r.H, r.B, static_cast<uint64_t>(r.k_sl) * 2,
+                        static_cast<uint64_t>(r.k_sh) * 2, static_cast<uint64_t>(r.k_sb) * 2) ||
+       !make_gather_map(&maps.k_dst, k_out, r.cap, r.H, r.B, out_s1, out_s2, out_s3)))
+    return cudaErrorInvalidValue;
+  if (v_out != nullptr &&
+      (!make_gather_map(&maps.v_src, v, r.L, r.H, r.B, static_cast<uint64_t>(r.v_sl) * 2,
+                        static_cast<uint64_t>(r.v_sh) * 2, static_cast<uint64_t>(r.v_sb) * 2) ||
+       !make_gather_map(&maps.v_dst, v_out, r.cap, r.H, r.B, out_s1, out_s2, out_s3)))
+    return cudaErrorInvalidValue;
+  FilterTail t = {};
+  t.sel.g = g_out; t.sel.i = i_out; t.sel.key_idx = key_idx; t.sel.key_cnt = key_cnt;
+  t.sel.kept_idx = kept_idx; t.sel.kept_cnt = kept_cnt; t.sel.s_out = s_out; t.sel.workspace = workspace;
+  t.sel.M = r.M; t.sel.key_max = r.key_max; t.sel.mode = r.mode; t.sel.criteria = r.criteria;
+  t.sel.budget = r.budget; t.sel.cap = r.cap; t.sel.gamma = r.gamma; t.sel.alpha = r.alpha;
+  t.hidden = static_cast<const unsigned char*>(hidden);
+  t.hidden_out = static_cast<unsigned char*>(hidden_out);
+  t.hid_sb = r.hid_sb * 2; t.hid_sl = r.hid_sl * 2;
+  t.hidden_bytes = hidden_out != nullptr ? r.hidden * 2 : 0;
+  t.hidden_pad = (t.hidden_bytes + 127) / 128 * 128;
+  t.kv_bytes = r.H * 256;
+  t.has_k = k_out != nullptr; t.has_v = v_out != nullptr;
+  t.slot_bytes = plan.filter.slot_bytes; t.n_slot = plan.filter.n_slot;
+  t.vis_start = r.vis_start;
+  return launch_fused_common(plan, q_text, k, g_out, i_out, workspace, &maps, &t, plan.filter.smem_bytes, stream);
 }
 
 }  // namespace mustdrop

@@ -1,0 +1,156 @@
+"""GPU parity of the single-call filter (score, selection and gather in one launch where the
+plan allows it) against the CPU oracle, and bit-equality with the three separate calls."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2411_10803_b200 import binding as md
+from paper_2411_10803_b200 import build as md_build
+from paper_2411_10803_b200 import synth
+
+from parity_util import assert_kept_matches, bf16_bits, host_gather, to_dev, to_dev_bf16
+from test_gpu_parity import key_args, run_chain_and_check, small
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    md_build.build()
+    assert torch.cuda.is_available()
+
+
+@pytest.fixture
+def cluster(request, monkeypatch):
+    monkeypatch.delenv("MUSTDROP_SCORE_VARIANT", raising=False)
+    monkeypatch.delenv("MUSTDROP_FILTER", raising=False)
+    if request.param:
+        monkeypatch.setenv("MUSTDROP_CLUSTER", str(request.param))
+    else:
+        monkeypatch.delenv("MUSTDROP_CLUSTER", raising=False)
+    return request.param
+
+
+def test_filter_tiny_reference_config_is_one_launch():
+    run_chain_and_check(synth.WORKLOADS["c1_tiny"], path="filter", expect_launches=1)
+
+
+@pytest.mark.parametrize("cluster", [0, 1, 2, 3, 5, 8], indirect=True)
+def test_filter_small_ragged_batch(cluster):
+    # 5 requests, ragged sizes, vision span not at 0, more kept rows than CTAs in the cluster
+    w = small(batch=5, n_vis=333, n_txt=21, n_heads=3, hidden=384, key_cnt=9, budget=40, vis_start=2)
+    run_chain_and_check(w, path="filter", expect_launches=1)
+
+
+@pytest.mark.parametrize("cluster", [0, 4], indirect=True)
+def test_filter_fewer_kept_rows_than_ctas(cluster):
+    w = small(batch=3, n_vis=200, n_txt=9, key_cnt=1, budget=2)
+    run_chain_and_check(w, path="filter", expect_launches=1)
+
+
+@pytest.mark.parametrize("budget", [192, 64])
+def test_filter_llava7b_batch16(budget):
+    run_chain_and_check(synth.WORKLOADS["c2_llava7b_b16"].with_(budget=budget), sample=[0, 9], path="filter",
+                        expect_launches=1)
+
+
+def test_filter_llava7b_batch64_sampled():
+    run_chain_and_check(synth.WORKLOADS["c2_llava7b_b64"], sample=[0, 31, 63], path="filter", expect_launches=1)
+
+
+def test_filter_13b_batch64_sampled():
+    run_chain_and_check(synth.WORKLOADS["c5_13b_b64"], sample=[17], path="filter", expect_launches=1)
+
+
+def test_filter_falls_back_to_separate_launches_for_long_sequences():
+    # 2880 vision tokens are outside the fused kernel's key range: the call still does the whole step
+    w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
+    run_chain_and_check(w, sample=[1], path="filter", expect_launches=4)
+
+
+def _run_both(w, monkeypatch, cfg_kw=None, drop=()):
+    """The single call and the three calls on the same inputs -> two dicts of host arrays."""
+    d = synth.make_batch(w)
+    q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
+    ki, kc = key_args(w, d)
+    out = []
+    for staged in (False, True):
+        if staged:
+            monkeypatch.setenv("MUSTDROP_FILTER", "staged")
+        else:
+            monkeypatch.delenv("MUSTDROP_FILTER", raising=False)
+        f = md.Filter(md.config_for(w, **(cfg_kw or {})))
+        assert f.filter_launches == (3 if staged else 1)
+        f.filter(q, k, None if "v" in drop else v, None if "hidden" in drop else hid, ki, kc, want_s=True)
+        torch.cuda.synchronize()
+        assert f.device_status() == (0, 0)
+        out.append(dict(g=f.g.cpu().numpy(), i=f.i.cpu().numpy(), s=f.s.cpu().numpy(),
+                        idx=f.kept_idx.cpu().numpy(), cnt=f.kept_cnt.cpu().numpy(), ho=bf16_bits(f.hidden_out),
+                        ko=bf16_bits(f.k_out), vo=bf16_bits(f.v_out)))
+        f.close()
+    return d, out[0], out[1]
+
+
+@pytest.mark.parametrize("mode_kw", [
+    dict(),
+    dict(mode=md.MUSTDROP_MODE_THRESHOLD),
+    dict(criteria=md.MUSTDROP_CRIT_GLOBAL_ONLY),
+    dict(criteria=md.MUSTDROP_CRIT_INDIVIDUAL_ONLY),
+    dict(causal=0),
+])
+def test_filter_equals_the_three_calls_bit_for_bit(mode_kw, monkeypatch):
+    w = small(batch=4, n_vis=777, n_txt=33, n_heads=5, hidden=640, key_cnt=11, budget=100)
+    d, one, three = _run_both(w, monkeypatch, mode_kw)
+    for name in ("g", "i", "s", "cnt"):
+        assert np.array_equal(one[name], three[name]), name
+    for b in range(w.batch):
+        n = one["cnt"][b]
+        assert np.array_equal(one["idx"][b, :n], three["idx"][b, :n])
+        assert np.array_equal(one["ho"][b, :n], three["ho"][b, :n])
+        assert np.array_equal(one["ko"][b, :, :n], three["ko"][b, :, :n])
+        assert np.array_equal(one["vo"][b, :, :n], three["vo"][b, :, :n])
+    if mode_kw.get("mode") == md.MUSTDROP_MODE_THRESHOLD:
+        # the oracle's rule on the GPU's own scores: Eq. 9 and Eq. 10 as printed, key set kept
+        ref_idx, ref_cnt, _, _ = oracle.select(one["g"], one["i"], w.seq_len, d["key_idx"], d["key_cnt"],
+                                                mode=oracle.MODE_THRESHOLD)
+        assert np.array_equal(ref_cnt, one["cnt"])
+        for b in range(w.batch):
+            assert np.array_equal(ref_idx[b, :ref_cnt[b]], one["idx"][b, :ref_cnt[b]])
+
+
+@pytest.mark.parametrize("drop", [("v",), ("hidden",), ("v", "hidden")])
+def test_filter_copies_only_the_tensors_it_is_given(drop, monkeypatch):
+    w = small(batch=3, n_vis=300, n_txt=12, n_heads=4, hidden=512, key_cnt=5, budget=37)
+    d, one, three = _run_both(w, monkeypatch, drop=drop)
+    idx, cnt = one["idx"], one["cnt"]
+    assert np.array_equal(idx, three["idx"]) and np.array_equal(cnt, three["cnt"])
+    zh, zk, zv = np.zeros_like(one["ho"]), np.zeros_like(one["ko"]), np.zeros_like(one["vo"])
+    eh, ek, ev = host_gather(idx, cnt, w.vis_start, d["hidden"], d["k"], d["v"], zh, zk, zv)
+    assert np.array_equal(one["ko"], ek)
+    # a tensor that was not given stays as allocated (zeros)
+    assert np.array_equal(one["ho"], zh if "hidden" in drop else eh)
+    assert np.array_equal(one["vo"], zv if "v" in drop else ev)
+
+
+def test_filter_without_a_key_set_and_keep_all():
+    w = small(batch=2, n_vis=130, n_txt=5, key_cnt=0, budget=130)
+    run_chain_and_check(w, path="filter", expect_launches=1)
+
+
+def test_filter_is_deterministic_and_repeatable_on_one_stream():
+    w = synth.WORKLOADS["c2_llava7b_b16"].with_(batch=6)
+    d = synth.make_batch(w)
+    f = md.Filter(md.config_for(w))
+    q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
+    ki, kc = key_args(w, d)
+    f.filter(q, k, v, hid, ki, kc)
+    first = (f.g.clone(), f.i.clone(), f.kept_idx.clone(), f.hidden_out.clone(), f.k_out.clone(), f.v_out.clone())
+    for _ in range(5):   # back to back: each launch overlaps the tail of the one before
+        f.filter(q, k, v, hid, ki, kc)
+    torch.cuda.synchronize()
+    assert f.device_status() == (0, 0)
+    now = (f.g, f.i, f.kept_idx, f.hidden_out, f.k_out, f.v_out)
+    for a, b in zip(first, now):
+        assert torch.equal(a, b)
+    f.close()

@@ -285,14 +285,20 @@ def test_compact_skips_an_out_of_range_index_and_reports_it():
 
 # ---- the chain -------------------------------------------------------------------------------
 
-def run_chain_and_check(w, sample=None, check_scores=True):
-    """score -> select -> compact on the GPU for the whole batch; oracle on `sample` requests."""
+def run_chain_and_check(w, sample=None, check_scores=True, path="staged", expect_launches=None):
+    """score -> select -> compact on the GPU for the whole batch (three calls, or the single
+    mustdrop_filter call with path="filter"); oracle on `sample` requests."""
     d = synth.make_batch(w)
     sample = list(range(w.batch)) if sample is None else sample
     f = md.Filter(md.config_for(w))
     q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
     ki, kc = key_args(w, d)
-    f.run(q, k, v, hid, ki, kc, want_s=True)
+    if path == "filter":
+        if expect_launches is not None:
+            assert f.filter_launches == expect_launches
+        f.filter(q, k, v, hid, ki, kc, want_s=True)
+    else:
+        f.run(q, k, v, hid, ki, kc, want_s=True)
     torch.cuda.synchronize()
     assert f.device_status() == (0, 0)
     g, i = f.g.cpu().numpy(), f.i.cpu().numpy()
