@@ -570,13 +570,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 
   // ---------------- common exit ----------------
   if (kRealloc && FILTER) {
-    // The tail below runs on every warp: back to the 128 registers per thread the kernel was
-    // compiled for (8 x 112 + 4 x 224 + 4 x 40 warps' worth become 16 x 128, the whole file).
-    // The add warps release theirs when they get here; the others wait for that inside inc.
+    // The tail below runs on every warp: give them all the exp warps' 112 registers.  The add
+    // warps release theirs when they get here; the TMA / MMA warps wait for that inside inc.
+    // (16 x 112 warps' worth is less than the kernel held so far, so inc can always be served.)
     __syncwarp();
-    if (warp >= kTmaWarp) asm volatile("setmaxnreg.inc.sync.aligned.u32 128;");
-    else if (warp >= kExpWarps) asm volatile("setmaxnreg.dec.sync.aligned.u32 128;");
-    else asm volatile("setmaxnreg.inc.sync.aligned.u32 128;");
+    if (warp >= kTmaWarp) asm volatile("setmaxnreg.inc.sync.aligned.u32 112;");
+    else if (warp >= kExpWarps) asm volatile("setmaxnreg.dec.sync.aligned.u32 112;");
   }
   tc_fence_before();
   __syncthreads();
