@@ -183,3 +183,38 @@ def make_batch(w: Workload, with_values: bool = True, requests: Optional[range] 
 
 def sha256_of(a: np.ndarray) -> str:
     return hashlib.sha256(np.ascontiguousarray(a).tobytes()).hexdigest()
+
+
+PAD_BITS = 0x7FC0   # bf16 quiet NaN: padding rows must never influence a result
+
+
+def draw_vis_cnt(w: Workload, lo: float = 0.6, hi: float = 0.95, salt: int = 7) -> np.ndarray:
+    """Per-request number of vision tokens left by the spatial merge: uniform in
+    [lo*M, hi*M] (the paper reports 576 -> 440 on average, Table 3), at least the key set."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([w.seed, salt])))
+    m = rng.integers(max(int(lo * w.n_vis), w.key_cnt, 1), max(int(hi * w.n_vis), w.key_cnt, 1) + 1, size=w.batch)
+    return m.astype(np.int32)
+
+
+def pack_ragged(d: Dict[str, np.ndarray], w: Workload, vis_cnt) -> Dict[str, np.ndarray]:
+    """Turn a dense batch into a ragged one (data movement only): request b keeps its first
+    vis_cnt[b] vision rows, its text rows move directly behind them, every later row of k, v
+    and hidden is filled with NaN bits; key indices at or beyond vis_cnt[b] are dropped."""
+    out = {n: a.copy() for n, a in d.items()}
+    vs, M, N = w.vis_start, w.n_vis, w.n_txt
+    for b in range(d["k"].shape[0]):
+        m = int(vis_cnt[b])
+        for name in ("k", "v"):
+            if name in out:
+                a = out[name][b]
+                a[:, vs + m:vs + m + N] = d[name][b][:, vs + M:vs + M + N]
+                a[:, vs + m + N:] = PAD_BITS
+        if "hidden" in out:
+            out["hidden"][b, vs + m:vs + m + N] = d["hidden"][b, vs + M:vs + M + N]
+            out["hidden"][b, vs + m + N:] = PAD_BITS
+        keys = [j for j in d["key_idx"][b, :d["key_cnt"][b]].tolist() if j < m]
+        out["key_idx"][b] = -1
+        out["key_idx"][b, :len(keys)] = keys
+        out["key_cnt"][b] = len(keys)
+    out["vis_cnt"] = np.asarray(vis_cnt, np.int32).copy()
+    return out
