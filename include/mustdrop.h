@@ -58,6 +58,17 @@ typedef enum {
   MUSTDROP_CRIT_INDIVIDUAL_ONLY = 2
 } mustdrop_criteria_t;
 
+/*
+ * MUSTDROP_FLAG_REBUILD_SEQUENCE: the compacted outputs hold the request's whole next sequence
+ * instead of the kept vision rows only: the vis_start prefix rows, the kept vision rows, then
+ * the n_txt text rows, packed without a gap - the input layout of the next pruning layer
+ * (Sec. 3.4 filters "from the shallow layers" on, every layer on what the last one kept).
+ * Outputs then have vis_start + cap + n_txt rows per request (and head); rows behind a
+ * request's own end are left untouched.  Requires txt_start == vis_start + n_vis and
+ * seq_len == txt_start + n_txt.
+ */
+#define MUSTDROP_FLAG_REBUILD_SEQUENCE 1
+
 typedef struct {
   int32_t batch;      /* B, independent requests */
   int32_t n_heads;    /* H */
@@ -76,7 +87,7 @@ typedef struct {
   float   gamma;      /* Eq. 9 threshold; 0 => 1/n_vis */
   float   alpha;      /* Eq. 10 threshold; 0 => 2/seq_len */
   int32_t key_max;    /* capacity of key_idx per request; 0 = no key set */
-  int32_t reserved;   /* must be 0 */
+  int32_t flags;      /* bit set of MUSTDROP_FLAG_*; other bits must be 0 */
   /* Strides in ELEMENTS (bf16); 0 => contiguous.  Head rows themselves are contiguous
    * (head_dim elements).  Every stride must be a multiple of 8 (16 bytes). */
   int64_t k_stride_b, k_stride_h, k_stride_l;       /* K      [B,H,L,D] */
@@ -195,6 +206,43 @@ mustdrop_status_t mustdrop_filter(const mustdrop_plan_t *plan, const void *q_tex
                                   const int32_t *key_cnt, float *g_out, float *i_out, float *s_out,
                                   int32_t *kept_idx, int32_t *kept_cnt, void *hidden_out, void *k_out,
                                   void *v_out, void *workspace, void *cuda_stream);
+
+/*
+ * One pruning layer of a chain of layers (Sec. 3.4: the filter is applied at successive layers,
+ * each on the tokens the previous one kept; after the spatial merge of Sec. 3.3 requests hold
+ * different numbers of vision tokens; the set left after the last layer is the S_few of the
+ * decoding-stage cache policy, Sec. 3.5).  mustdrop_filter with four optional additions, all
+ * device pointers, each may be NULL:
+ *   vis_cnt  int32 [B]       vision tokens request b actually holds, 1..n_vis (values outside
+ *                            are clamped).  Its text tokens then sit directly behind them, at
+ *                            rows vis_start + vis_cnt[b] .. + n_txt of k / v / hidden; later rows
+ *                            are padding and are never read.  Scores of the absent tokens come
+ *                            out 0, they are never selected, a request with fewer tokens than the
+ *                            budget keeps them all, and thresholds left at 0 default per request
+ *                            (gamma = 1 / vis_cnt[b], alpha = 2 / (vis_start + vis_cnt[b] + n_txt)).
+ *                            Needs txt_start == vis_start + n_vis and seq_len == txt_start + n_txt.
+ *                            May be the kept_cnt an earlier call on the same stream wrote.
+ *   orig_idx int32 [B,n_vis] original id of every current vision token (NULL: 0, 1, 2, ...)
+ *   orig_out int32 [B,cap]   receives the original ids of the kept tokens, ascending: the next
+ *                            layer's orig_idx; after the last layer, S_few
+ *   key_idx_out int32 [B,key_max], key_cnt_out int32 [B]
+ *                            positions of the key tokens among the kept tokens: the next layer's
+ *                            key_idx / key_cnt
+ * With MUSTDROP_FLAG_REBUILD_SEQUENCE the outputs of one layer are laid out as the inputs of the
+ * next (vis_cnt = this layer's kept_cnt).  One kernel launch where mustdrop_filter is one.
+ */
+typedef struct {
+  const void *q_text, *k, *v, *hidden;       /* as in mustdrop_filter */
+  const int32_t *key_idx, *key_cnt;
+  const int32_t *vis_cnt, *orig_idx;
+  float *g_out, *i_out, *s_out;
+  int32_t *kept_idx, *kept_cnt;
+  int32_t *orig_out, *key_idx_out, *key_cnt_out;
+  void *hidden_out, *k_out, *v_out;
+} mustdrop_layer_io_t;
+
+mustdrop_status_t mustdrop_filter_layer(const mustdrop_plan_t *plan, const mustdrop_layer_io_t *io /* (host) */,
+                                        void *workspace, void *cuda_stream);
 
 /* Kernel launches one mustdrop_filter call enqueues for this plan (-1: invalid plan). */
 int32_t mustdrop_plan_filter_launches(const mustdrop_plan_t *plan);

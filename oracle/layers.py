@@ -35,7 +35,7 @@ def filter_layer_ragged(q_text: np.ndarray, k: np.ndarray, v: np.ndarray, hidden
     per request (gamma = 1 / vis_cnt[b], alpha = 2 / its own sequence length).  A request with
     fewer tokens than the budget keeps them all.
 
-    Returns G, I [B,M] (zero past vis_cnt[b]), kept_idx [B,budget] (-1 unused), kept_cnt [B],
+    Returns G, I and the selection score s [B,M] (zero past vis_cnt[b]), kept_idx [B,budget] (-1 unused), kept_cnt [B],
     orig_out [B,budget] (orig_idx composed with kept_idx; identity when orig_idx is None) and
     the gathered tensors: the kept vision rows only, or with ``rebuild`` the whole next
     sequence [prefix ; kept vision ; text] packed the same way (zero elsewhere).
@@ -46,6 +46,7 @@ def filter_layer_ragged(q_text: np.ndarray, k: np.ndarray, v: np.ndarray, hidden
     hid = hidden.shape[2]
     G = np.zeros((B, M), np.float32)
     I = np.zeros((B, M), np.float32)
+    S = np.zeros((B, M), np.float32)
     kept_idx = np.full((B, budget), -1, np.int32)
     kept_cnt = np.zeros((B,), np.int32)
     orig_out = np.full((B, budget), -1, np.int32)
@@ -63,7 +64,8 @@ def filter_layer_ragged(q_text: np.ndarray, k: np.ndarray, v: np.ndarray, hidden
         ki = kc = None
         if key_idx is not None:
             ki, kc = key_idx[b:b + 1], key_cnt[b:b + 1]
-        idx, cnt, _, _ = oracle.select(g, i, lb, ki, kc, budget=kb, criteria=criteria)
+        idx, cnt, sc, _ = oracle.select(g, i, lb, ki, kc, budget=kb, criteria=criteria)
+        S[b, :m] = sc[0]
         n = int(cnt[0])
         kept_idx[b, :n], kept_cnt[b] = idx[0, :n], n
         src = orig_idx[b] if orig_idx is not None else np.arange(M, dtype=np.int32)
@@ -74,7 +76,7 @@ def filter_layer_ragged(q_text: np.ndarray, k: np.ndarray, v: np.ndarray, hidden
         ho[b, :len(rows)] = hidden[b, rows]
         ko[b, :, :len(rows)] = k[b][:, rows]
         vo[b, :, :len(rows)] = v[b][:, rows]
-    return dict(G=G, I=I, kept_idx=kept_idx, kept_cnt=kept_cnt, orig_out=orig_out, hidden_out=ho, k_out=ko, v_out=vo)
+    return dict(G=G, I=I, s=S, kept_idx=kept_idx, kept_cnt=kept_cnt, orig_out=orig_out, hidden_out=ho, k_out=ko, v_out=vo)
 
 
 def progressive_filter(layers: List[Dict[str, np.ndarray]], vis_start: int, vis_cnt0: Sequence[int],

@@ -34,6 +34,7 @@ EXPORTS = (
     "mustdrop_compact", "mustdrop_device_status", "mustdrop_status_string",
     "mustdrop_last_cuda_error", "mustdrop_plan_score_variant", "mustdrop_score_static",
     "mustdrop_score_static_max_rows", "mustdrop_filter", "mustdrop_plan_filter_launches",
+    "mustdrop_filter_layer",
 )
 
 
@@ -44,11 +45,20 @@ class mustdrop_config_t(ctypes.Structure):
         ("n_vis", ctypes.c_int32), ("txt_start", ctypes.c_int32), ("n_txt", ctypes.c_int32),
         ("causal", ctypes.c_int32), ("scale", ctypes.c_float), ("mode", ctypes.c_int32),
         ("criteria", ctypes.c_int32), ("budget", ctypes.c_int32), ("gamma", ctypes.c_float),
-        ("alpha", ctypes.c_float), ("key_max", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("alpha", ctypes.c_float), ("key_max", ctypes.c_int32), ("flags", ctypes.c_int32),
         ("k_stride_b", ctypes.c_int64), ("k_stride_h", ctypes.c_int64), ("k_stride_l", ctypes.c_int64),
         ("v_stride_b", ctypes.c_int64), ("v_stride_h", ctypes.c_int64), ("v_stride_l", ctypes.c_int64),
         ("hid_stride_b", ctypes.c_int64), ("hid_stride_l", ctypes.c_int64),
     ]
+
+
+MUSTDROP_FLAG_REBUILD_SEQUENCE = 1
+
+
+class mustdrop_layer_io_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in (
+        "q_text", "k", "v", "hidden", "key_idx", "key_cnt", "vis_cnt", "orig_idx", "g_out", "i_out", "s_out",
+        "kept_idx", "kept_cnt", "orig_out", "key_idx_out", "key_cnt_out", "hidden_out", "k_out", "v_out")]
 
 
 class MustDropError(RuntimeError):
@@ -83,6 +93,7 @@ def lib() -> ctypes.CDLL:
         L.mustdrop_score_static_max_rows.restype = ctypes.c_size_t
         L.mustdrop_compact.argtypes = [vp] * 11
         L.mustdrop_filter.argtypes = [vp] * 17
+        L.mustdrop_filter_layer.argtypes = [vp, ctypes.POINTER(mustdrop_layer_io_t), vp, vp]
         L.mustdrop_plan_filter_launches.argtypes = [vp]
         L.mustdrop_plan_filter_launches.restype = ctypes.c_int32
         L.mustdrop_device_status.argtypes = [vp, vp, vp, i32p, i32p]
@@ -92,7 +103,7 @@ def lib() -> ctypes.CDLL:
         L.mustdrop_plan_score_variant.argtypes = [vp]
         L.mustdrop_plan_score_variant.restype = ctypes.c_char_p
         for n in ("mustdrop_filter_plan", "mustdrop_plan_destroy", "mustdrop_score", "mustdrop_select",
-                  "mustdrop_compact", "mustdrop_filter", "mustdrop_device_status"):
+                  "mustdrop_compact", "mustdrop_filter", "mustdrop_filter_layer", "mustdrop_device_status"):
             getattr(L, n).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -135,7 +146,7 @@ class Config:
     gamma: float = 0.0
     alpha: float = 0.0
     key_max: int = 0
-    reserved: int = 0
+    flags: int = 0
     k_stride_b: int = 0
     k_stride_h: int = 0
     k_stride_l: int = 0
@@ -154,6 +165,13 @@ class Config:
     @property
     def cap(self) -> int:
         return self.budget if self.mode == MUSTDROP_MODE_BUDGET else self.n_vis
+
+    @property
+    def out_rows(self) -> int:
+        """Rows per request (and head) of the compacted outputs."""
+        if self.flags & MUSTDROP_FLAG_REBUILD_SEQUENCE:
+            return self.vis_start + self.cap + self.n_txt
+        return self.cap
 
 
 def mustdrop_filter_plan(config: Config) -> Tuple[int, int, int]:
@@ -202,6 +220,17 @@ def mustdrop_filter(plan, q_text, k, v, hidden, key_idx, key_cnt, g_out, i_out, 
                                  _ptr(hidden_out), _ptr(k_out), _ptr(v_out), _ptr(workspace), _stream(stream))
 
 
+def mustdrop_filter_layer(plan, workspace, stream=None, **tensors) -> int:
+    """Keyword arguments are the fields of mustdrop_layer_io_t (torch tensors, ints or None)."""
+    io = mustdrop_layer_io_t()
+    names = {n for n, _ in mustdrop_layer_io_t._fields_}
+    for n, t in tensors.items():
+        if n not in names:
+            raise TypeError("mustdrop_layer_io_t has no field %r" % n)
+        setattr(io, n, _ptr(t))
+    return lib().mustdrop_filter_layer(plan, ctypes.byref(io), _ptr(workspace), _stream(stream))
+
+
 def mustdrop_plan_filter_launches(plan) -> int:
     return lib().mustdrop_plan_filter_launches(plan)
 
@@ -235,6 +264,7 @@ class Filter:
         if st != MUSTDROP_OK:
             raise MustDropError(st, "mustdrop_filter_plan")
         B, M, H, cap = config.batch, config.n_vis, config.n_heads, config.cap
+        rows = config.out_rows
         self.device = torch.device(device)
         self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device=self.device)
         self.g = torch.empty((B, M), dtype=torch.float32, device=self.device)
@@ -242,9 +272,12 @@ class Filter:
         self.s = torch.empty((B, M), dtype=torch.float32, device=self.device)
         self.kept_idx = torch.full((B, cap), -1, dtype=torch.int32, device=self.device)
         self.kept_cnt = torch.zeros((B,), dtype=torch.int32, device=self.device)
-        self.hidden_out = torch.zeros((B, cap, config.hidden), dtype=torch.bfloat16, device=self.device)
-        self.k_out = torch.zeros((B, H, cap, config.head_dim), dtype=torch.bfloat16, device=self.device)
-        self.v_out = torch.zeros((B, H, cap, config.head_dim), dtype=torch.bfloat16, device=self.device)
+        self.hidden_out = torch.zeros((B, rows, config.hidden), dtype=torch.bfloat16, device=self.device)
+        self.k_out = torch.zeros((B, H, rows, config.head_dim), dtype=torch.bfloat16, device=self.device)
+        self.v_out = torch.zeros((B, H, rows, config.head_dim), dtype=torch.bfloat16, device=self.device)
+        self.orig_out = torch.full((B, cap), -1, dtype=torch.int32, device=self.device)
+        self.key_idx_out = torch.full((B, max(config.key_max, 1)), -1, dtype=torch.int32, device=self.device)
+        self.key_cnt_out = torch.zeros((B,), dtype=torch.int32, device=self.device)
 
     def close(self):
         if getattr(self, "plan", 0):
@@ -294,6 +327,19 @@ class Filter:
                                     self.hidden_out if hidden is not None else None, self.k_out,
                                     self.v_out if v is not None else None, self.workspace, stream),
                     "mustdrop_filter")
+        return self.hidden_out, self.k_out, self.v_out
+
+    def filter_layer(self, q_text, k, v, hidden, key_idx=None, key_cnt=None, vis_cnt=None, orig_idx=None,
+                     stream=None, want_s=False):
+        """One layer of a chain (ragged token counts, original ids, key positions for the next layer)."""
+        self._check(mustdrop_filter_layer(
+            self.plan, self.workspace, stream, q_text=q_text, k=k, v=v, hidden=hidden, key_idx=key_idx,
+            key_cnt=key_cnt, vis_cnt=vis_cnt, orig_idx=orig_idx, g_out=self.g, i_out=self.i,
+            s_out=self.s if want_s else None, kept_idx=self.kept_idx, kept_cnt=self.kept_cnt, orig_out=self.orig_out,
+            key_idx_out=self.key_idx_out if self.config.key_max > 0 else None,
+            key_cnt_out=self.key_cnt_out if self.config.key_max > 0 else None,
+            hidden_out=self.hidden_out if hidden is not None else None, k_out=self.k_out,
+            v_out=self.v_out if v is not None else None), "mustdrop_filter_layer")
         return self.hidden_out, self.k_out, self.v_out
 
     @property

@@ -38,11 +38,14 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   *workspace_bytes = 0;
   if (c->batch <= 0 || c->n_heads <= 0 || c->head_dim <= 0 || c->hidden <= 0 || c->seq_len <= 0 ||
       c->n_vis <= 0 || c->n_txt <= 0 || c->vis_start < 0 || c->txt_start < 0 || c->key_max < 0 ||
-      c->reserved != 0)
+      (c->flags & ~MUSTDROP_FLAG_REBUILD_SEQUENCE) != 0)
     return MUSTDROP_ERR_INVALID_ARG;
   // the vision span precedes the text span and both lie inside the sequence
   if (static_cast<int64_t>(c->vis_start) + c->n_vis > c->txt_start ||
       static_cast<int64_t>(c->txt_start) + c->n_txt > c->seq_len)
+    return MUSTDROP_ERR_INVALID_ARG;
+  if ((c->flags & MUSTDROP_FLAG_REBUILD_SEQUENCE) &&
+      (c->txt_start != c->vis_start + c->n_vis || c->seq_len != c->txt_start + c->n_txt))
     return MUSTDROP_ERR_INVALID_ARG;
   if (c->causal != 0 && c->causal != 1) return MUSTDROP_ERR_INVALID_ARG;
   if (c->mode != MUSTDROP_MODE_BUDGET && c->mode != MUSTDROP_MODE_THRESHOLD) return MUSTDROP_ERR_INVALID_ARG;
@@ -74,6 +77,10 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   r.causal = c->causal; r.mode = c->mode; r.criteria = c->criteria; r.budget = c->budget;
   r.key_max = c->key_max;
   r.cap = (c->mode == MUSTDROP_MODE_BUDGET) ? c->budget : c->n_vis;
+  r.rebuild = (c->flags & MUSTDROP_FLAG_REBUILD_SEQUENCE) ? 1 : 0;
+  r.out_rows = r.rebuild ? c->vis_start + r.cap + c->n_txt : r.cap;
+  r.gamma_default = c->gamma == 0.0f;
+  r.alpha_default = c->alpha == 0.0f;
   r.scale = (c->scale == 0.0f) ? 1.0f / sqrtf(static_cast<float>(c->head_dim)) : c->scale;
   r.scale_log2e = r.scale * 1.4426950408889634f;
   r.gamma = (c->gamma == 0.0f) ? 1.0f / static_cast<float>(c->n_vis) : c->gamma;
@@ -217,6 +224,53 @@ mustdrop_status_t mustdrop_filter(const mustdrop_plan_t* plan, const void* q_tex
   if (st != MUSTDROP_OK) return st;
   return mustdrop_compact(plan, kept_idx, kept_cnt, hidden, k_out != nullptr ? k : nullptr, v, hidden_out, k_out,
                           v_out, workspace, cuda_stream);
+}
+
+mustdrop_status_t mustdrop_filter_layer(const mustdrop_plan_t* plan, const mustdrop_layer_io_t* io, void* workspace,
+                                        void* cuda_stream) {
+  if (!valid_plan(plan) || io == nullptr) return MUSTDROP_ERR_INVALID_ARG;
+  if (io->q_text == nullptr || io->k == nullptr || io->g_out == nullptr || io->i_out == nullptr ||
+      io->kept_idx == nullptr || io->kept_cnt == nullptr)
+    return MUSTDROP_ERR_INVALID_ARG;
+  const mustdrop::Resolved& r = plan->r;
+  if (r.key_max > 0 && (io->key_idx == nullptr || io->key_cnt == nullptr)) return MUSTDROP_ERR_INVALID_ARG;
+  if ((io->hidden == nullptr) != (io->hidden_out == nullptr) || (io->v == nullptr) != (io->v_out == nullptr))
+    return MUSTDROP_ERR_INVALID_ARG;
+  if ((io->key_idx_out == nullptr) != (io->key_cnt_out == nullptr)) return MUSTDROP_ERR_INVALID_ARG;
+  // a ragged batch packs each request's text directly behind its own vision tokens
+  if (io->vis_cnt != nullptr && (r.txt_start != r.vis_start + r.M || r.L != r.txt_start + r.N))
+    return MUSTDROP_ERR_INVALID_ARG;
+  if (workspace == nullptr) return MUSTDROP_ERR_WORKSPACE;
+  const void* ptrs[] = {io->q_text, io->k, io->v, io->hidden, io->key_idx, io->key_cnt, io->vis_cnt, io->orig_idx,
+                        io->g_out, io->i_out, io->s_out, io->kept_idx, io->kept_cnt, io->orig_out, io->key_idx_out,
+                        io->key_cnt_out, io->hidden_out, io->k_out, io->v_out, workspace};
+  for (const void* q : ptrs)
+    if (q != nullptr && !aligned16(q)) return MUSTDROP_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  mustdrop::LayerArgs la;
+  la.vis_cnt = io->vis_cnt; la.orig_in = io->orig_idx; la.orig_out = io->orig_out;
+  la.key_idx_out = io->key_idx_out; la.key_cnt_out = io->key_cnt_out;
+  cudaError_t e;
+  if (plan->filter_single) {
+    e = mustdrop::launch_filter_fused(*plan, io->q_text, io->k, io->v, io->hidden, io->key_idx, io->key_cnt, io->g_out,
+                                      io->i_out, io->s_out, io->kept_idx, io->kept_cnt, io->hidden_out, io->k_out,
+                                      io->v_out, workspace, stream, la);
+    return e == cudaSuccess ? MUSTDROP_OK : cuda_fail(e);
+  }
+  if (plan->score_variant == mustdrop::kScoreFusedCluster) {
+    e = mustdrop::launch_score_fused(*plan, io->q_text, io->k, io->g_out, io->i_out, workspace, stream, la.vis_cnt);
+  } else {
+    void* rowstats = static_cast<unsigned char*>(workspace) + plan->ws_rowstats_off;
+    e = mustdrop::launch_score_two_pass(*plan, io->q_text, io->k, io->g_out, io->i_out, rowstats, stream, la.vis_cnt);
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = mustdrop::launch_select(*plan, io->g_out, io->i_out, io->key_idx, io->key_cnt, io->kept_idx, io->kept_cnt,
+                              io->s_out, workspace, stream, la);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (io->hidden_out == nullptr && io->k_out == nullptr && io->v_out == nullptr) return MUSTDROP_OK;
+  e = mustdrop::launch_compact(*plan, io->kept_idx, io->kept_cnt, io->hidden, io->k_out != nullptr ? io->k : nullptr,
+                               io->v, io->hidden_out, io->k_out, io->v_out, workspace, stream, la.vis_cnt);
+  return e == cudaSuccess ? MUSTDROP_OK : cuda_fail(e);
 }
 
 int32_t mustdrop_plan_filter_launches(const mustdrop_plan_t* plan) {

@@ -44,9 +44,24 @@ struct FilterGeometry {
 struct Resolved {
   int32_t B, H, D, hidden, L, vis_start, M, txt_start, N;
   int32_t causal, mode, criteria, budget, key_max, cap;
+  int32_t rebuild;        // outputs hold [prefix ; kept vision ; text] instead of the kept vision rows only
+  int32_t out_rows;       // rows per request (and head) of hidden_out / k_out / v_out
+  int32_t gamma_default, alpha_default;   // thresholds follow each request's own sizes (ragged batches)
   float scale, scale_log2e, gamma, alpha;
   int64_t k_sb, k_sh, k_sl, v_sb, v_sh, v_sl, hid_sb, hid_sl;
 };
+
+// Optional per-call arguments of a layer in a chain of pruning layers (all device pointers, all nullable).
+struct LayerArgs {
+  const int32_t* vis_cnt = nullptr;     // [B] vision tokens each request actually holds (<= n_vis)
+  const int32_t* orig_in = nullptr;     // [B, n_vis] original id of each current vision token (null: identity)
+  int32_t* orig_out = nullptr;          // [B, cap] original ids of the kept tokens
+  int32_t* key_idx_out = nullptr;       // [B, key_max] positions of the key tokens among the kept tokens
+  int32_t* key_cnt_out = nullptr;       // [B]
+};
+
+// Number of vision tokens of request b: the plan's n_vis, or vis_cnt[b] clamped to [1, n_vis].
+__host__ __device__ inline int32_t clamp_vis_cnt(int32_t v, int32_t M) { return v < 1 ? 1 : (v > M ? M : v); }
 
 }  // namespace mustdrop
 
@@ -70,21 +85,23 @@ constexpr uint32_t kPlanMagic = 0x4d445250u;  // "MDRP"
 
 // Each launcher enqueues on `stream` and returns the launch error (cudaGetLastError).
 cudaError_t launch_score_two_pass(const mustdrop_plan& p, const void* q_text, const void* k,
-                                  float* g_out, float* i_out, void* rowstats, cudaStream_t stream);
+                                  float* g_out, float* i_out, void* rowstats, cudaStream_t stream,
+                                  const int32_t* vis_cnt = nullptr);
 bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out);
 cudaError_t launch_score_fused(const mustdrop_plan& p, const void* q_text, const void* k, float* g_out,
-                               float* i_out, void* workspace, cudaStream_t stream);
+                               float* i_out, void* workspace, cudaStream_t stream, const int32_t* vis_cnt = nullptr);
 bool plan_filter_single(const Resolved& r, const FusedGeometry& geo, FilterGeometry* out);
 cudaError_t launch_filter_fused(const mustdrop_plan& p, const void* q_text, const void* k, const void* v,
                                 const void* hidden, const int32_t* key_idx, const int32_t* key_cnt, float* g_out,
                                 float* i_out, float* s_out, int32_t* kept_idx, int32_t* kept_cnt, void* hidden_out,
-                                void* k_out, void* v_out, void* workspace, cudaStream_t stream);
+                                void* k_out, void* v_out, void* workspace, cudaStream_t stream,
+                                const LayerArgs& la = LayerArgs());
 cudaError_t launch_select(const mustdrop_plan& p, const float* g, const float* i, const int32_t* key_idx,
                           const int32_t* key_cnt, int32_t* kept_idx, int32_t* kept_cnt, float* s_out,
-                          void* workspace, cudaStream_t stream);
+                          void* workspace, cudaStream_t stream, const LayerArgs& la = LayerArgs());
 cudaError_t launch_compact(const mustdrop_plan& p, const int32_t* kept_idx, const int32_t* kept_cnt,
                            const void* hidden, const void* k, const void* v, void* hidden_out, void* k_out,
-                           void* v_out, void* workspace, cudaStream_t stream);
+                           void* v_out, void* workspace, cudaStream_t stream, const int32_t* vis_cnt = nullptr);
 
 // Remember the cudaError_t of a failed runtime call for mustdrop_last_cuda_error (per thread).
 void set_last_cuda_error(cudaError_t e);

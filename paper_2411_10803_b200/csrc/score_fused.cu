@@ -55,6 +55,7 @@ struct FusedParams {
   float* g_out;
   float* i_out;
   void* workspace;
+  const int32_t* vis_cnt;             // [B] or null: vision tokens the request holds; its text keys follow them
   int32_t H, N, L, M, vis_start, txt_start, causal;
   int32_t cluster, tk, cpl, n_stage;  // CTAs per request, keys per CTA, columns per TMEM lane
   int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (= 2 * n_buf)
@@ -74,6 +75,7 @@ struct FilterTail {
   int32_t has_k, has_v;
   int32_t slot_bytes, n_slot;    // gather ring in dynamic shared memory
   int32_t vis_start;
+  int32_t rebuild, N, out_rows;  // rebuild: outputs are [prefix ; kept vision ; text] (out_rows rows per request)
 };
 
 // ---- small PTX wrappers ------------------------------------------------------------------------
@@ -310,6 +312,15 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   // warps wait just before they store g_out / i_out, which an earlier select may still be reading.
   pdl_launch_dependents();
   const uint32_t tmem_base = tmem_base_holder;
+  // This request's own sequence.  In a ragged batch the token count comes from an earlier
+  // kernel in the stream (the previous layer's selection), so it is read after the wait.
+  int Mb = p.M, Lb = p.L, txt_start = p.txt_start;
+  if (p.vis_cnt != nullptr) {
+    pdl_wait();
+    Mb = clamp_vis_cnt(p.vis_cnt[b], p.M);
+    txt_start = p.vis_start + Mb;
+    Lb = txt_start + p.N;
+  }
 
   if (warp >= kTmaWarp) {
     if (kRealloc) asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
@@ -385,8 +396,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const int total_chunks = p.cpl / kChunk;
     const int my_chunks = (total_chunks - g + kColGroups - 1) / kColGroups;   // chunks g, g+2, ... (uniform per warp)
     const int key_lane0 = static_cast<int>(rank) * p.tk + half * p.cpl;        // key of this lane's column 0
-    int lim = p.causal ? (p.txt_start + row + 1) : p.L;                        // keys below lim are visible
-    lim = (lim < p.L ? lim : p.L) - key_lane0;                                 // ... as a column count of this lane
+    int lim = p.causal ? (txt_start + row + 1) : Lb;                           // keys below lim are visible
+    lim = (lim < Lb ? lim : Lb) - key_lane0;                                   // ... as a column count of this lane
     const bool all_visible = lim >= p.cpl;
     const bool sender = (half == 0);           // with two halves, lanes s and s+16 share a row: the lower one sends
     const uint32_t pair_idx = (rank * NROWS + row) * EPR + g;                  // this thread's pair in a slot
@@ -562,8 +573,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           s += v;
           mx = fmaxf(mx, v);
         }
-        p.g_out[static_cast<size_t>(b) * p.M + j] = s * p.inv_heads;
-        p.i_out[static_cast<size_t>(b) * p.M + j] = mx * p.inv_heads;
+        const bool present = j < Mb;    // beyond the request's own tokens: zeros
+        p.g_out[static_cast<size_t>(b) * p.M + j] = present ? s * p.inv_heads : 0.0f;
+        p.i_out[static_cast<size_t>(b) * p.M + j] = present ? mx * p.inv_heads : 0.0f;
       }
     }
   }
@@ -618,19 +630,32 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       fence_proxy_async();   // earlier generic-proxy accesses to the slots precede the async-proxy writes
       const int total = kept_total_s < ft.sel.cap ? kept_total_s : ft.sel.cap;
       const int C = p.cluster;
-      const int n_mine = total > static_cast<int>(rank) ? (total - static_cast<int>(rank) + C - 1) / C : 0;
+      // items: the kept vision rows, then (rebuild) the prefix rows and the request's text rows
+      const int n_items = total + (ft.rebuild ? ft.vis_start + ft.N : 0);
+      const int n_mine = n_items > static_cast<int>(rank) ? (n_items - static_cast<int>(rank) + C - 1) / C : 0;
       const int S = ft.n_slot, ahead = S - 2;
       const uint32_t ring = stage_base + kKeptListBytes;
       const uint32_t payload = static_cast<uint32_t>(ft.hidden_bytes) + static_cast<uint32_t>(ft.has_k + ft.has_v) * ft.kv_bytes;
       const uint64_t once = l2_evict_first_policy();
+      // item -> (source row, destination row)
+      auto src_row = [&](int it) {
+        if (it < total) return ft.vis_start + kept_list[it];
+        const int x = it - total;
+        return x < ft.vis_start ? x : ft.vis_start + Mb + (x - ft.vis_start);
+      };
+      auto dst_row = [&](int it) {
+        if (!ft.rebuild) return it;
+        if (it < total) return ft.vis_start + it;
+        const int x = it - total;
+        return x < ft.vis_start ? x : ft.vis_start + total + (x - ft.vis_start);
+      };
       bool ok = true;
       int loaded = 0;
       for (int i = 0; i < n_mine + ahead && ok; ++i) {
         if (i < n_mine) {
           const int slot = i % S;
-          if (i >= S) bulk_wait_read_1();   // the stores of row i - S have finished reading the slot
-          const int r = static_cast<int>(rank) + i * C;
-          const int row = ft.vis_start + kept_list[r];
+          if (i >= S) bulk_wait_read_1();   // the stores of item i - S have finished reading the slot
+          const int row = src_row(static_cast<int>(rank) + i * C);
           const uint32_t bar = smem_u32(&bars.gfull[slot]);
           uint32_t dst = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
           mbar_expect_tx(bar, payload);
@@ -649,10 +674,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         if (c >= 0) {
           const int slot = c % S;
           if (!mbar_wait(smem_u32(&bars.gfull[slot]), static_cast<uint32_t>(c / S) & 1u, abort_flag)) { ok = false; break; }
-          const int r = static_cast<int>(rank) + c * C;
+          const int r = dst_row(static_cast<int>(rank) + c * C);
           uint32_t src = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
           if (ft.hidden_bytes > 0) {
-            bulk_store_1d(ft.hidden_out + (static_cast<int64_t>(b) * ft.sel.cap + r) * ft.hidden_bytes, src, ft.hidden_bytes);
+            bulk_store_1d(ft.hidden_out + (static_cast<int64_t>(b) * ft.out_rows + r) * ft.hidden_bytes, src, ft.hidden_bytes);
             src += ft.hidden_pad;
           }
           if (ft.has_k) {
@@ -827,7 +852,7 @@ namespace {
 // Common launch of the score kernel, with (tail != nullptr) or without the selection / gather tail.
 cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, const void* k, float* g_out,
                                 float* i_out, void* workspace, const GatherMaps* maps, const FilterTail* tail,
-                                size_t smem_bytes, cudaStream_t stream) {
+                                size_t smem_bytes, cudaStream_t stream, const int32_t* vis_cnt) {
   const Resolved& r = plan.r;
   const FusedGeometry& geo = plan.fused;
   const int nrows = 128 / geo.halves;
@@ -839,6 +864,7 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, c
     return cudaErrorInvalidValue;
   FusedParams p;
   p.g_out = g_out; p.i_out = i_out; p.workspace = workspace;
+  p.vis_cnt = vis_cnt;
   p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
   p.causal = r.causal;
   p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_stage = geo.n_stage;
@@ -872,8 +898,9 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, c
 }  // namespace
 
 cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, const void* k, float* g_out,
-                               float* i_out, void* workspace, cudaStream_t stream) {
-  return launch_fused_common(plan, q_text, k, g_out, i_out, workspace, nullptr, nullptr, plan.fused.smem_bytes, stream);
+                               float* i_out, void* workspace, cudaStream_t stream, const int32_t* vis_cnt) {
+  return launch_fused_common(plan, q_text, k, g_out, i_out, workspace, nullptr, nullptr, plan.fused.smem_bytes, stream,
+                             vis_cnt);
 }
 
 // Shared-memory plan of the gather tail; false when a row does not fit the ring at least three times.
@@ -899,25 +926,30 @@ bool plan_filter_single(const Resolved& r, const FusedGeometry& geo, FilterGeome
 cudaError_t launch_filter_fused(const mustdrop_plan& plan, const void* q_text, const void* k, const void* v,
                                 const void* hidden, const int32_t* key_idx, const int32_t* key_cnt, float* g_out,
                                 float* i_out, float* s_out, int32_t* kept_idx, int32_t* kept_cnt, void* hidden_out,
-                                void* k_out, void* v_out, void* workspace, cudaStream_t stream) {
+                                void* k_out, void* v_out, void* workspace, cudaStream_t stream, const LayerArgs& la) {
   const Resolved& r = plan.r;
   GatherMaps maps = {};
-  const uint64_t out_s1 = 256, out_s2 = static_cast<uint64_t>(r.cap) * 256, out_s3 = static_cast<uint64_t>(r.H) * out_s2;
+  const uint64_t out_s1 = 256, out_s2 = static_cast<uint64_t>(r.out_rows) * 256, out_s3 = static_cast<uint64_t>(r.H) * out_s2;
   if (k_out != nullptr &&
       (!make_gather_map(&maps.k_src, k, r.L, r.H, r.B, static_cast<uint64_t>(r.k_sl) * 2,
                         static_cast<uint64_t>(r.k_sh) * 2, static_cast<uint64_t>(r.k_sb) * 2) ||
-       !make_gather_map(&maps.k_dst, k_out, r.cap, r.H, r.B, out_s1, out_s2, out_s3)))
+       !make_gather_map(&maps.k_dst, k_out, r.out_rows, r.H, r.B, out_s1, out_s2, out_s3)))
     return cudaErrorInvalidValue;
   if (v_out != nullptr &&
       (!make_gather_map(&maps.v_src, v, r.L, r.H, r.B, static_cast<uint64_t>(r.v_sl) * 2,
                         static_cast<uint64_t>(r.v_sh) * 2, static_cast<uint64_t>(r.v_sb) * 2) ||
-       !make_gather_map(&maps.v_dst, v_out, r.cap, r.H, r.B, out_s1, out_s2, out_s3)))
+       !make_gather_map(&maps.v_dst, v_out, r.out_rows, r.H, r.B, out_s1, out_s2, out_s3)))
     return cudaErrorInvalidValue;
   FilterTail t = {};
   t.sel.g = g_out; t.sel.i = i_out; t.sel.key_idx = key_idx; t.sel.key_cnt = key_cnt;
   t.sel.kept_idx = kept_idx; t.sel.kept_cnt = kept_cnt; t.sel.s_out = s_out; t.sel.workspace = workspace;
   t.sel.M = r.M; t.sel.key_max = r.key_max; t.sel.mode = r.mode; t.sel.criteria = r.criteria;
   t.sel.budget = r.budget; t.sel.cap = r.cap; t.sel.gamma = r.gamma; t.sel.alpha = r.alpha;
+  t.sel.vis_cnt = la.vis_cnt; t.sel.orig_in = la.orig_in; t.sel.orig_out = la.orig_out;
+  t.sel.key_idx_out = la.key_idx_out; t.sel.key_cnt_out = la.key_cnt_out;
+  t.sel.vis_start = r.vis_start; t.sel.N = r.N;
+  t.sel.gamma_default = r.gamma_default; t.sel.alpha_default = r.alpha_default;
+  t.rebuild = r.rebuild; t.N = r.N; t.out_rows = r.out_rows;
   t.hidden = static_cast<const unsigned char*>(hidden);
   t.hidden_out = static_cast<unsigned char*>(hidden_out);
   t.hid_sb = r.hid_sb * 2; t.hid_sl = r.hid_sl * 2;
@@ -927,7 +959,8 @@ cudaError_t launch_filter_fused(const mustdrop_plan& plan, const void* q_text, c
   t.has_k = k_out != nullptr; t.has_v = v_out != nullptr;
   t.slot_bytes = plan.filter.slot_bytes; t.n_slot = plan.filter.n_slot;
   t.vis_start = r.vis_start;
-  return launch_fused_common(plan, q_text, k, g_out, i_out, workspace, &maps, &t, plan.filter.smem_bytes, stream);
+  return launch_fused_common(plan, q_text, k, g_out, i_out, workspace, &maps, &t, plan.filter.smem_bytes, stream,
+                             la.vis_cnt);
 }
 
 }  // namespace mustdrop

@@ -26,6 +26,7 @@ struct ScoreParams {
   float2* rowstats;         // [B,H,N]
   float* g_out;             // [B,M]
   float* i_out;             // [B,M]
+  const int32_t* vis_cnt;   // [B] or null: vision tokens the request holds; its text keys follow them
   int32_t H, N, L, M, vis_start, txt_start, causal, n_warps;
   float scale_log2e, inv_heads;
   int64_t k_sb, k_sh, k_sl;
@@ -97,18 +98,21 @@ __global__ void __launch_bounds__(256) rowstats_kernel(ScoreParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int n_threads = blockDim.x;
   pdl_wait();   // the row-statistics scratch may still be read by an earlier launch
+  // this request's own sequence: its text keys follow its vision tokens
+  const int txt_start = p.vis_cnt ? p.vis_start + clamp_vis_cnt(p.vis_cnt[b], p.M) : p.txt_start;
+  const int L = p.vis_cnt ? txt_start + p.N : p.L;
   const __nv_bfloat16* qg = p.q + (static_cast<int64_t>(b) * p.H + h) * p.N * kHeadDim;
   const __nv_bfloat16* kg = p.k + b * p.k_sb + h * p.k_sh;
-  const int n_tiles = (p.L + kTileKeys - 1) / kTileKeys;
+  const int n_tiles = (L + kTileKeys - 1) / kTileKeys;
 
   stage_rows(q_s, qg, kHeadDim, n_rows, p.N, n_threads);
-  stage_rows(k_s0, kg, p.k_sl, kTileKeys, p.L, n_threads);
+  stage_rows(k_s0, kg, p.k_sl, kTileKeys, L, n_threads);
   cp_async_commit();
 
   const int row0 = warp * 16 + g, row1 = row0 + 8;
   // last visible key of each of this thread's two text rows
-  const int last0 = p.causal ? p.txt_start + row0 : p.L - 1;
-  const int last1 = p.causal ? p.txt_start + row1 : p.L - 1;
+  const int last0 = p.causal ? txt_start + row0 : L - 1;
+  const int last1 = p.causal ? txt_start + row1 : L - 1;
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.0f, l1 = 0.0f;
   uint32_t a[8][4];
 
@@ -117,7 +121,7 @@ __global__ void __launch_bounds__(256) rowstats_kernel(ScoreParams p) {
     __nv_bfloat16* nxt = (tile & 1) ? k_s0 : k_s1;
     if (tile + 1 < n_tiles) {
       const int base = (tile + 1) * kTileKeys;
-      stage_rows(nxt, kg + static_cast<int64_t>(base) * p.k_sl, p.k_sl, kTileKeys, p.L - base, n_threads);
+      stage_rows(nxt, kg + static_cast<int64_t>(base) * p.k_sl, p.k_sl, kTileKeys, L - base, n_threads);
       cp_async_commit();
       cp_async_wait<1>();
     } else {
@@ -134,8 +138,8 @@ __global__ void __launch_bounds__(256) rowstats_kernel(ScoreParams p) {
       const int key = key_base + nb * 8 + 2 * t;
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        z[nb][e] = (key + e <= last0 && key + e < p.L) ? z[nb][e] * p.scale_log2e : -INFINITY;
-        z[nb][2 + e] = (key + e <= last1 && key + e < p.L) ? z[nb][2 + e] * p.scale_log2e : -INFINITY;
+        z[nb][e] = (key + e <= last0 && key + e < L) ? z[nb][e] * p.scale_log2e : -INFINITY;
+        z[nb][2 + e] = (key + e <= last1 && key + e < L) ? z[nb][2 + e] * p.scale_log2e : -INFINITY;
         tmax0 = fmaxf(tmax0, z[nb][e]);
         tmax1 = fmaxf(tmax1, z[nb][2 + e]);
       }
@@ -189,7 +193,8 @@ __global__ void __launch_bounds__(256) accumulate_kernel(ScoreParams p) {
   const int n_threads = blockDim.x;
   pdl_wait();
   const int j_base = vt * kTileKeys;            // first vision token of this tile
-  const int valid_keys = p.M - j_base;          // rows of the tile that exist
+  const int Mb = p.vis_cnt ? clamp_vis_cnt(p.vis_cnt[b], p.M) : p.M;
+  const int valid_keys = Mb - j_base;           // rows of the tile that exist (<= 0: none, zeros are stored)
   const __nv_bfloat16* qg = p.q + static_cast<int64_t>(b) * p.H * p.N * kHeadDim;
   const __nv_bfloat16* kg = p.k + b * p.k_sb + static_cast<int64_t>(p.vis_start + j_base) * p.k_sl;
   const float2* stats = p.rowstats + static_cast<int64_t>(b) * p.H * p.N;
@@ -256,12 +261,13 @@ __global__ void __launch_bounds__(256) accumulate_kernel(ScoreParams p) {
   }
   __syncthreads();
   for (int col = threadIdx.x; col < kTileKeys; col += n_threads) {
-    if (col >= valid_keys) continue;
+    if (j_base + col >= p.M) continue;
     float s = 0.0f, mx = -INFINITY;
     for (int w = 0; w < p.n_warps; ++w) {
       s += red[w * kTileKeys + col];
       mx = fmaxf(mx, red[(p.n_warps + w) * kTileKeys + col]);
     }
+    if (col >= valid_keys) s = mx = 0.0f;   // beyond the request's own tokens
     p.g_out[static_cast<int64_t>(b) * p.M + j_base + col] = s * p.inv_heads;
     p.i_out[static_cast<int64_t>(b) * p.M + j_base + col] = mx * p.inv_heads;
   }
@@ -270,13 +276,14 @@ __global__ void __launch_bounds__(256) accumulate_kernel(ScoreParams p) {
 }  // namespace
 
 cudaError_t launch_score_two_pass(const mustdrop_plan& plan, const void* q_text, const void* k, float* g_out,
-                                  float* i_out, void* rowstats, cudaStream_t stream) {
+                                  float* i_out, void* rowstats, cudaStream_t stream, const int32_t* vis_cnt) {
   const Resolved& r = plan.r;
   ScoreParams p;
   p.q = static_cast<const __nv_bfloat16*>(q_text);
   p.k = static_cast<const __nv_bfloat16*>(k);
   p.rowstats = static_cast<float2*>(rowstats);
   p.g_out = g_out; p.i_out = i_out;
+  p.vis_cnt = vis_cnt;
   p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
   p.causal = r.causal;
   p.n_warps = (r.N + 15) / 16;

@@ -33,13 +33,16 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
 
 cudaError_t launch_select(const mustdrop_plan& plan, const float* g, const float* i, const int32_t* key_idx,
                           const int32_t* key_cnt, int32_t* kept_idx, int32_t* kept_cnt, float* s_out,
-                          void* workspace, cudaStream_t stream) {
+                          void* workspace, cudaStream_t stream, const LayerArgs& la) {
   const Resolved& r = plan.r;
   SelectParams p;
   p.g = g; p.i = i; p.key_idx = key_idx; p.key_cnt = key_cnt; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt;
   p.s_out = s_out; p.workspace = workspace;
   p.M = r.M; p.key_max = r.key_max; p.mode = r.mode; p.criteria = r.criteria; p.budget = r.budget; p.cap = r.cap;
   p.gamma = r.gamma; p.alpha = r.alpha;
+  p.vis_cnt = la.vis_cnt; p.orig_in = la.orig_in; p.orig_out = la.orig_out;
+  p.key_idx_out = la.key_idx_out; p.key_cnt_out = la.key_cnt_out;
+  p.vis_start = r.vis_start; p.N = r.N; p.gamma_default = r.gamma_default; p.alpha_default = r.alpha_default;
   const int own = (r.M + kSelThreads - 1) / kSelThreads;
   static_assert(kMaxOwn == 16, "dispatch below covers up to 16 tokens per thread");
   if (own <= 1) return launch_pdl(select_kernel<1>, dim3(r.B), dim3(kSelThreads), 0, stream, p);

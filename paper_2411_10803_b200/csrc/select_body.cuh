@@ -32,6 +32,15 @@ struct SelectParams {
   void* workspace;
   int32_t M, key_max, mode, criteria, budget, cap;
   float gamma, alpha;
+  // a layer in a chain of pruning layers (all nullable): per-request token counts, original ids
+  // in and out, and the key tokens' positions among the kept tokens
+  const int32_t* vis_cnt;
+  const int32_t* orig_in;
+  int32_t* orig_out;
+  int32_t* key_idx_out;
+  int32_t* key_cnt_out;
+  int32_t vis_start, N;                   // this request's sequence length = vis_start + its tokens + N
+  int32_t gamma_default, alpha_default;   // 1: gamma = 1 / (the request's tokens), alpha = 2 / (its length)
 };
 
 struct SelectShared {
@@ -110,11 +119,17 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
   constexpr int own = OWN;
   static_assert(kSelThreads == 256, "one thread per radix bin");
   const int lane = tid & 31, warp = tid >> 5;
-  const int M = p.M;
+  const int ld = p.M;                                    // row length of g / i / s_out / orig_in
+  const int M = p.vis_cnt ? clamp_vis_cnt(p.vis_cnt[b], p.M) : p.M;   // this request's tokens
   const int j0 = tid * own;                              // this thread's first token
+  float gamma = p.gamma, alpha = p.alpha;
+  if (p.vis_cnt != nullptr) {                            // thresholds that default follow the request's own sizes
+    if (p.gamma_default) gamma = __fdiv_rn(1.0f, static_cast<float>(M));
+    if (p.alpha_default) alpha = __fdiv_rn(2.0f, static_cast<float>(p.vis_start + M + p.N));
+  }
 
-  const float* g = p.g + static_cast<size_t>(b) * M;
-  const float* in = p.i + static_cast<size_t>(b) * M;
+  const float* g = p.g + static_cast<size_t>(b) * ld;
+  const float* in = p.i + static_cast<size_t>(b) * ld;
   // the key-set loads are issued first so that their latency overlaps the score loads
   int key_c = 0, key_j = -1;
   if (p.key_max > 0) {
@@ -155,7 +170,7 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
 #pragma unroll
   for (int w = 0; w < kSelWarps; ++w) tsum += s.dsum[w];
   const float T = static_cast<float>(tsum);
-  const float gt = __fmul_rn(p.gamma, T);
+  const float gt = __fmul_rn(gamma, T);
 
   // scores of the thread's tokens, as ordered integers
   uint32_t u[kOwn];
@@ -165,13 +180,13 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
     u[e] = 0u;
     if (e < own && j < M) {
       const float gj = __fdiv_rn(gv[e], gt);
-      const float rj = __fdiv_rn(iv[e], p.alpha);
+      const float rj = __fdiv_rn(iv[e], alpha);
       float sc;
       if (p.criteria == MUSTDROP_CRIT_GLOBAL_ONLY) sc = gj;
       else if (p.criteria == MUSTDROP_CRIT_INDIVIDUAL_ONLY) sc = rj;
       else sc = (gj > rj) ? gj : rj;
       u[e] = ordered_bits(sc);
-      if (write_out && p.s_out != nullptr) p.s_out[static_cast<size_t>(b) * M + j] = sc;
+      if (write_out && p.s_out != nullptr) p.s_out[static_cast<size_t>(b) * ld + j] = sc;
     }
   }
   SEL_STAMP(4);
@@ -195,7 +210,7 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
     for (int e = 0; e < kOwn; ++e) {
       if ((valid >> e) & 1u) {
         const bool in_d = gv[e] <= gt;            // Eq. 9
-        const bool small = iv[e] < p.alpha;       // Eq. 10
+        const bool small = iv[e] < alpha;         // Eq. 10
         bool drop;
         if (p.criteria == MUSTDROP_CRIT_GLOBAL_ONLY) drop = in_d;
         else if (p.criteria == MUSTDROP_CRIT_INDIVIDUAL_ONLY) drop = small;
@@ -287,19 +302,34 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
   // index-ordered emit
   int total;
   int pos = group_exclusive_scan<Sync>(__popc(keep), tid, s.warp, &total);
+  // a chain of layers also wants the kept tokens' original ids and where the key tokens went
+  const bool emit_keys = p.key_idx_out != nullptr && p.key_max > 0;   // uniform over the group
+  int key_pos = 0, key_total = 0;
+  if (emit_keys) key_pos = group_exclusive_scan<Sync>(__popc(key & keep), tid, s.warp, &key_total);
   int32_t* out = p.kept_idx + static_cast<size_t>(b) * p.cap;
 #pragma unroll
   for (int e = 0; e < kOwn; ++e) {
     if ((keep >> e) & 1u) {
       if (pos < p.cap) {
-        if (write_out) out[pos] = j0 + e;
+        if (write_out) {
+          out[pos] = j0 + e;
+          if (p.orig_out != nullptr)
+            p.orig_out[static_cast<size_t>(b) * p.cap + pos] =
+                p.orig_in != nullptr ? p.orig_in[static_cast<size_t>(b) * ld + j0 + e] : j0 + e;
+          if (emit_keys && ((key >> e) & 1u) && key_pos < p.key_max)
+            p.key_idx_out[static_cast<size_t>(b) * p.key_max + key_pos] = pos;
+        }
         if (kept_list != nullptr) kept_list[pos] = j0 + e;
       }
+      if ((key >> e) & 1u) ++key_pos;
       ++pos;
     }
   }
   if (tid == 0) {
-    if (write_out) p.kept_cnt[b] = total;
+    if (write_out) {
+      p.kept_cnt[b] = total;
+      if (p.key_cnt_out != nullptr) p.key_cnt_out[b] = emit_keys ? (key_total < p.key_max ? key_total : p.key_max) : 0;
+    }
     if (kept_total != nullptr) *kept_total = total;
   }
 }

@@ -1,0 +1,185 @@
+"""GPU parity of a pruning layer on a ragged batch and of a chain of pruning layers
+(mustdrop_filter_layer) against the CPU oracle of oracle/layers.py."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import layers
+from paper_2411_10803_b200 import binding as md
+from paper_2411_10803_b200 import build as md_build
+from paper_2411_10803_b200 import synth
+
+from parity_util import assert_kept_matches, assert_scores_close, bf16_bits, to_dev, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+TINY = synth.WORKLOADS["c1_tiny"]
+
+PATHS = ["one_launch", "three_launches", "two_pass"]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    md_build.build()
+    assert torch.cuda.is_available()
+
+
+@pytest.fixture
+def path(request, monkeypatch):
+    for n in ("MUSTDROP_SCORE_VARIANT", "MUSTDROP_CLUSTER", "MUSTDROP_FILTER"):
+        monkeypatch.delenv(n, raising=False)
+    if request.param == "three_launches":
+        monkeypatch.setenv("MUSTDROP_FILTER", "staged")
+    elif request.param == "two_pass":
+        monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "two_pass")
+    return request.param
+
+
+def small(**kw):
+    base = dict(batch=4, n_vis=300, n_txt=19, n_heads=3, hidden=384, n_salient=3, key_cnt=6, budget=48, vis_start=3)
+    base.update(kw)
+    return TINY.with_(**base)
+
+
+def check_layer(f, w, p, ref, rebuild, sample=None):
+    """Compare one layer's GPU results (in Filter f) with the oracle's dict `ref`; p = the inputs."""
+    sample = range(w.batch) if sample is None else sample
+    sel = np.array(list(sample))
+    g, i = f.g.cpu().numpy(), f.i.cpu().numpy()
+    idx, cnt = f.kept_idx.cpu().numpy(), f.kept_cnt.cpu().numpy()
+    orig = f.orig_out.cpu().numpy()
+    ho, ko, vo = bf16_bits(f.hidden_out), bf16_bits(f.k_out), bf16_bits(f.v_out)
+    assert_scores_close(g[sel], ref["G"], "G")
+    assert_scores_close(i[sel], ref["I"], "I")
+    for n, b in enumerate(sel):
+        m = int(p["vis_cnt"][b])
+        assert not g[b, m:].any() and not i[b, m:].any()          # absent tokens score 0
+    kidx = p["key_idx"][sel] if w.key_cnt else None
+    kcnt = p["key_cnt"][sel] if w.key_cnt else None
+    swapped = assert_kept_matches(idx[sel], cnt[sel], ref["kept_idx"], ref["kept_cnt"], ref["s"], kidx, kcnt)
+    vs, N = w.vis_start, w.n_txt
+    for n, b in enumerate(sel):
+        c, m = int(cnt[b]), int(p["vis_cnt"][b])
+        src = p["orig_idx"][b] if "orig_idx" in p else np.arange(w.n_vis)
+        assert np.array_equal(orig[b, :c], src[idx[b, :c]])        # original ids of the kept tokens
+        rows = vs + idx[b, :c]
+        if rebuild:
+            rows = np.concatenate([np.arange(vs), rows, vs + m + np.arange(N)])
+        assert np.array_equal(ho[b, :len(rows)], p["hidden"][b, rows])
+        assert np.array_equal(ko[b][:, :len(rows)], p["k"][b][:, rows])
+        assert np.array_equal(vo[b][:, :len(rows)], p["v"][b][:, rows])
+        assert not ho[b, len(rows):].any() and not ko[b][:, len(rows):].any()   # nothing written behind the end
+        if w.key_cnt:
+            kc = int(p["key_cnt"][b])
+            pos = [int(np.nonzero(idx[b, :c] == j)[0][0]) for j in sorted(p["key_idx"][b, :kc].tolist())]
+            assert f.key_cnt_out.cpu().numpy()[b] == kc
+            assert f.key_idx_out.cpu().numpy()[b, :kc].tolist() == pos
+    if swapped == 0:
+        assert np.array_equal(orig[sel], ref["orig_out"])
+        assert np.array_equal(ho[sel], ref["hidden_out"]) and np.array_equal(ko[sel], ref["k_out"])
+        assert np.array_equal(vo[sel], ref["v_out"])
+    return swapped
+
+
+def run_ragged_layer(w, vis_cnt, rebuild, sample=None, with_orig=False):
+    d = synth.make_batch(w)
+    p = synth.pack_ragged(d, w, vis_cnt)
+    if with_orig:
+        p["orig_idx"] = (np.arange(w.n_vis, dtype=np.int32)[None, :] * 3 + 1).repeat(w.batch, 0)
+    f = md.Filter(md.config_for(w, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE if rebuild else 0))
+    q, k, v, hid = (to_dev_bf16(p[n]) for n in ("q_text", "k", "v", "hidden"))
+    ki, kc = (to_dev(p["key_idx"]), to_dev(p["key_cnt"])) if w.key_cnt else (None, None)
+    f.filter_layer(q, k, v, hid, ki, kc, vis_cnt=to_dev(p["vis_cnt"]),
+                   orig_idx=to_dev(p["orig_idx"]) if with_orig else None, want_s=True)
+    torch.cuda.synchronize()
+    assert f.device_status() == (0, 0)
+    sel = list(range(w.batch)) if sample is None else sample
+    ref = layers.filter_layer_ragged(p["q_text"][sel], p["k"][sel], p["v"][sel], p["hidden"][sel], w.vis_start,
+                                     p["vis_cnt"][sel], w.budget, p["key_idx"][sel] if w.key_cnt else None,
+                                     p["key_cnt"][sel] if w.key_cnt else None,
+                                     orig_idx=p["orig_idx"][sel] if with_orig else None, rebuild=rebuild)
+    check_layer(f, w, p, ref, rebuild, sel)
+    launches = f.filter_launches
+    f.close()
+    return launches
+
+
+@pytest.mark.parametrize("path", PATHS, indirect=True)
+@pytest.mark.parametrize("rebuild", [False, True])
+def test_ragged_layer_matches_oracle(path, rebuild):
+    w = small()
+    launches = run_ragged_layer(w, np.array([300, 48, 131, 17], np.int32), rebuild, with_orig=rebuild)
+    assert launches == {"one_launch": 1, "three_launches": 3, "two_pass": 4}[path]
+
+
+@pytest.mark.parametrize("path", PATHS, indirect=True)
+def test_ragged_layer_without_key_set_many_text_rows(path):
+    w = small(batch=3, n_vis=200, n_txt=100, n_heads=2, hidden=256, key_cnt=0, budget=30, vis_start=0)
+    run_ragged_layer(w, np.array([200, 30, 97], np.int32), True)
+
+
+def test_ragged_layer_llava7b_batch16_sampled():
+    w = synth.WORKLOADS["c2_llava7b_b16"]
+    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[0, 11]) == 1
+
+
+def test_ragged_layer_next7b_falls_back():
+    w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
+    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[1]) == 4
+
+
+@pytest.mark.parametrize("path", ["one_launch", "two_pass"], indirect=True)
+def test_chain_of_three_layers_matches_oracle(path):
+    w = small(batch=4, n_vis=320, key_cnt=5, n_txt=16, budget=0)
+    budgets, caps = [128, 64, 24], [320, 128, 64]
+    vis_cnt0 = np.array([320, 100, 251, 77], np.int32)
+    cnts = [vis_cnt0]
+    for kp in budgets[:-1]:
+        cnts.append(np.minimum(cnts[-1], kp))
+    d0 = synth.make_batch(w.with_(key_cnt=5))
+    key_idx, key_cnt = np.minimum(d0["key_idx"], 70), d0["key_cnt"].copy()
+    for b in range(w.batch):                      # distinct keys below the shortest request
+        ks = sorted(set(key_idx[b].tolist()))
+        key_idx[b] = -1
+        key_idx[b, :len(ks)], key_cnt[b] = ks, len(ks)
+    tensors = []
+    for l, (cap, cnt) in enumerate(zip(caps, cnts)):
+        wl = w.with_(n_vis=cap, seed=w.seed + 100 * (l + 1), key_cnt=0, n_salient=3)
+        tensors.append(synth.pack_ragged(synth.make_batch(wl), wl, cnt))
+    ref = layers.progressive_filter(tensors, w.vis_start, vis_cnt0, budgets, key_idx, key_cnt)
+
+    # the GPU chain: every layer's outputs feed the next, no host synchronisation in between
+    filters, dev = [], []
+    for l, (cap, kp) in enumerate(zip(caps, budgets)):
+        wl = w.with_(n_vis=cap, budget=kp)
+        filters.append(md.Filter(md.config_for(wl, key_max=5, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE)))
+        dev.append([to_dev_bf16(tensors[l][n]) for n in ("q_text", "k", "v", "hidden")])
+    ki, kc, vc, orig = to_dev(key_idx), to_dev(key_cnt), to_dev(vis_cnt0), None
+    for l, f in enumerate(filters):
+        q, k, v, hid = dev[l]
+        f.filter_layer(q, k, v, hid, ki, kc, vis_cnt=vc, orig_idx=orig)
+        ki, kc, vc, orig = f.key_idx_out, f.key_cnt_out, f.kept_cnt, f.orig_out
+    torch.cuda.synchronize()
+    for l, f in enumerate(filters):
+        assert f.device_status() == (0, 0)
+        r = ref[l]
+        idx, cnt = f.kept_idx.cpu().numpy(), f.kept_cnt.cpu().numpy()
+        assert_scores_close(f.g.cpu().numpy(), r["G"], "G layer %d" % l)
+        swapped = assert_kept_matches(idx, cnt, r["kept_idx"], r["kept_cnt"], r["s"], r["key_idx"], r["key_cnt"])
+        assert swapped == 0, "a near-tie at layer %d: later layers cannot be compared" % l
+        assert np.array_equal(f.orig_out.cpu().numpy(), r["orig_out"])
+        assert np.array_equal(bf16_bits(f.hidden_out), r["hidden_out"])
+        assert np.array_equal(bf16_bits(f.k_out), r["k_out"]) and np.array_equal(bf16_bits(f.v_out), r["v_out"])
+        if l + 1 < len(filters):
+            nk = ref[l + 1]["key_cnt"]
+            assert np.array_equal(f.key_cnt_out.cpu().numpy(), nk)
+            for b in range(w.batch):
+                assert np.array_equal(f.key_idx_out.cpu().numpy()[b, :nk[b]], ref[l + 1]["key_idx"][b, :nk[b]])
+    # S_few: what the last layer kept, in original ids, is inside every earlier layer's set
+    s_few = filters[-1].orig_out.cpu().numpy()
+    for b in range(w.batch):
+        last = set(s_few[b, :filters[-1].kept_cnt.cpu().numpy()[b]].tolist())
+        for f in filters:
+            assert last <= set(f.orig_out.cpu().numpy()[b].tolist())
+    for f in filters:
+        f.close()
