@@ -244,6 +244,33 @@ typedef struct {
 mustdrop_status_t mustdrop_filter_layer(const mustdrop_plan_t *plan, const mustdrop_layer_io_t *io /* (host) */,
                                         void *workspace, void *cuda_stream);
 
+/*
+ * Decoding-stage cache compaction (Sec. 3.5, output-aware cache policy: the layers following
+ * the second one keep, of the vision tokens, only S_few - the tokens still retained after the
+ * last pruning layer).  One launch rebuilds the K and V caches of n_layers such layers.
+ *   k_cache, v_cache bf16 [n_layers, B, H, rows_in, D] contiguous: layer y of request b holds
+ *       vis_start prefix rows, then the vision tokens listed in layer_ids[y][b][0 .. layer_cnt[y][b])
+ *       (original ids, strictly ascending), then n_tail further rows (text);
+ *   layer_ids int32 [n_layers, B, ids_max], layer_cnt int32 [n_layers, B];
+ *   s_few int32 [B, cap] original ids, ascending (the last layer's orig_out), s_few_cnt int32 [B];
+ *   k_out, v_out bf16 [n_layers, B, H, vis_start + cap + n_tail, D]: prefix rows, the rows of the
+ *       tokens of S_few in order, the tail rows directly behind them; later rows are untouched.
+ * A token of S_few that a layer does not hold is skipped and recorded as
+ * MUSTDROP_ERR_BAD_KEY_INDEX in the status word of `workspace` (>= 256 zeroed bytes, may be NULL).
+ * (k_cache, k_out) or (v_cache, v_out) may be NULL together.  vis_start + ids_max + n_tail <= rows_in,
+ * cap <= ids_max, head_dim == 128.
+ */
+typedef struct {
+  int32_t n_layers, batch, n_heads, head_dim;
+  int32_t rows_in, vis_start, n_tail, ids_max, cap;
+} mustdrop_cache_config_t;
+
+mustdrop_status_t mustdrop_cache_compact(const mustdrop_cache_config_t *config /* (host) */, const void *k_cache,
+                                         const void *v_cache, const int32_t *layer_ids,
+                                         const int32_t *layer_cnt, const int32_t *s_few,
+                                         const int32_t *s_few_cnt, void *k_out, void *v_out,
+                                         void *workspace, void *cuda_stream);
+
 /* Kernel launches one mustdrop_filter call enqueues for this plan (-1: invalid plan). */
 int32_t mustdrop_plan_filter_launches(const mustdrop_plan_t *plan);
 

@@ -34,7 +34,7 @@ EXPORTS = (
     "mustdrop_compact", "mustdrop_device_status", "mustdrop_status_string",
     "mustdrop_last_cuda_error", "mustdrop_plan_score_variant", "mustdrop_score_static",
     "mustdrop_score_static_max_rows", "mustdrop_filter", "mustdrop_plan_filter_launches",
-    "mustdrop_filter_layer",
+    "mustdrop_filter_layer", "mustdrop_cache_compact",
 )
 
 
@@ -59,6 +59,11 @@ class mustdrop_layer_io_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in (
         "q_text", "k", "v", "hidden", "key_idx", "key_cnt", "vis_cnt", "orig_idx", "g_out", "i_out", "s_out",
         "kept_idx", "kept_cnt", "orig_out", "key_idx_out", "key_cnt_out", "hidden_out", "k_out", "v_out")]
+
+
+class mustdrop_cache_config_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "n_layers", "batch", "n_heads", "head_dim", "rows_in", "vis_start", "n_tail", "ids_max", "cap")]
 
 
 class MustDropError(RuntimeError):
@@ -94,6 +99,8 @@ def lib() -> ctypes.CDLL:
         L.mustdrop_compact.argtypes = [vp] * 11
         L.mustdrop_filter.argtypes = [vp] * 17
         L.mustdrop_filter_layer.argtypes = [vp, ctypes.POINTER(mustdrop_layer_io_t), vp, vp]
+        L.mustdrop_cache_compact.argtypes = [ctypes.POINTER(mustdrop_cache_config_t)] + [vp] * 10
+        L.mustdrop_cache_compact.restype = ctypes.c_int
         L.mustdrop_plan_filter_launches.argtypes = [vp]
         L.mustdrop_plan_filter_launches.restype = ctypes.c_int32
         L.mustdrop_device_status.argtypes = [vp, vp, vp, i32p, i32p]
@@ -229,6 +236,18 @@ def mustdrop_filter_layer(plan, workspace, stream=None, **tensors) -> int:
             raise TypeError("mustdrop_layer_io_t has no field %r" % n)
         setattr(io, n, _ptr(t))
     return lib().mustdrop_filter_layer(plan, ctypes.byref(io), _ptr(workspace), _stream(stream))
+
+
+def mustdrop_cache_compact(k_cache, v_cache, layer_ids, layer_cnt, s_few, s_few_cnt, k_out, v_out, workspace=None,
+                           stream=None, **sizes) -> int:
+    """sizes: the fields of mustdrop_cache_config_t (head_dim defaults to 128)."""
+    c = mustdrop_cache_config_t()
+    c.head_dim = 128
+    for n, val in sizes.items():
+        setattr(c, n, int(val))
+    return lib().mustdrop_cache_compact(ctypes.byref(c), _ptr(k_cache), _ptr(v_cache), _ptr(layer_ids),
+                                        _ptr(layer_cnt), _ptr(s_few), _ptr(s_few_cnt), _ptr(k_out), _ptr(v_out),
+                                        _ptr(workspace), _stream(stream))
 
 
 def mustdrop_plan_filter_launches(plan) -> int:

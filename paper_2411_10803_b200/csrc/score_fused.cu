@@ -322,6 +322,25 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     Lb = txt_start + p.N;
   }
 
+  // End of the score part, executed by every thread: tensor memory freed, and no CTA goes on
+  // while a peer may still write into its shared memory.  The cluster barrier also orders every
+  // CTA's g_out / i_out stores before what the filter tail loads.  (In the filter kernel each
+  // warp role calls this from its own branch and continues there with its part of the tail, so
+  // every role keeps the register count setmaxnreg gave it; no second setmaxnreg is needed.)
+  __shared__ int32_t kept_total_s;
+  auto common_exit = [&]() {
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag != 0) record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
+    if (warp == kMmaWarp) {
+      tc_fence_after();
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+    cluster_sync_all();
+    MD_PIPE(p.workspace, 0, true, false);
+  };
+  int32_t* const kept_list = reinterpret_cast<int32_t*>(stage_ptr);   // filter tail: the request's kept indices
+
   if (warp >= kTmaWarp) {
     if (kRealloc) asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
     if (warp == kTmaWarp && lane == 0) {
@@ -385,6 +404,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         tc_commit(smem_u32(&bars.empty[s]));
         tc_commit(smem_u32(&bars.tfull[buf]));
       }
+    }
+    if constexpr (FILTER) {
+      // filter tail, TMA / MMA warps: nothing to do but to meet the others
+      __syncwarp();
+      common_exit();
+      if (*abort_flag == 0) __syncthreads();   // (the flag no longer changes: same decision in every thread)
+      return;
     }
   } else if (warp < kExpWarps) {
     // ---------------- exp warps ----------------
@@ -476,6 +502,27 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars.eready[last_buf]));
+    }
+    if constexpr (FILTER) {
+      // filter tail, exp warps: selection of this request.  Dynamic shared memory is free by now:
+      // all copies have landed, all MMAs have read them and every statistics pair sent to this CTA
+      // has been consumed.  Each CTA of the cluster runs the same selection on its own (identical
+      // inputs, fixed order: identical lists); rank 0 stores the list.
+      __shared__ SelectShared sel_sh;
+      common_exit();
+      pdl_wait();   // the outputs written below may still be read by an earlier kernel in the stream
+      if (*abort_flag != 0) return;
+      const int tid = threadIdx.x;
+      select_clear(sel_sh, tid);
+      const bool writer = rank == 0;
+      const int own = (ft.sel.M + kSelThreads - 1) / kSelThreads;
+      if (own <= 1) select_request<1, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      else if (own <= 2) select_request<2, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      else if (own <= 4) select_request<4, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      else if (own <= 8) select_request<8, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      else select_request<16, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      __syncthreads();   // the list is complete: the copy thread may start
+      return;
     }
   } else {
     // ---------------- add warps ----------------
@@ -578,128 +625,93 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         p.i_out[static_cast<size_t>(b) * p.M + j] = present ? mx * p.inv_heads : 0.0f;
       }
     }
-  }
-
-  // ---------------- common exit ----------------
-  if (kRealloc && FILTER) {
-    // The tail below runs on every warp: give them all the exp warps' 112 registers.  The add
-    // warps release theirs when they get here; the TMA / MMA warps wait for that inside inc.
-    // (16 x 112 warps' worth is less than the kernel held so far, so inc can always be served.)
-    __syncwarp();
-    if (warp >= kTmaWarp) asm volatile("setmaxnreg.inc.sync.aligned.u32 112;");
-    else if (warp >= kExpWarps) asm volatile("setmaxnreg.dec.sync.aligned.u32 112;");
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (threadIdx.x == 0 && *abort_flag != 0) record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
-  if (warp == kMmaWarp) {
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-  }
-  cluster_sync_all();   // no CTA leaves while a peer may still write into its shared memory
-  MD_PIPE(p.workspace, 0, true, false);
-
-  if constexpr (FILTER) {
-    // ---------------- selection and gather of this request ----------------
-    // The cluster barrier above also ordered every CTA's g_out / i_out stores before the loads
-    // below.  Dynamic shared memory is free: all copies have landed, all MMAs have read them and
-    // every statistics pair sent to this CTA has been consumed.  Each CTA of the cluster runs the
-    // same selection on its own (identical inputs, fixed order: identical lists); rank 0 stores
-    // the list.  Row r of the compacted outputs is then copied by CTA r mod cluster.
-    __shared__ SelectShared sel_sh;
-    __shared__ int32_t kept_total_s;
-    int32_t* kept_list = reinterpret_cast<int32_t*>(stage_ptr);
-    pdl_wait();   // the outputs written below may still be read by an earlier kernel in the stream
-    if (*abort_flag != 0) return;
-    if (warp < kSelWarps) {
-      const int tid = threadIdx.x;
-      select_clear(sel_sh, tid);
-      const bool writer = rank == 0;
-      const int own = (ft.sel.M + kSelThreads - 1) / kSelThreads;
-      if (own <= 1) select_request<1, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-      else if (own <= 2) select_request<2, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-      else if (own <= 4) select_request<4, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-      else if (own <= 8) select_request<8, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-      else select_request<16, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-    }
-    __syncthreads();
-    if (warp == kExpWarps && lane == 0) {
-      // One thread drives the copies: rows are loaded into a ring of shared-memory slots by bulk
-      // copies that count on the slot's mbarrier, and stored from there by bulk copies tracked in
-      // bulk groups.  Loads run n_slot - 2 rows ahead of the stores.
-      fence_proxy_async();   // earlier generic-proxy accesses to the slots precede the async-proxy writes
-      const int total = kept_total_s < ft.sel.cap ? kept_total_s : ft.sel.cap;
-      const int C = p.cluster;
-      // items: the kept vision rows, then (rebuild) the prefix rows and the request's text rows
-      const int n_items = total + (ft.rebuild ? ft.vis_start + ft.N : 0);
-      const int n_mine = n_items > static_cast<int>(rank) ? (n_items - static_cast<int>(rank) + C - 1) / C : 0;
-      const int S = ft.n_slot, ahead = S - 2;
-      const uint32_t ring = stage_base + kKeptListBytes;
-      const uint32_t payload = static_cast<uint32_t>(ft.hidden_bytes) + static_cast<uint32_t>(ft.has_k + ft.has_v) * ft.kv_bytes;
-      const uint64_t once = l2_evict_first_policy();
-      // item -> (source row, destination row)
-      auto src_row = [&](int it) {
-        if (it < total) return ft.vis_start + kept_list[it];
-        const int x = it - total;
-        return x < ft.vis_start ? x : ft.vis_start + Mb + (x - ft.vis_start);
-      };
-      auto dst_row = [&](int it) {
-        if (!ft.rebuild) return it;
-        if (it < total) return ft.vis_start + it;
-        const int x = it - total;
-        return x < ft.vis_start ? x : ft.vis_start + total + (x - ft.vis_start);
-      };
-      bool ok = true;
-      int loaded = 0;
-      for (int i = 0; i < n_mine + ahead && ok; ++i) {
-        if (i < n_mine) {
-          const int slot = i % S;
-          if (i >= S) bulk_wait_read_1();   // the stores of item i - S have finished reading the slot
-          const int row = src_row(static_cast<int>(rank) + i * C);
-          const uint32_t bar = smem_u32(&bars.gfull[slot]);
-          uint32_t dst = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
-          mbar_expect_tx(bar, payload);
-          if (ft.hidden_bytes > 0) {
-            bulk_load_1d(dst, ft.hidden + b * ft.hid_sb + row * ft.hid_sl, ft.hidden_bytes, bar, once);
-            dst += ft.hidden_pad;
+    if constexpr (FILTER) {
+      // filter tail, add warps: row r of the compacted outputs is copied by CTA r mod cluster
+      common_exit();
+      pdl_wait();
+      if (*abort_flag != 0) return;
+      __syncthreads();   // the exp warps have finished the selection
+      if (warp == kExpWarps && lane == 0) {
+        // One thread drives the copies: rows are loaded into a ring of shared-memory slots by bulk
+        // copies that count on the slot's mbarrier, and stored from there by bulk copies tracked in
+        // bulk groups.  Loads run n_slot - 2 rows ahead of the stores.
+        fence_proxy_async();   // earlier generic-proxy accesses to the slots precede the async-proxy writes
+        const int total = kept_total_s < ft.sel.cap ? kept_total_s : ft.sel.cap;
+        const int C = p.cluster;
+        // items: the kept vision rows, then (rebuild) the prefix rows and the request's text rows
+        const int n_items = total + (ft.rebuild ? ft.vis_start + ft.N : 0);
+        const int n_mine = n_items > static_cast<int>(rank) ? (n_items - static_cast<int>(rank) + C - 1) / C : 0;
+        const int S = ft.n_slot, ahead = S - 2;
+        const uint32_t ring = stage_base + kKeptListBytes;
+        const uint32_t payload = static_cast<uint32_t>(ft.hidden_bytes) + static_cast<uint32_t>(ft.has_k + ft.has_v) * ft.kv_bytes;
+        const uint64_t once = l2_evict_first_policy();
+        // item -> (source row, destination row)
+        auto src_row = [&](int it) {
+          if (it < total) return ft.vis_start + kept_list[it];
+          const int x = it - total;
+          return x < ft.vis_start ? x : ft.vis_start + Mb + (x - ft.vis_start);
+        };
+        auto dst_row = [&](int it) {
+          if (!ft.rebuild) return it;
+          if (it < total) return ft.vis_start + it;
+          const int x = it - total;
+          return x < ft.vis_start ? x : ft.vis_start + total + (x - ft.vis_start);
+        };
+        bool ok = true;
+        int loaded = 0;
+        for (int i = 0; i < n_mine + ahead && ok; ++i) {
+          if (i < n_mine) {
+            const int slot = i % S;
+            if (i >= S) bulk_wait_read_1();   // the stores of item i - S have finished reading the slot
+            const int row = src_row(static_cast<int>(rank) + i * C);
+            const uint32_t bar = smem_u32(&bars.gfull[slot]);
+            uint32_t dst = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
+            mbar_expect_tx(bar, payload);
+            if (ft.hidden_bytes > 0) {
+              bulk_load_1d(dst, ft.hidden + b * ft.hid_sb + row * ft.hid_sl, ft.hidden_bytes, bar, once);
+              dst += ft.hidden_pad;
+            }
+            if (ft.has_k) {
+              tma_load_4d_hint(dst, &gm.k_src, 0, row, 0, b, bar, once);
+              dst += ft.kv_bytes;
+            }
+            if (ft.has_v) tma_load_4d_hint(dst, &gm.v_src, 0, row, 0, b, bar, once);
+            loaded = i + 1;
           }
-          if (ft.has_k) {
-            tma_load_4d_hint(dst, &gm.k_src, 0, row, 0, b, bar, once);
-            dst += ft.kv_bytes;
+          const int c = i - ahead;
+          if (c >= 0) {
+            const int slot = c % S;
+            if (!mbar_wait(smem_u32(&bars.gfull[slot]), static_cast<uint32_t>(c / S) & 1u, abort_flag)) { ok = false; break; }
+            const int r = dst_row(static_cast<int>(rank) + c * C);
+            uint32_t src = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
+            if (ft.hidden_bytes > 0) {
+              bulk_store_1d(ft.hidden_out + (static_cast<int64_t>(b) * ft.out_rows + r) * ft.hidden_bytes, src, ft.hidden_bytes);
+              src += ft.hidden_pad;
+            }
+            if (ft.has_k) {
+              tma_store_4d(&gm.k_dst, 0, r, 0, b, src);
+              src += ft.kv_bytes;
+            }
+            if (ft.has_v) tma_store_4d(&gm.v_dst, 0, r, 0, b, src);
+            bulk_commit();
           }
-          if (ft.has_v) tma_load_4d_hint(dst, &gm.v_src, 0, row, 0, b, bar, once);
-          loaded = i + 1;
         }
-        const int c = i - ahead;
-        if (c >= 0) {
-          const int slot = c % S;
-          if (!mbar_wait(smem_u32(&bars.gfull[slot]), static_cast<uint32_t>(c / S) & 1u, abort_flag)) { ok = false; break; }
-          const int r = dst_row(static_cast<int>(rank) + c * C);
-          uint32_t src = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
-          if (ft.hidden_bytes > 0) {
-            bulk_store_1d(ft.hidden_out + (static_cast<int64_t>(b) * ft.out_rows + r) * ft.hidden_bytes, src, ft.hidden_bytes);
-            src += ft.hidden_pad;
+        if (!ok) {
+          // gave up: still leave only when every load this thread started has landed (bounded)
+          record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
+          for (int i = (loaded > S ? loaded - S : 0); i < loaded; ++i) {
+            const uint32_t bar = smem_u32(&bars.gfull[i % S]);
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar, static_cast<uint32_t>(i / S) & 1u) && clock64() - t0 < kWaitCycles) {}
           }
-          if (ft.has_k) {
-            tma_store_4d(&gm.k_dst, 0, r, 0, b, src);
-            src += ft.kv_bytes;
-          }
-          if (ft.has_v) tma_store_4d(&gm.v_dst, 0, r, 0, b, src);
-          bulk_commit();
         }
+        bulk_wait_all();   // the stores have been written before the CTA (and its shared memory) goes away
       }
-      if (!ok) {
-        // gave up: still leave only when every load this thread started has landed (bounded)
-        record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
-        for (int i = (loaded > S ? loaded - S : 0); i < loaded; ++i) {
-          const uint32_t bar = smem_u32(&bars.gfull[i % S]);
-          const long long t0 = clock64();
-          while (!mbar_try_wait(bar, static_cast<uint32_t>(i / S) & 1u) && clock64() - t0 < kWaitCycles) {}
-        }
-      }
-      bulk_wait_all();   // the stores have been written before the CTA (and its shared memory) goes away
+      return;
     }
   }
+
+  common_exit();   // (score-only kernel; the filter kernel's roles have left above)
 }
 
 // ---- host side ------------------------------------------------------------------------------------

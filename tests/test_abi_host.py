@@ -114,3 +114,20 @@ def test_shard_ranges_partition_the_batch():
             assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
             sizes = [hi - lo for lo, hi in spans]
             assert max(sizes) - min(sizes) <= 1
+
+
+def test_cache_compact_rejects_bad_sizes_without_a_gpu():
+    ok = dict(n_layers=2, batch=2, n_heads=2, rows_in=40, vis_start=1, n_tail=4, ids_max=20, cap=10)
+    for bad in (dict(n_layers=0), dict(cap=21), dict(rows_in=24), dict(n_tail=-1)):
+        kw = dict(ok)
+        kw.update(bad)
+        assert md.mustdrop_cache_compact(256, 256, 256, 256, 256, 256, 256, 256, None, stream=0, **kw) == \
+            md.MUSTDROP_ERR_INVALID_ARG
+    assert md.mustdrop_cache_compact(256, 256, 256, 256, 256, 256, 256, 256, None, stream=0, head_dim=64, **ok) == \
+        md.MUSTDROP_ERR_UNSUPPORTED
+    assert md.mustdrop_cache_compact(256, 256, None, 256, 256, 256, 256, 256, None, stream=0, **ok) == \
+        md.MUSTDROP_ERR_INVALID_ARG                                   # no layer_ids
+    assert md.mustdrop_cache_compact(256, None, 256, 256, 256, 256, 256, 256, None, stream=0, **ok) == \
+        md.MUSTDROP_ERR_INVALID_ARG                                   # v_out without v_cache
+    assert md.mustdrop_cache_compact(264, 256, 256, 256, 256, 256, 256, 256, None, stream=0, **ok) == \
+        md.MUSTDROP_ERR_INVALID_ARG                                   # misaligned

@@ -183,3 +183,73 @@ def test_chain_of_three_layers_matches_oracle(path):
             assert last <= set(f.orig_out.cpu().numpy()[b].tolist())
     for f in filters:
         f.close()
+
+
+# ---- decoding-stage cache compaction -----------------------------------------------------------
+
+def _cache_case(seed, Lyr, B, H, vs, tail, ids_max, cap, universe):
+    rng = np.random.default_rng(seed)
+    s_few = np.full((B, cap), -1, np.int32)
+    s_few_cnt = rng.integers(1, cap + 1, B).astype(np.int32)
+    layer_ids = np.full((Lyr, B, ids_max), -1, np.int32)
+    layer_cnt = np.zeros((Lyr, B), np.int32)
+    for b in range(B):
+        few = np.sort(rng.choice(universe, s_few_cnt[b], replace=False))
+        s_few[b, :s_few_cnt[b]] = few
+        rest = np.setdiff1d(np.arange(universe), few)
+        for y in range(Lyr):
+            n = int(rng.integers(s_few_cnt[b], ids_max + 1))
+            extra = rng.choice(rest, n - s_few_cnt[b], replace=False)
+            layer_ids[y, b, :n] = np.sort(np.concatenate([few, extra]))
+            layer_cnt[y, b] = n
+    R = vs + ids_max + tail
+    kc = rng.integers(0, 2 ** 16, (Lyr, B, H, R, 128)).astype(np.uint16)
+    vc = rng.integers(0, 2 ** 16, (Lyr, B, H, R, 128)).astype(np.uint16)
+    return kc, vc, layer_ids, layer_cnt, s_few, s_few_cnt, R
+
+
+@pytest.mark.parametrize("shape", [(3, 2, 2, 1, 4, 12, 6, 40), (5, 3, 8, 0, 7, 64, 45, 576), (2, 4, 3, 5, 0, 33, 33, 100)])
+def test_cache_compact_matches_oracle(shape):
+    Lyr, B, H, vs, tail, ids_max, cap, universe = shape
+    kc, vc, layer_ids, layer_cnt, s_few, s_few_cnt, R = _cache_case(11, *shape)
+    rk, rv = layers.cache_compact(kc, vc, layer_ids, layer_cnt, s_few, s_few_cnt, vs, tail)
+    rows_out = vs + cap + tail
+    ko = torch.zeros((Lyr, B, H, rows_out, 128), dtype=torch.bfloat16, device="cuda")
+    vo = torch.zeros_like(ko)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    st = md.mustdrop_cache_compact(to_dev_bf16(kc), to_dev_bf16(vc), to_dev(layer_ids), to_dev(layer_cnt), to_dev(s_few),
+                                   to_dev(s_few_cnt), ko, vo, ws, n_layers=Lyr, batch=B, n_heads=H, rows_in=R,
+                                   vis_start=vs, n_tail=tail, ids_max=ids_max, cap=cap)
+    assert st == md.MUSTDROP_OK
+    torch.cuda.synchronize()
+    assert ws[:8].cpu().numpy().view(np.int32).tolist() == [0, 0]
+    assert np.array_equal(bf16_bits(ko), rk) and np.array_equal(bf16_bits(vo), rv)
+
+
+def test_cache_compact_reports_a_token_the_layer_does_not_hold_and_takes_one_tensor():
+    shape = (2, 2, 2, 1, 3, 10, 5, 30)
+    Lyr, B, H, vs, tail, ids_max, cap, universe = shape
+    kc, vc, layer_ids, layer_cnt, s_few, s_few_cnt, R = _cache_case(3, *shape)
+    gone = s_few[1, 0]
+    pos = layer_ids[1, 1].tolist().index(gone)
+    layer_ids[1, 1, pos] = gone - 1 if pos == 0 or layer_ids[1, 1, pos - 1] < gone - 1 else gone   # keep ascending
+    missing = layer_ids[1, 1, pos] != gone
+    ko = torch.zeros((Lyr, B, H, vs + cap + tail, 128), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    st = md.mustdrop_cache_compact(to_dev_bf16(kc), None, to_dev(layer_ids), to_dev(layer_cnt), to_dev(s_few),
+                                   to_dev(s_few_cnt), ko, None, ws, n_layers=Lyr, batch=B, n_heads=H, rows_in=R,
+                                   vis_start=vs, n_tail=tail, ids_max=ids_max, cap=cap)
+    assert st == md.MUSTDROP_OK
+    torch.cuda.synchronize()
+    code, detail = ws[:8].cpu().numpy().view(np.int32).tolist()
+    if missing:
+        assert code == md.MUSTDROP_ERR_BAD_KEY_INDEX and detail == 1 * 65536 + 0
+        assert not bf16_bits(ko)[1, 1][:, vs + 0].any()                 # the row was skipped
+    # every other row is the brute-force gather
+    out = bf16_bits(ko)
+    for y in range(Lyr):
+        for b in range(B):
+            ids = layer_ids[y, b, :layer_cnt[y, b]].tolist()
+            for r, o in enumerate(s_few[b, :s_few_cnt[b]].tolist()):
+                if o in ids:
+                    assert np.array_equal(out[y, b][:, vs + r], kc[y, b][:, vs + ids.index(o)])
