@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # captures summarised under profiles/.  Keyed by (workload, budget, "filter" | "score", kernel
 # variant); anything else (or a kernel changed since its capture) reports null.
 NCU_TRAFFIC_BYTES = {
-    ("c2_llava7b_b64", 64, "filter", "fused_cluster_tcgen05"): 468321024 + 44385536,   # profiles/filter_kernel_c2_llava7b_b64.md
+    ("c2_llava7b_b64", 64, "filter", "fused_cluster_tcgen05"): 468304128 + 45627136,   # profiles/filter_kernel_c2_llava7b_b64.md
     ("c2_llava7b_b64", 64, "score", "fused_cluster_tcgen05"): 369161472 + 3128064,     # profiles/score_fused_kernel_c2_llava7b_b64.md
 }
 
