@@ -389,6 +389,130 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def _time_steps(torch, stream, fn, steps, warmup):
+    for _ in range(max(warmup, 3)):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def run_layers(args, w):
+    """Side measurement: a chain of pruning layers on a ragged batch (mustdrop_filter_layer),
+    every layer feeding the next on one stream.  Prints its own JSON line (single GPU)."""
+    import torch
+    from paper_2411_10803_b200 import binding as md
+    from paper_2411_10803_b200 import build as md_build
+    md_build.build()
+    torch.cuda.set_device(0)
+    budgets = [int(x) for x in args.layer_budgets.split(",")]
+    caps = [w.n_vis] + budgets[:-1]
+    cnt = synth.draw_vis_cnt(w)
+    cnts = [cnt]
+    for kp in budgets[:-1]:
+        cnts.append(np.minimum(cnts[-1], kp))
+    filters, dev, moved = [], [], 0
+    for l, (cap, kp) in enumerate(zip(caps, budgets)):
+        wl = w.with_(n_vis=cap, budget=kp, seed=w.seed + 100 * l, key_cnt=w.key_cnt if l == 0 else 0,
+                     n_salient=min(w.n_salient, cap))
+        p = synth.pack_ragged(synth.make_batch(wl), wl, cnts[l])
+        filters.append(md.Filter(md.config_for(wl, key_max=w.key_cnt, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE)))
+        dev.append([torch.from_numpy(p[n].view(np.int16)).cuda().view(torch.bfloat16)
+                    for n in ("q_text", "k", "v", "hidden")])
+        if l == 0:
+            ki0, kc0 = torch.from_numpy(p["key_idx"]).cuda(), torch.from_numpy(p["key_cnt"]).cuda()
+        row = (w.hidden + 2 * w.n_heads * w.head_dim) * 2
+        for b in range(w.batch):
+            lb = w.vis_start + int(cnts[l][b]) + w.n_txt
+            out_rows = w.vis_start + min(int(cnts[l][b]), kp) + w.n_txt
+            moved += w.n_heads * (lb + w.n_txt) * w.head_dim * 2 + 2 * out_rows * row   # K + Q read, rows read + written
+    vc0 = torch.from_numpy(cnt).cuda()
+    stream = torch.cuda.current_stream()
+
+    def step():
+        ki, kc, vc, orig = ki0, kc0, vc0, None
+        for l, f in enumerate(filters):
+            q, k, v, hid = dev[l]
+            f.filter_layer(q, k, v, hid, ki if w.key_cnt else None, kc if w.key_cnt else None, vis_cnt=vc,
+                           orig_idx=orig, stream=stream)
+            ki, kc, vc, orig = f.key_idx_out, f.key_cnt_out, f.kept_cnt, f.orig_out
+
+    ms = _time_steps(torch, stream, step, args.steps, args.warmup)
+    for f in filters:
+        code, detail = f.device_status()
+        if code != 0:
+            raise RuntimeError("device status %d (detail %d)" % (code, detail))
+    peak, peak_kind = measured_peak()
+    tokens = int(cnt.sum())
+    print(json.dumps({
+        "op": "layers", "metric": "vision tokens filtered/sec through %d pruning layers" % len(budgets),
+        "value": tokens / (ms / 1e3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "ms_per_step": ms,
+        "config": {"workload": w.name + " ragged", "batch": w.batch, "vis_cnt_mean": float(cnt.mean()),
+                   "capacities": caps, "budgets": budgets, "launches_per_step": sum(f.filter_launches for f in filters)},
+        "roofline": {"bound": "hbm", "achieved": moved / (ms / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": moved / (ms / 1e3) / 1e9 / peak, "peak_kind": peak_kind, "algorithmic_bytes": moved,
+                     "traffic": None},
+        "data": "synthetic"}), flush=True)
+    for f in filters:
+        f.close()
+
+
+def run_cache(args, w):
+    """Side measurement: decoding-stage cache compaction of all sparse layers in one launch."""
+    import torch
+    from paper_2411_10803_b200 import binding as md
+    from paper_2411_10803_b200 import build as md_build
+    md_build.build()
+    torch.cuda.set_device(0)
+    Lyr, B, H, D = args.cache_layers, w.batch, w.n_heads, w.head_dim
+    ids_max = cap = w.budget
+    n_tail, vs = w.n_txt, w.vis_start
+    rng = np.random.Generator(np.random.PCG64(w.seed + 5))
+    few_cnt = rng.integers(int(0.6 * cap), int(0.8 * cap) + 1, B).astype(np.int32)      # 64 -> about 45 (Table 3)
+    s_few = np.full((B, cap), -1, np.int32)
+    layer_ids = np.full((Lyr, B, ids_max), -1, np.int32)
+    layer_cnt = np.full((Lyr, B), ids_max, np.int32)
+    for b in range(B):
+        held = np.sort(rng.choice(w.n_vis, ids_max, replace=False))
+        layer_ids[:, b] = held
+        s_few[b, :few_cnt[b]] = np.sort(rng.choice(held, few_cnt[b], replace=False))
+    R = vs + ids_max + n_tail
+    kc = torch.randn((Lyr, B, H, R, D), device="cuda", dtype=torch.bfloat16)
+    vc = torch.randn((Lyr, B, H, R, D), device="cuda", dtype=torch.bfloat16)
+    ko = torch.zeros((Lyr, B, H, vs + cap + n_tail, D), device="cuda", dtype=torch.bfloat16)
+    vo = torch.zeros_like(ko)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    args_dev = [torch.from_numpy(a).cuda() for a in (layer_ids, layer_cnt, s_few, few_cnt)]
+    stream = torch.cuda.current_stream()
+
+    def step():
+        st = md.mustdrop_cache_compact(kc, vc, *args_dev, ko, vo, ws, stream, n_layers=Lyr, batch=B, n_heads=H,
+                                       rows_in=R, vis_start=vs, n_tail=n_tail, ids_max=ids_max, cap=cap)
+        if st != md.MUSTDROP_OK:
+            raise RuntimeError("mustdrop_cache_compact: %d" % st)
+
+    ms = _time_steps(torch, stream, step, args.steps, args.warmup)
+    if ws[:4].cpu().numpy().view(np.int32)[0] != 0:
+        raise RuntimeError("device status set")
+    rows = int((vs + few_cnt + n_tail).sum())
+    moved = 2 * 2 * Lyr * rows * H * D * 2     # K and V, read and written
+    peak, peak_kind = measured_peak()
+    print(json.dumps({
+        "op": "cache_compact", "metric": "cache rows compacted/sec (K and V, all sparse layers)",
+        "value": Lyr * rows / (ms / 1e3), "unit": "rows/s", "n_gpus": 1, "steps": args.steps, "ms_per_step": ms,
+        "config": {"layers": Lyr, "batch": B, "n_heads": H, "held_per_layer": ids_max, "s_few_mean": float(few_cnt.mean()),
+                   "tail_rows": n_tail},
+        "roofline": {"bound": "hbm", "achieved": moved / (ms / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": moved / (ms / 1e3) / 1e9 / peak, "peak_kind": peak_kind, "algorithmic_bytes": moved,
+                     "traffic": None},
+        "data": "synthetic"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -400,11 +524,19 @@ def main():
     ap.add_argument("--path", default="filter", choices=["filter", "staged"],
                     help="filter: the one-call entry point; staged: score, select and compact as three calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--op", default="filter", choices=["filter", "layers", "cache_compact"],
+                    help="filter: the benchmark proper; layers / cache_compact: side measurements (1 GPU)")
+    ap.add_argument("--layer-budgets", default="192,128,64", help="--op layers: keep budget of each pruning layer")
+    ap.add_argument("--cache-layers", type=int, default=30, help="--op cache_compact: layers that keep only S_few")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.budget:
         w = w.with_(budget=args.budget)
-    if args.impl == "reference":
+    if args.op == "layers":
+        run_layers(args, w)
+    elif args.op == "cache_compact":
+        run_cache(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)
