@@ -271,6 +271,39 @@ mustdrop_status_t mustdrop_cache_compact(const mustdrop_cache_config_t *config /
                                          const int32_t *s_few_cnt, void *k_out, void *v_out,
                                          void *workspace, void *cuda_stream);
 
+/*
+ * Local Spatial Merging of the vision encoder's tokens (Sec. 3.3, Eq. 5).  The grid x grid
+ * tokens of an image (raster order) are cut into non-overlapping window x window squares; a
+ * square whose mean cosine similarity over its unordered token pairs exceeds tau is replaced by
+ * the plain average of its tokens, placed at the square's first slot; the surviving tokens are
+ * packed in raster order.  (The paper states neither the similarity measure nor tau nor the
+ * weights: cosine, caller's tau, uniform weights are this library's reading.)
+ *   tokens bf16 [B, grid*grid, channels]; merged bf16 [B, grid*grid, channels] receives the
+ *   merged_cnt[b] surviving rows of image b (later rows untouched); slots int32 [B, grid*grid]
+ *   the slot each surviving row came from; merged_cnt int32 [B] (the vis_cnt of
+ *   mustdrop_filter_layer); window_sim fp32 [B, (grid/window)^2] or NULL receives the similarities.
+ * fp32 accumulation; an average is rounded once to bf16.  window must be 2, grid even,
+ * grid*grid <= 4096, channels a multiple of 8 (else MUSTDROP_ERR_UNSUPPORTED).
+ */
+mustdrop_status_t mustdrop_spatial_merge(int32_t batch, int32_t grid, int32_t window, int32_t channels,
+                                         float tau, const void *tokens, void *merged, int32_t *slots,
+                                         int32_t *merged_cnt, float *window_sim, void *cuda_stream);
+
+/*
+ * Key Retaining (Sec. 3.3, Eq. 6-7): a_cls = mean over heads of softmax(q_cls k^T / sqrt(head_dim))
+ * over the n_tokens patch tokens; O = { j : a_cls[j] > mu }.  The paper calls mu "adaptive" and
+ * gives no rule; here mu = Q3 + 1.5 (Q3 - Q1) of a_cls (Tukey's upper fence, linearly interpolated
+ * quartiles).
+ *   q_cls bf16 [B, H, head_dim]; k bf16 [B, H, n_tokens, head_dim] contiguous;
+ *   key_idx int32 [B, key_max] receives O ascending (if O has more than key_max members, the
+ *   key_max lowest indices), key_cnt int32 [B] the number stored - the key_idx / key_cnt of the
+ *   filter calls; a_cls fp32 [B, n_tokens] and mu_out fp32 [B] may be NULL.
+ * head_dim a multiple of 8 up to 256, n_tokens <= 4096.
+ */
+mustdrop_status_t mustdrop_key_set(int32_t batch, int32_t n_heads, int32_t head_dim, int32_t n_tokens,
+                                   int32_t key_max, const void *q_cls, const void *k, float *a_cls,
+                                   float *mu_out, int32_t *key_idx, int32_t *key_cnt, void *cuda_stream);
+
 /* Kernel launches one mustdrop_filter call enqueues for this plan (-1: invalid plan). */
 int32_t mustdrop_plan_filter_launches(const mustdrop_plan_t *plan);
 

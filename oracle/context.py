@@ -19,25 +19,28 @@ def kv_cache_mb(tokens: int, layers: int = 32, hidden: int = 4096, bytes_per_el:
     return tokens * 2 * layers * hidden * bytes_per_el / 1e6
 
 
-def local_spatial_merge(tokens: np.ndarray, grid: int, window: int = 2, tau: float = 0.8
-                        ) -> Tuple[np.ndarray, np.ndarray]:
+def local_spatial_merge(tokens: np.ndarray, grid: int, window: int = 2, tau: float = 0.8,
+                        return_sims: bool = False):
     """Local Spatial Merging (Sec. 3.3, Eq. 5).
 
     tokens [grid*grid, C] in raster order.  The grid is cut into non-overlapping
     window x window squares; for each square S_w = mean over unordered pairs of the cosine
     similarity of its tokens; if S_w > tau the square is replaced by the plain average of
     its tokens, placed at the square's first raster slot.  Returns (merged tokens
-    [M', C], source slot of each output token [M']).
+    [M', C], source slot of each output token [M']), with ``return_sims`` also S_w of every
+    window (raster order of windows).
     """
     x = np.asarray(tokens, np.float64)
     assert x.shape[0] == grid * grid and grid % window == 0
     keep_rows: List[np.ndarray] = []
     slots: List[int] = []
+    all_sims: List[float] = []
     unit = x / np.maximum(np.linalg.norm(x, axis=1, keepdims=True), 1e-300)
     for wy in range(0, grid, window):
         for wx in range(0, grid, window):
             ids = [(wy + dy) * grid + (wx + dx) for dy in range(window) for dx in range(window)]
             sims = [float(unit[a] @ unit[b]) for ai, a in enumerate(ids) for b in ids[ai + 1:]]
+            all_sims.append(float(np.mean(sims)))
             if np.mean(sims) > tau:
                 keep_rows.append(x[ids].mean(axis=0))
                 slots.append(ids[0])
@@ -46,7 +49,8 @@ def local_spatial_merge(tokens: np.ndarray, grid: int, window: int = 2, tau: flo
                     keep_rows.append(x[t])
                     slots.append(t)
     order = np.argsort(np.asarray(slots), kind="stable")
-    return np.stack(keep_rows)[order], np.asarray(slots, np.int64)[order]
+    out = (np.stack(keep_rows)[order], np.asarray(slots, np.int64)[order])
+    return out + (np.asarray(all_sims),) if return_sims else out
 
 
 def key_set(q_cls: np.ndarray, k: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:

@@ -34,7 +34,7 @@ EXPORTS = (
     "mustdrop_compact", "mustdrop_device_status", "mustdrop_status_string",
     "mustdrop_last_cuda_error", "mustdrop_plan_score_variant", "mustdrop_score_static",
     "mustdrop_score_static_max_rows", "mustdrop_filter", "mustdrop_plan_filter_launches",
-    "mustdrop_filter_layer", "mustdrop_cache_compact",
+    "mustdrop_filter_layer", "mustdrop_cache_compact", "mustdrop_spatial_merge", "mustdrop_key_set",
 )
 
 
@@ -101,6 +101,11 @@ def lib() -> ctypes.CDLL:
         L.mustdrop_filter_layer.argtypes = [vp, ctypes.POINTER(mustdrop_layer_io_t), vp, vp]
         L.mustdrop_cache_compact.argtypes = [ctypes.POINTER(mustdrop_cache_config_t)] + [vp] * 10
         L.mustdrop_cache_compact.restype = ctypes.c_int
+        i32, f32 = ctypes.c_int32, ctypes.c_float
+        L.mustdrop_spatial_merge.argtypes = [i32, i32, i32, i32, f32, vp, vp, vp, vp, vp, vp]
+        L.mustdrop_spatial_merge.restype = ctypes.c_int
+        L.mustdrop_key_set.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.mustdrop_key_set.restype = ctypes.c_int
         L.mustdrop_plan_filter_launches.argtypes = [vp]
         L.mustdrop_plan_filter_launches.restype = ctypes.c_int32
         L.mustdrop_device_status.argtypes = [vp, vp, vp, i32p, i32p]
@@ -248,6 +253,18 @@ def mustdrop_cache_compact(k_cache, v_cache, layer_ids, layer_cnt, s_few, s_few_
     return lib().mustdrop_cache_compact(ctypes.byref(c), _ptr(k_cache), _ptr(v_cache), _ptr(layer_ids),
                                         _ptr(layer_cnt), _ptr(s_few), _ptr(s_few_cnt), _ptr(k_out), _ptr(v_out),
                                         _ptr(workspace), _stream(stream))
+
+
+def mustdrop_spatial_merge(batch, grid, window, channels, tau, tokens, merged, slots, merged_cnt, window_sim=None,
+                           stream=None) -> int:
+    return lib().mustdrop_spatial_merge(batch, grid, window, channels, tau, _ptr(tokens), _ptr(merged), _ptr(slots),
+                                        _ptr(merged_cnt), _ptr(window_sim), _stream(stream))
+
+
+def mustdrop_key_set(batch, n_heads, head_dim, n_tokens, key_max, q_cls, k, a_cls, mu_out, key_idx, key_cnt,
+                     stream=None) -> int:
+    return lib().mustdrop_key_set(batch, n_heads, head_dim, n_tokens, key_max, _ptr(q_cls), _ptr(k), _ptr(a_cls),
+                                  _ptr(mu_out), _ptr(key_idx), _ptr(key_cnt), _stream(stream))
 
 
 def mustdrop_plan_filter_launches(plan) -> int:

@@ -218,3 +218,31 @@ def pack_ragged(d: Dict[str, np.ndarray], w: Workload, vis_cnt) -> Dict[str, np.
         out["key_cnt"][b] = len(keys)
     out["vis_cnt"] = np.asarray(vis_cnt, np.int32).copy()
     return out
+
+
+def make_vit_tokens(seed: int, batch: int, grid: int, channels: int, merge_frac: float = 0.3) -> np.ndarray:
+    """Vision-encoder tokens [B, grid*grid, C] as bf16 bits: i.i.d. N(0,1), except that in a
+    fraction of the 2x2 windows the four tokens are one common vector plus 5 % noise (flat image
+    regions, which the spatial merge is meant to collapse)."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, 11])))
+    x = rng.standard_normal((batch, grid, grid, channels)).astype(np.float32)
+    flat = rng.random((batch, grid // 2, grid // 2)) < merge_frac
+    for b, wy, wx in zip(*np.nonzero(flat)):
+        base = rng.standard_normal(channels).astype(np.float32)
+        x[b, 2 * wy:2 * wy + 2, 2 * wx:2 * wx + 2] = base + 0.05 * x[b, 2 * wy:2 * wy + 2, 2 * wx:2 * wx + 2]
+    return f32_to_bf16_bits(x.reshape(batch, grid * grid, channels))
+
+
+def make_cls_attention(seed: int, batch: int, n_heads: int, head_dim: int, n_tokens: int, n_outliers: int):
+    """[CLS] query [B,H,D] and patch keys [B,H,M,D] (bf16 bits): N(0,1), with n_outliers keys per
+    image pulled towards the query of every head (the tokens the key set should contain)."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, 13])))
+    q = rng.standard_normal((batch, n_heads, head_dim)).astype(np.float32)
+    k = rng.standard_normal((batch, n_heads, n_tokens, head_dim)).astype(np.float32)
+    planted = np.zeros((batch, n_outliers), np.int32)
+    for b in range(batch):
+        idx = np.sort(rng.choice(n_tokens, n_outliers, replace=False))
+        planted[b] = idx
+        unit = q[b] / np.linalg.norm(q[b], axis=1, keepdims=True)
+        k[b][:, idx] += 0.6 * np.sqrt(head_dim) * unit[:, None, :]
+    return f32_to_bf16_bits(q), f32_to_bf16_bits(k), planted

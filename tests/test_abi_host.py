@@ -131,3 +131,15 @@ def test_cache_compact_rejects_bad_sizes_without_a_gpu():
         md.MUSTDROP_ERR_INVALID_ARG                                   # v_out without v_cache
     assert md.mustdrop_cache_compact(264, 256, 256, 256, 256, 256, 256, 256, None, stream=0, **ok) == \
         md.MUSTDROP_ERR_INVALID_ARG                                   # misaligned
+
+
+def test_upstream_calls_reject_bad_sizes_without_a_gpu():
+    assert md.mustdrop_spatial_merge(1, 24, 3, 1024, 0.8, 256, 256, 256, 256, None, stream=0) == md.MUSTDROP_ERR_UNSUPPORTED
+    assert md.mustdrop_spatial_merge(1, 25, 2, 1024, 0.8, 256, 256, 256, 256, None, stream=0) == md.MUSTDROP_ERR_UNSUPPORTED
+    assert md.mustdrop_spatial_merge(1, 24, 2, 1020, 0.8, 256, 256, 256, 256, None, stream=0) == md.MUSTDROP_ERR_UNSUPPORTED
+    assert md.mustdrop_spatial_merge(0, 24, 2, 1024, 0.8, 256, 256, 256, 256, None, stream=0) == md.MUSTDROP_ERR_INVALID_ARG
+    assert md.mustdrop_spatial_merge(1, 24, 2, 1024, 0.8, None, 256, 256, 256, None, stream=0) == md.MUSTDROP_ERR_INVALID_ARG
+    assert md.mustdrop_key_set(1, 16, 60, 576, 64, 256, 256, None, None, 256, 256, stream=0) == md.MUSTDROP_ERR_UNSUPPORTED
+    assert md.mustdrop_key_set(1, 16, 64, 5000, 64, 256, 256, None, None, 256, 256, stream=0) == md.MUSTDROP_ERR_UNSUPPORTED
+    assert md.mustdrop_key_set(1, 16, 64, 576, 0, 256, 256, None, None, 256, 256, stream=0) == md.MUSTDROP_ERR_INVALID_ARG
+    assert md.mustdrop_key_set(1, 16, 64, 576, 64, 256, 264, None, None, 256, 256, stream=0) == md.MUSTDROP_ERR_INVALID_ARG
