@@ -513,6 +513,51 @@ def run_cache(args, w):
         "data": "synthetic"}), flush=True)
 
 
+def run_upstream(args, w):
+    """Side measurement: the vision-encoding stage kernels (spatial merge, [CLS] key set)."""
+    import torch
+    from paper_2411_10803_b200 import binding as md
+    from paper_2411_10803_b200 import build as md_build
+    md_build.build()
+    torch.cuda.set_device(0)
+    B, grid, C, H, D = w.batch, 24, 1024, 16, 64          # CLIP ViT-L/14 at 336 px: 24 x 24 patches, 1024 channels
+    M = grid * grid
+    tok = torch.from_numpy(synth.make_vit_tokens(w.seed, B, grid, C).view(np.int16)).cuda().view(torch.bfloat16)
+    qb, kb, _ = synth.make_cls_attention(w.seed, B, H, D, M, 29)
+    q = torch.from_numpy(qb.view(np.int16)).cuda().view(torch.bfloat16)
+    k = torch.from_numpy(kb.view(np.int16)).cuda().view(torch.bfloat16)
+    merged = torch.zeros((B, M, C), dtype=torch.bfloat16, device="cuda")
+    slots = torch.zeros((B, M), dtype=torch.int32, device="cuda")
+    cnt = torch.zeros((B,), dtype=torch.int32, device="cuda")
+    ki = torch.zeros((B, 64), dtype=torch.int32, device="cuda")
+    kc = torch.zeros((B,), dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+    peak, peak_kind = measured_peak()
+
+    def merge():
+        st = md.mustdrop_spatial_merge(B, grid, 2, C, 0.8, tok, merged, slots, cnt, None, stream)
+        assert st == md.MUSTDROP_OK
+
+    def keys():
+        st = md.mustdrop_key_set(B, H, D, M, 64, q, k, None, None, ki, kc, stream)
+        assert st == md.MUSTDROP_OK
+
+    ms_m = _time_steps(torch, stream, merge, args.steps, args.warmup)
+    ms_k = _time_steps(torch, stream, keys, args.steps, args.warmup)
+    kept = int(cnt.sum())
+    bytes_m = B * M * C * 2 + kept * C * 2
+    bytes_k = B * H * M * D * 2
+    print(json.dumps({
+        "op": "upstream", "unit": "images/s", "n_gpus": 1, "steps": args.steps,
+        "config": {"batch": B, "grid": grid, "channels": C, "vit_heads": H, "vit_head_dim": D,
+                   "tokens_after_merge_mean": kept / B, "key_set_mean": float(kc.float().mean())},
+        "spatial_merge": {"ms": ms_m, "images_per_s": B / (ms_m / 1e3), "algorithmic_bytes": bytes_m,
+                          "achieved_gbs": bytes_m / (ms_m / 1e3) / 1e9, "frac": bytes_m / (ms_m / 1e3) / 1e9 / peak},
+        "key_set": {"ms": ms_k, "images_per_s": B / (ms_k / 1e3), "algorithmic_bytes": bytes_k,
+                    "achieved_gbs": bytes_k / (ms_k / 1e3) / 1e9, "frac": bytes_k / (ms_k / 1e3) / 1e9 / peak},
+        "peak": peak, "peak_kind": peak_kind, "data": "synthetic"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -524,7 +569,7 @@ def main():
     ap.add_argument("--path", default="filter", choices=["filter", "staged"],
                     help="filter: the one-call entry point; staged: score, select and compact as three calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--op", default="filter", choices=["filter", "layers", "cache_compact"],
+    ap.add_argument("--op", default="filter", choices=["filter", "layers", "cache_compact", "upstream"],
                     help="filter: the benchmark proper; layers / cache_compact: side measurements (1 GPU)")
     ap.add_argument("--layer-budgets", default="192,128,64", help="--op layers: keep budget of each pruning layer")
     ap.add_argument("--cache-layers", type=int, default=30, help="--op cache_compact: layers that keep only S_few")
@@ -536,6 +581,8 @@ def main():
         run_layers(args, w)
     elif args.op == "cache_compact":
         run_cache(args, w)
+    elif args.op == "upstream":
+        run_upstream(args, w)
     elif args.impl == "reference":
         run_reference(args, w)
     else:

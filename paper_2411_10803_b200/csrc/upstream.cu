@@ -5,8 +5,10 @@
 //   Key Retaining (Eq. 6-7): head-averaged [CLS] attention over the patch tokens, and the tokens
 //     above an adaptive threshold form the key set O.  The paper names no threshold rule; here it
 //     is Tukey's upper fence Q3 + 1.5 (Q3 - Q1) with linearly interpolated quartiles.
-// Both are one CTA of 256 threads per image; both are bound by reading their input once
-// (1.2 MB per image at 576 tokens x 1024 channels).
+// A thread-block cluster of up to eight CTAs of 256 threads works on one image (windows, rows and
+// heads are dealt out over the cluster's CTAs; flags and partial attention sums cross through
+// distributed shared memory, in a fixed order); both kernels are bound by reading their input
+// once (1.2 MB per image at 576 tokens x 1024 channels).
 #include <cuda_bf16.h>
 
 #include "mustdrop_internal.h"
@@ -26,6 +28,28 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
   return v;
+}
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_size() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of a shared-memory object of this CTA, as seen in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t peer_addr(const void* local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+               : "=r"(r)
+               : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(local))), "r"(rank));
+  return r;
 }
 
 // Exclusive prefix sum of one int per thread over the CTA (fixed order); returns the total too.
@@ -65,14 +89,16 @@ struct MergeParams {
 __global__ void __launch_bounds__(kThreads) spatial_merge_kernel(MergeParams p) {
   __shared__ unsigned char merged_flag[kMaxSlots / 4];
   __shared__ int warp_sums[kWarps];
-  const int b = blockIdx.x, g = p.grid, gw = g / 2, n_win = gw * gw, n_slot = g * g;
+  const int C = static_cast<int>(cluster_size()), rank = static_cast<int>(cluster_rank());
+  const int b = blockIdx.x / C, g = p.grid, gw = g / 2, n_win = gw * gw, n_slot = g * g;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   pdl_launch_dependents();
   pdl_wait();
   const uint4* in = p.tokens + static_cast<size_t>(b) * n_slot * p.vecs;
 
-  // 1. per window: the four norms and six dot products, fp32 accumulation
-  for (int w = warp; w < n_win; w += kWarps) {
+  // 1. per window: the four norms and six dot products, fp32 accumulation.  The cluster's warps
+  //    share the windows; a window's flag is stored into every CTA's copy of the flag array.
+  for (int w = rank * kWarps + warp; w < n_win; w += C * kWarps) {
     const int wy = w / gw, wx = w % gw;
     const int s0 = (2 * wy) * g + 2 * wx;
     const uint4* r0 = in + static_cast<size_t>(s0) * p.vecs;
@@ -107,14 +133,16 @@ __global__ void __launch_bounds__(kThreads) spatial_merge_kernel(MergeParams p) 
                   l3 = fmaxf(sqrtf(n3), tiny);
       const float sim = (d01 / (l0 * l1) + d02 / (l0 * l2) + d03 / (l0 * l3) + d12 / (l1 * l2) + d13 / (l1 * l3) +
                          d23 / (l2 * l3)) * (1.0f / 6.0f);
-      merged_flag[w] = sim > p.tau ? 1 : 0;
+      const uint32_t flag = sim > p.tau ? 1u : 0u;
+      for (int c = 0; c < C; ++c)
+        asm volatile("st.shared::cluster.u8 [%0], %1;" ::"r"(peer_addr(&merged_flag[w], c)), "r"(flag) : "memory");
       if (p.window_sim != nullptr) p.window_sim[static_cast<size_t>(b) * n_win + w] = sim;
     }
   }
-  __syncthreads();
+  cluster_barrier();   // every flag has arrived in every CTA; no remote store after this point
 
-  // 2. which slots emit a token (all slots of an unmerged window, the first slot of a merged one)
-  //    and where: exclusive scan in raster order
+  // 2. which slots emit a token (all slots of an unmerged window, the first slot of a merged
+  //    one) and where: exclusive scan in raster order, by every CTA for itself; CTA 0 stores it
   const int j0 = threadIdx.x * kOwn;
   uint32_t emit = 0;
 #pragma unroll
@@ -135,19 +163,19 @@ __global__ void __launch_bounds__(kThreads) spatial_merge_kernel(MergeParams p) 
     if (s < n_slot) {
       if ((emit >> e) & 1u) {
         out_pos[s] = static_cast<int16_t>(pos);
-        p.slots[static_cast<size_t>(b) * n_slot + pos] = s;
+        if (rank == 0) p.slots[static_cast<size_t>(b) * n_slot + pos] = s;
         ++pos;
       } else {
         out_pos[s] = -1;
       }
     }
   }
-  if (threadIdx.x == 0) p.merged_cnt[b] = total;
+  if (threadIdx.x == 0 && rank == 0) p.merged_cnt[b] = total;
   __syncthreads();
 
   // 3. write the surviving rows: a copy, or the plain average of the window in fp32, rounded once
   uint4* out = p.merged + static_cast<size_t>(b) * n_slot * p.vecs;
-  for (int s = warp; s < n_slot; s += kWarps) {
+  for (int s = rank * kWarps + warp; s < n_slot; s += C * kWarps) {
     const int o = out_pos[s];
     if (o < 0) continue;
     const int y = s / g, x = s % g;
@@ -197,14 +225,16 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
   __shared__ float red[kWarps];
   __shared__ float order[4];          // the four order statistics the quartiles interpolate
   __shared__ int warp_sums[kWarps];
-  const int b = blockIdx.x, M = p.M, dv = p.D / 8;
+  extern __shared__ float slab[];     // CTA 0: [cluster size][M] partial sums of the cluster's CTAs
+  const int C = static_cast<int>(cluster_size()), rank = static_cast<int>(cluster_rank());
+  const int b = blockIdx.x / C, M = p.M, dv = p.D / 8;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   pdl_launch_dependents();
   pdl_wait();
   for (int j = threadIdx.x; j < M; j += kThreads) a[j] = 0.0f;
   const float inv_h = 1.0f / static_cast<float>(p.H);
 
-  for (int h = 0; h < p.H; ++h) {
+  for (int h = rank; h < p.H; h += C) {   // the cluster's CTAs share the heads
     __syncthreads();   // q_s, z and red are free again
     for (int d = threadIdx.x; d < p.D; d += kThreads)
       q_s[d] = __bfloat162float(p.q_cls[(static_cast<size_t>(b) * p.H + h) * p.D + d]);
@@ -248,6 +278,17 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
     for (int w = 0; w < kWarps; ++w) sum += red[w];   // fixed order
     const float f = inv_h / sum;
     for (int j = threadIdx.x; j < M; j += kThreads) a[j] = fmaf(z[j], f, a[j]);
+  }
+  // every CTA hands its partial sums to CTA 0, which adds them in rank order
+  for (int j = threadIdx.x; j < M; j += kThreads)
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr(&slab[static_cast<size_t>(rank) * M + j], 0)), "f"(a[j])
+                 : "memory");
+  cluster_barrier();
+  if (rank != 0) return;
+  for (int j = threadIdx.x; j < M; j += kThreads) {
+    float sum = 0.0f;
+    for (int c = 0; c < C; ++c) sum += slab[static_cast<size_t>(c) * M + j];
+    a[j] = sum;
   }
   __syncthreads();
 
@@ -298,6 +339,25 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
 
 inline bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
 
+template <typename Kernel, typename Params>
+cudaError_t launch_cluster(Kernel kernel, int batch, int cluster, size_t smem, cudaStream_t stream, const Params& p) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(batch * cluster));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
 inline mustdrop_status_t finish(cudaError_t e) {
   if (e == cudaSuccess) return MUSTDROP_OK;
   set_last_cuda_error(e);
@@ -324,8 +384,10 @@ extern "C" mustdrop_status_t mustdrop_spatial_merge(int32_t batch, int32_t grid,
   p.merged = static_cast<uint4*>(merged);
   p.slots = slots; p.merged_cnt = merged_cnt; p.window_sim = window_sim;
   p.grid = grid; p.vecs = channels / 8; p.tau = tau;
-  return finish(launch_pdl(spatial_merge_kernel, dim3(static_cast<unsigned>(batch)), dim3(kThreads), 0,
-                           static_cast<cudaStream_t>(cuda_stream), p));
+  const int n_win = (grid / 2) * (grid / 2);
+  int cluster = 8;                                   // no more CTAs than there are rounds of windows for them
+  while (cluster > 1 && (cluster - 1) * kWarps >= n_win) cluster >>= 1;
+  return finish(launch_cluster(spatial_merge_kernel, batch, cluster, 0, static_cast<cudaStream_t>(cuda_stream), p));
 }
 
 extern "C" mustdrop_status_t mustdrop_key_set(int32_t batch, int32_t n_heads, int32_t head_dim, int32_t n_tokens,
@@ -345,6 +407,11 @@ extern "C" mustdrop_status_t mustdrop_key_set(int32_t batch, int32_t n_heads, in
   p.a_cls = a_cls; p.mu_out = mu_out; p.key_idx = key_idx; p.key_cnt = key_cnt;
   p.H = n_heads; p.D = head_dim; p.M = n_tokens; p.key_max = key_max;
   p.scale_log2e = 1.4426950408889634f / sqrtf(static_cast<float>(head_dim));
-  return finish(launch_pdl(key_set_kernel, dim3(static_cast<unsigned>(batch)), dim3(kThreads), 0,
-                           static_cast<cudaStream_t>(cuda_stream), p));
+  int cluster = 8;
+  while (cluster > n_heads) cluster >>= 1;           // 1, 2, 4 or 8 CTAs, at most one per head
+  const size_t smem = static_cast<size_t>(cluster) * n_tokens * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(key_set_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(8 * kMaxSlots * sizeof(float)));
+  if (e != cudaSuccess) return finish(e);
+  return finish(launch_cluster(key_set_kernel, batch, cluster, smem, static_cast<cudaStream_t>(cuda_stream), p));
 }
