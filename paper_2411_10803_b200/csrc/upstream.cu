@@ -219,13 +219,13 @@ struct KeySetParams {
 };
 
 __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
-  __shared__ float a[kMaxSlots];      // head-mean attention
+  __shared__ __align__(16) float a[kMaxSlots];      // head-mean attention
   __shared__ float z[kMaxSlots];      // one head's logits (log2 units)
-  __shared__ float q_s[256];
+  __shared__ __align__(16) float q_s[256];
   __shared__ float red[kWarps];
   __shared__ float order[4];          // the four order statistics the quartiles interpolate
   __shared__ int warp_sums[kWarps];
-  extern __shared__ float slab[];     // CTA 0: [cluster size][M] partial sums of the cluster's CTAs
+  extern __shared__ float slab[];     // [cluster size][M] partial sums of the cluster's CTAs
   const int C = static_cast<int>(cluster_size()), rank = static_cast<int>(cluster_rank());
   const int b = blockIdx.x / C, M = p.M, dv = p.D / 8;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -243,13 +243,22 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
     float mx = -INFINITY;
     for (int j = threadIdx.x; j < M; j += kThreads) {   // one token per thread: its row is D contiguous bf16
       float dot = 0.0f;
-      for (int v = 0; v < dv; ++v) {
-        const uint4 kv = kh[static_cast<size_t>(j) * dv + v];
-        const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
+      const uint4* krow = kh + static_cast<size_t>(j) * dv;
+      for (int v0 = 0; v0 < dv; v0 += 4) {                 // four 16-byte loads in flight per thread
+        uint4 kv[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          dot = fmaf(bf16_lo(w[q]), q_s[v * 8 + 2 * q], dot);
-          dot = fmaf(bf16_hi(w[q]), q_s[v * 8 + 2 * q + 1], dot);
+        for (int u = 0; u < 4; ++u)
+          if (v0 + u < dv) kv[u] = krow[v0 + u];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (v0 + u < dv) {
+            const float4 qa = *reinterpret_cast<const float4*>(&q_s[(v0 + u) * 8]);
+            const float4 qb = *reinterpret_cast<const float4*>(&q_s[(v0 + u) * 8 + 4]);
+            dot = fmaf(bf16_lo(kv[u].x), qa.x, dot); dot = fmaf(bf16_hi(kv[u].x), qa.y, dot);
+            dot = fmaf(bf16_lo(kv[u].y), qa.z, dot); dot = fmaf(bf16_hi(kv[u].y), qa.w, dot);
+            dot = fmaf(bf16_lo(kv[u].z), qb.x, dot); dot = fmaf(bf16_hi(kv[u].z), qb.y, dot);
+            dot = fmaf(bf16_lo(kv[u].w), qb.z, dot); dot = fmaf(bf16_hi(kv[u].w), qb.w, dot);
+          }
         }
       }
       const float zz = dot * p.scale_log2e;
@@ -279,36 +288,43 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
     const float f = inv_h / sum;
     for (int j = threadIdx.x; j < M; j += kThreads) a[j] = fmaf(z[j], f, a[j]);
   }
-  // every CTA hands its partial sums to CTA 0, which adds them in rank order
-  for (int j = threadIdx.x; j < M; j += kThreads)
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr(&slab[static_cast<size_t>(rank) * M + j], 0)), "f"(a[j])
-                 : "memory");
+  // every CTA hands its partial sums to every CTA; each adds them in rank order (same result everywhere)
+  for (int c = 0; c < C; ++c)
+    for (int j = threadIdx.x; j < M; j += kThreads)
+      asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr(&slab[static_cast<size_t>(rank) * M + j], c)), "f"(a[j])
+                   : "memory");
   cluster_barrier();
-  if (rank != 0) return;
   for (int j = threadIdx.x; j < M; j += kThreads) {
     float sum = 0.0f;
     for (int c = 0; c < C; ++c) sum += slab[static_cast<size_t>(c) * M + j];
     a[j] = sum;
   }
+  const int M4 = (M + 3) & ~3;
+  if (threadIdx.x < M4 - M) a[M + threadIdx.x] = INFINITY;   // padding that is never counted
   __syncthreads();
 
-  // quartiles by rank counting: the element with r smaller ones (ties by index) is order statistic r
+  // quartiles by rank counting: the element with r smaller ones (ties by index) is order statistic r.
+  // The cluster's CTAs share the tokens; whoever finds one of the four needed statistics stores it in CTA 0.
   const float p1 = 0.25f * static_cast<float>(M - 1), p3 = 0.75f * static_cast<float>(M - 1);
   const int r1 = static_cast<int>(floorf(p1)), r3 = static_cast<int>(floorf(p3));
   const int r1h = min(r1 + 1, M - 1), r3h = min(r3 + 1, M - 1);
-  for (int j = threadIdx.x; j < M; j += kThreads) {
+  for (int j = threadIdx.x * C + rank; j < M; j += kThreads * C) {
     const float aj = a[j];
-    int rank = 0;
-    for (int i = 0; i < M; ++i) {
-      const float ai = a[i];
-      rank += (ai < aj || (ai == aj && i < j)) ? 1 : 0;
+    int rk = 0;
+    for (int i = 0; i < M4; i += 4) {                          // four candidates per shared load
+      const float4 v = *reinterpret_cast<const float4*>(&a[i]);
+      rk += (v.x < aj || (v.x == aj && i < j)) ? 1 : 0;
+      rk += (v.y < aj || (v.y == aj && i + 1 < j)) ? 1 : 0;
+      rk += (v.z < aj || (v.z == aj && i + 2 < j)) ? 1 : 0;
+      rk += (v.w < aj || (v.w == aj && i + 3 < j)) ? 1 : 0;
     }
-    if (rank == r1) order[0] = aj;
-    if (rank == r1h) order[1] = aj;
-    if (rank == r3) order[2] = aj;
-    if (rank == r3h) order[3] = aj;
+    if (rk == r1) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr(&order[0], 0)), "f"(aj) : "memory");
+    if (rk == r1h) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr(&order[1], 0)), "f"(aj) : "memory");
+    if (rk == r3) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr(&order[2], 0)), "f"(aj) : "memory");
+    if (rk == r3h) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr(&order[3], 0)), "f"(aj) : "memory");
   }
-  __syncthreads();
+  cluster_barrier();
+  if (rank != 0) return;   // CTA 0 finishes alone; no store into another CTA's memory after this point
   const float q1 = order[0] + (order[1] - order[0]) * (p1 - static_cast<float>(r1));
   const float q3 = order[2] + (order[3] - order[2]) * (p3 - static_cast<float>(r3));
   const float mu = q3 + 1.5f * (q3 - q1);
