@@ -112,7 +112,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   (void)cudaGetLastError();
 
   // Score kernel: the fused single-pass kernel where its geometry covers the shape, else the
-  // two-pass kernel.  MUSTDROP_SCORE_VARIANT (two_pass | fused) and MUSTDROP_CLUSTER (1..8) are
+  // two-pass kernel.  MUSTDROP_SCORE_VARIANT (two_pass | fused) and MUSTDROP_CLUSTER (1..16) are
   // debugging overrides read here, once per plan.
   p->score_variant = kScoreTwoPassMma;
   {

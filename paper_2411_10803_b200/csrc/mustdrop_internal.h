@@ -30,6 +30,7 @@ struct FusedGeometry {
   int32_t cpl;        // tensor-memory columns per lane and head (= tk / halves)
   int32_t n_stage;    // shared-memory stages
   int32_t n_buf;      // tensor-memory buffers
+  int32_t n_slot;     // statistics slots: 2 x n_buf, or 4 with the exp warps held within two heads of the add warps
   int32_t ach;        // chunks of 16 columns per accumulating thread (kernel variant: 5 or 10)
   size_t smem_bytes;  // dynamic shared memory
 };

@@ -41,7 +41,8 @@ constexpr int kTmaWarp = kExpWarps + kAddWarps;   // warp 12
 constexpr int kMmaWarp = kTmaWarp + 1;            // warp 13; warps 14-15 only fill the last warpgroup
 constexpr int kThreads = 16 * 32;
 constexpr int kChunk = 16;                  // TMEM columns per tcgen05.ld / st
-constexpr int kMaxCluster = 8;
+constexpr int kMaxCluster = 16;               // beyond 8 the cluster size is non-portable (opt-in per kernel)
+constexpr int kTightSlots = 4;                // statistics slots when the exp warps are held within two heads of the add warps
 constexpr int kMaxStages = 4;
 constexpr int kMinBufs = 3;                 // tensor-memory buffers: MMA, exp and add stages in flight ...
 constexpr int kMaxBufs = 8;                 // ... more when the columns per head allow, to hide the per-head latency chain
@@ -58,7 +59,8 @@ struct FusedParams {
   const int32_t* vis_cnt;             // [B] or null: vision tokens the request holds; its text keys follow them
   int32_t H, N, L, M, vis_start, txt_start, causal;
   int32_t cluster, tk, cpl, n_stage;  // CTAs per request, keys per CTA, columns per TMEM lane
-  int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (= 2 * n_buf)
+  int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (2 * n_buf, or 4 when tight)
+  int32_t tight;                      // 1: the exp warps start head h only when the add warps are done with head h - 2
   float scale_log2e, inv_heads;
 };
 
@@ -433,6 +435,16 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const int buf = h % p.n_buf;
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
       const int slot = h % p.n_slot;
+      if (p.tight && h >= 2) {
+        // Few statistics slots (large clusters): stay within two heads of the local add warps.
+        // A peer then sends for head h only after this CTA's add warps are done with head h - 4
+        // (peer at h => its add warps done with h - 2 => our pairs of h - 2 sent => ours done with
+        // h - 4), so four slots are enough whatever the number of buffers.
+        const int u = h - 2;
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tempty[u % p.n_buf]),
+                                               static_cast<uint32_t>(u / p.n_buf) & 1u, abort_flag)))
+          break;
+      }
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag))) break;
       if (threadIdx.x == 0) {
         MD_TRACE(h, 3);
@@ -779,6 +791,11 @@ int max_resident_clusters(int halves, int ach, int cluster, size_t smem_bytes) {
     (void)cudaGetLastError();
     return 0;
   }
+  if (cluster > 8 &&
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 0;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(cluster));
   cfg.blockDim = dim3(kThreads);
@@ -818,19 +835,30 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     const int ach = cpl <= 5 * kChunk ? 5 : 10;             // chunks per add thread (kernel variant)
     const int epr = kColGroups;                             // (max, sum) pairs per row and CTA
     // As many tensor-memory buffers as the columns allow (3..8), fewer if their statistics
-    // slots (2 x buffers x cluster x rows x pairs x 8 bytes) would leave no room for 2 stages.
+    // slots (2 x buffers x cluster x rows x pairs x 8 bytes) would leave no room for 2 stages;
+    // if even three buffers' slots do not fit (large clusters), four slots with the exp warps
+    // held within two heads of the add warps.
     int n_buf = kTmemCols / cpl;
     if (n_buf > kMaxBufs) n_buf = kMaxBufs;
     if (n_buf < kMinBufs) continue;
+    const int max_buf = n_buf;
     size_t extra = 0;
-    int n_stage = 0;
+    int n_stage = 0, n_slot = 0;
     for (; n_buf >= kMinBufs; --n_buf) {
-      extra = static_cast<size_t>(2 * n_buf) * c * nrows * epr * 8;
+      n_slot = 2 * n_buf;
+      extra = static_cast<size_t>(n_slot) * c * nrows * epr * 8;
       const size_t reserved = 4096 /* static */ + 1024 /* alignment */ + extra;
       if (reserved + 2 * stage > 227 * 1024) continue;
       n_stage = static_cast<int>((227 * 1024 - reserved) / stage);
       // a stage is held for a load latency plus an MMA (~2.3 us): prefer four stages over more buffers
       if (n_stage >= kMaxStages || n_buf == kMinBufs) break;
+    }
+    if (n_stage < 2) {
+      n_buf = max_buf;
+      n_slot = kTightSlots;
+      extra = static_cast<size_t>(n_slot) * c * nrows * epr * 8;
+      const size_t reserved = 4096 + 1024 + extra;
+      n_stage = reserved + 2 * stage > 227 * 1024 ? 0 : static_cast<int>((227 * 1024 - reserved) / stage);
     }
     if (n_stage < 2) continue;
     if (n_stage > kMaxStages) n_stage = kMaxStages;
@@ -841,16 +869,18 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     // at least 116 KB, so that two CTAs (each wanting all of tensor memory) never share an SM
     if (smem_bytes < 116 * 1024) smem_bytes = 116 * 1024;
     int resident = max_resident_clusters(halves, ach, c, smem_bytes);
-    if (resident <= 0) resident = sm_count / c;    // no device to ask: ignore GPC boundaries
+    if (resident <= 0 && c <= 8) resident = sm_count / c;    // no device to ask: ignore GPC boundaries
+    // (a cluster of more than 8 CTAs is used only where the device says it can hold one)
     if (resident <= 0) continue;
     const long waves = (r.B + resident - 1) / resident;
     const double t_stream = static_cast<double>(stage) / 45.0e3;
-    const double t_chain = 4.5 / n_buf;
+    const double t_chain = 4.5 / (n_slot < 2 * n_buf ? 2 : n_buf);   // tight slots: two heads in flight
     const double t_head = t_stream > t_chain ? t_stream : t_chain;
     const double score = 1.0 / (static_cast<double>(waves) * t_head) - 1e-4 * c;   // prefer smaller clusters among equals
     if (score > best) {
       best = score;
       g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_stage = n_stage; g.n_buf = n_buf; g.ach = ach;
+      g.n_slot = n_slot;
       g.smem_bytes = smem_bytes;
     }
   }
@@ -880,7 +910,7 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, c
   p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
   p.causal = r.causal;
   p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_stage = geo.n_stage;
-  p.n_buf = geo.n_buf; p.n_slot = 2 * geo.n_buf;
+  p.n_buf = geo.n_buf; p.n_slot = geo.n_slot; p.tight = geo.n_slot < 2 * geo.n_buf;
   p.scale_log2e = r.scale_log2e;
   p.inv_heads = 1.0f / static_cast<float>(r.H);
 
@@ -888,6 +918,10 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, c
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem_bytes));
   if (e != cudaSuccess) return e;
+  if (geo.cluster > 8) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(r.B * geo.cluster));
   cfg.blockDim = dim3(kThreads);

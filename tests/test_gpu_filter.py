@@ -44,7 +44,7 @@ def _skip_unless_fused(w):
         pytest.skip("this shape does not fit the fused kernel at that cluster size")
 
 
-@pytest.mark.parametrize("cluster", [0, 1, 2, 3, 5, 8], indirect=True)
+@pytest.mark.parametrize("cluster", [0, 1, 2, 3, 5, 8, 11, 16], indirect=True)
 def test_filter_small_ragged_batch(cluster):
     # 5 requests, ragged sizes, vision span not at 0, more kept rows than CTAs in the cluster
     w = small(batch=5, n_vis=333 if cluster != 1 else 270, n_txt=21, n_heads=3, hidden=384, key_cnt=9, budget=40,
@@ -73,10 +73,16 @@ def test_filter_13b_batch64_sampled():
     run_chain_and_check(synth.WORKLOADS["c5_13b_b64"], sample=[17], path="filter", expect_launches=1)
 
 
-def test_filter_falls_back_to_separate_launches_for_long_sequences():
-    # 2880 vision tokens are outside the fused kernel's key range: the call still does the whole step
-    w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
+def test_filter_falls_back_to_separate_launches_where_the_fused_geometry_does_not_fit():
+    # 2048 vision tokens with 96 text rows are outside the fused kernel's range: the call still does the whole step
+    w = synth.WORKLOADS["c4_video"].with_(batch=2)
     run_chain_and_check(w, sample=[1], path="filter", expect_launches=4)
+
+
+def test_filter_next7b_runs_on_a_cluster_of_more_than_eight():
+    # 2944 keys per request need more than 8 CTAs x 320 keys: non-portable cluster size, four statistics slots
+    w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
+    run_chain_and_check(w, sample=[1], path="filter", expect_launches=1)
 
 
 def _run_both(w, monkeypatch, cfg_kw=None, drop=()):

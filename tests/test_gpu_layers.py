@@ -123,9 +123,14 @@ def test_ragged_layer_llava7b_batch16_sampled():
     assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[0, 11]) == 1
 
 
-def test_ragged_layer_next7b_falls_back():
-    w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
+def test_ragged_layer_video_falls_back_to_the_two_pass_score():
+    w = synth.WORKLOADS["c4_video"].with_(batch=2)
     assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[1]) == 4
+
+
+def test_ragged_layer_next7b_on_a_large_cluster():
+    w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
+    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[1]) == 1
 
 
 @pytest.mark.parametrize("path", ["one_launch", "two_pass"], indirect=True)

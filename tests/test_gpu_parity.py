@@ -29,7 +29,7 @@ def small(**kw):
     return TINY.with_(**base)
 
 
-VARIANTS = ["auto", "two_pass", "fused:1", "fused:2", "fused:3", "fused:5", "fused:8"]
+VARIANTS = ["auto", "two_pass", "fused:1", "fused:2", "fused:3", "fused:5", "fused:8", "fused:12", "fused:16"]
 
 
 @pytest.fixture
