@@ -356,7 +356,7 @@ def run_ours(args, w):
                        "n_heads": w.n_heads, "hidden": w.hidden, "budget": w.budget, "key_set": w.key_cnt,
                        "parallelism": "dp%d (independent requests, no collective)" % world,
                        "l2": "inputs exceed L2 (K alone is %.0f MB per GPU)" % (bm["score"] / 1e6),
-                       "score_variant": f.score_variant,
+                       "score_variant": f.score_variant, "plan": f.description,
                        "path": ("mustdrop_filter, %d launch(es) per step" % launches_per_step) if single_call
                        else "mustdrop_score + mustdrop_select + mustdrop_compact"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bm["h2d"], "d2h_bytes_per_step": bm["d2h"],

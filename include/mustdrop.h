@@ -324,6 +324,13 @@ int32_t mustdrop_last_cuda_error(void);
 /* Name of the score kernel variant the plan selected (static string; for logs and benchmarks). */
 const char *mustdrop_plan_score_variant(const mustdrop_plan_t *plan);
 
+/*
+ * One-line description of what the plan will launch (kernel variant, cluster size, keys per CTA,
+ * stages, buffers), for logs and benchmarks.  buf (host) receives at most n bytes including the
+ * terminating zero; returns the length the full text needs.
+ */
+int32_t mustdrop_plan_describe(const mustdrop_plan_t *plan, char *buf /* (host) */, size_t n);
+
 #ifdef __cplusplus
 }
 #endif

@@ -35,6 +35,7 @@ EXPORTS = (
     "mustdrop_last_cuda_error", "mustdrop_plan_score_variant", "mustdrop_score_static",
     "mustdrop_score_static_max_rows", "mustdrop_filter", "mustdrop_plan_filter_launches",
     "mustdrop_filter_layer", "mustdrop_cache_compact", "mustdrop_spatial_merge", "mustdrop_key_set",
+    "mustdrop_plan_describe",
 )
 
 
@@ -267,6 +268,15 @@ def mustdrop_key_set(batch, n_heads, head_dim, n_tokens, key_max, q_cls, k, a_cl
                                   _ptr(mu_out), _ptr(key_idx), _ptr(key_cnt), _stream(stream))
 
 
+def mustdrop_plan_describe(plan) -> str:
+    buf = ctypes.create_string_buffer(256)
+    L = lib()
+    L.mustdrop_plan_describe.argtypes = [ctypes.c_void_p, ctypes.c_char_p, ctypes.c_size_t]
+    L.mustdrop_plan_describe.restype = ctypes.c_int32
+    L.mustdrop_plan_describe(plan, buf, 256)
+    return buf.value.decode()
+
+
 def mustdrop_plan_filter_launches(plan) -> int:
     return lib().mustdrop_plan_filter_launches(plan)
 
@@ -386,6 +396,10 @@ class Filter:
         st, code, detail = mustdrop_device_status(self.plan, self.workspace, stream)
         self._check(st, "mustdrop_device_status")
         return code, detail
+
+    @property
+    def description(self) -> str:
+        return mustdrop_plan_describe(self.plan)
 
     @property
     def score_variant(self) -> str:

@@ -1,6 +1,7 @@
 // C-ABI layer: configuration checks, plan object, argument checks, kernel dispatch.
 // The operations themselves are defined by Sec. 3.4 (Eq. 8-10) of the paper; see mustdrop.h.
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -120,7 +121,17 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
     const char* cl = std::getenv("MUSTDROP_CLUSTER");
     const int forced_cluster = cl ? std::atoi(cl) : 0;
     const bool allow_fused = !(want && std::strcmp(want, "two_pass") == 0);
-    if (allow_fused && plan_score_fused(r, p->sm_count, forced_cluster, &p->fused)) p->score_variant = kScoreFusedCluster;
+    if (allow_fused && plan_score_fused(r, p->sm_count, forced_cluster, &p->fused)) {
+      p->score_variant = kScoreFusedCluster;
+      // A fused plan that had to fall back to few statistics slots (sequences needing clusters of
+      // more than 8 CTAs) can be slower than reading K twice: compare with the two-pass kernel's
+      // measured rate (about 0.6 + 0.7 * N / 128 us per MB of keys) unless the variant is forced.
+      const bool tight = p->fused.n_slot < 2 * p->fused.n_buf;
+      const double k_mb = 256.0e-6 * r.B * r.H * r.L;
+      const double two_pass_us = k_mb * (0.6 + 0.7 * r.N / 128.0);
+      if (tight && want == nullptr && forced_cluster == 0 && p->fused.est_us > two_pass_us)
+        p->score_variant = kScoreTwoPassMma;
+    }
     // mustdrop_filter: one launch where the fused kernel covers the shape and a kept row fits its
     // shared-memory ring; MUSTDROP_FILTER=staged forces the three launches (debugging override).
     const char* fw = std::getenv("MUSTDROP_FILTER");
@@ -319,6 +330,24 @@ const char* mustdrop_plan_score_variant(const mustdrop_plan_t* plan) {
     case mustdrop::kScoreFusedCluster: return "fused_cluster_tcgen05";
   }
   return "unknown";
+}
+
+int32_t mustdrop_plan_describe(const mustdrop_plan_t* plan, char* buf, size_t n) {
+  if (!valid_plan(plan)) return -1;
+  char text[256];
+  int len;
+  if (plan->score_variant == mustdrop::kScoreFusedCluster) {
+    const mustdrop::FusedGeometry& g = plan->fused;
+    len = std::snprintf(text, sizeof(text),
+                        "fused tcgen05 score: cluster %d, %d keys per CTA, %d stages, %d tensor-memory buffers, "
+                        "%d statistics slots, %d clusters resident; filter = %d launch(es)",
+                        g.cluster, g.tk, g.n_stage, g.n_buf, g.n_slot, g.resident, mustdrop_plan_filter_launches(plan));
+  } else {
+    len = std::snprintf(text, sizeof(text), "two-pass mma.sync score; filter = %d launch(es)",
+                        mustdrop_plan_filter_launches(plan));
+  }
+  if (buf != nullptr && n > 0) std::snprintf(buf, n, "%s", text);
+  return len;
 }
 
 }  // extern "C"

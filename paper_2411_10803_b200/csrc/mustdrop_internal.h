@@ -30,8 +30,10 @@ struct FusedGeometry {
   int32_t cpl;        // tensor-memory columns per lane and head (= tk / halves)
   int32_t n_stage;    // shared-memory stages
   int32_t n_buf;      // tensor-memory buffers
-  int32_t n_slot;     // statistics slots: 2 x n_buf, or 4 with the exp warps held within two heads of the add warps
+  int32_t n_slot;     // statistics slots: 2 x n_buf, or 2d (d = 2 or 1) with the exp warps held within d heads of the add warps
   int32_t ach;        // chunks of 16 columns per accumulating thread (kernel variant: 5 or 10)
+  int32_t resident;   // clusters the device can hold at once (0: not asked)
+  float est_us;       // the planner's estimate of the score time
   size_t smem_bytes;  // dynamic shared memory
 };
 

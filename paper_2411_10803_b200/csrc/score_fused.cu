@@ -42,7 +42,6 @@ constexpr int kMmaWarp = kTmaWarp + 1;            // warp 13; warps 14-15 only f
 constexpr int kThreads = 16 * 32;
 constexpr int kChunk = 16;                  // TMEM columns per tcgen05.ld / st
 constexpr int kMaxCluster = 16;               // beyond 8 the cluster size is non-portable (opt-in per kernel)
-constexpr int kTightSlots = 4;                // statistics slots when the exp warps are held within two heads of the add warps
 constexpr int kMaxStages = 4;
 constexpr int kMinBufs = 3;                 // tensor-memory buffers: MMA, exp and add stages in flight ...
 constexpr int kMaxBufs = 8;                 // ... more when the columns per head allow, to hide the per-head latency chain
@@ -60,7 +59,7 @@ struct FusedParams {
   int32_t H, N, L, M, vis_start, txt_start, causal;
   int32_t cluster, tk, cpl, n_stage;  // CTAs per request, keys per CTA, columns per TMEM lane
   int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (2 * n_buf, or 4 when tight)
-  int32_t tight;                      // 1: the exp warps start head h only when the add warps are done with head h - 2
+  int32_t tight;                      // d = 1 or 2: the exp warps start head h only when the add warps are done with head h - d (0: no such rule)
   float scale_log2e, inv_heads;
 };
 
@@ -435,12 +434,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const int buf = h % p.n_buf;
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
       const int slot = h % p.n_slot;
-      if (p.tight && h >= 2) {
-        // Few statistics slots (large clusters): stay within two heads of the local add warps.
-        // A peer then sends for head h only after this CTA's add warps are done with head h - 4
-        // (peer at h => its add warps done with h - 2 => our pairs of h - 2 sent => ours done with
-        // h - 4), so four slots are enough whatever the number of buffers.
-        const int u = h - 2;
+      if (p.tight && h >= p.tight) {
+        // Few statistics slots (large clusters): stay within d = p.tight heads of the local add
+        // warps.  A peer then sends for head h only after this CTA's add warps are done with head
+        // h - 2d (peer at h => its add warps done with h - d => our pairs of h - d sent => ours
+        // done with h - 2d), so 2d slots are enough whatever the number of buffers.
+        const int u = h - p.tight;
         if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tempty[u % p.n_buf]),
                                                static_cast<uint32_t>(u / p.n_buf) & 1u, abort_flag)))
           break;
@@ -461,7 +460,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 #pragma unroll
       for (int t = 0; t < ECH; ++t)
         if (t < my_chunks) tc_ld16(tbuf + kChunk * (g + t * kColGroups), z[t]);
-      if (h > 0) {
+      if (h > 0 && !p.tight) {
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -507,6 +506,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           st_async_f32x2(map_to_cta(slot_addr, c), mx, lsum, map_to_cta(bar_addr, c));
       }
       last_buf = buf;
+      if (p.tight) {   // hand over at once: the add warps of this head gate our next heads
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[buf]));
+        last_buf = -1;
+      }
       if (threadIdx.x == 0) MD_TRACE(h, 4);
     }
     if (last_buf >= 0) {   // hand over the last head that was worked on
@@ -853,9 +859,9 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
       // a stage is held for a load latency plus an MMA (~2.3 us): prefer four stages over more buffers
       if (n_stage >= kMaxStages || n_buf == kMinBufs) break;
     }
-    if (n_stage < 2) {
+    for (int d = 2; d >= 1 && n_stage < 2; --d) {   // tight: 2d slots, exp warps within d heads of the add warps
       n_buf = max_buf;
-      n_slot = kTightSlots;
+      n_slot = 2 * d;
       extra = static_cast<size_t>(n_slot) * c * nrows * epr * 8;
       const size_t reserved = 4096 + 1024 + extra;
       n_stage = reserved + 2 * stage > 227 * 1024 ? 0 : static_cast<int>((227 * 1024 - reserved) / stage);
@@ -874,13 +880,20 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     if (resident <= 0) continue;
     const long waves = (r.B + resident - 1) / resident;
     const double t_stream = static_cast<double>(stage) / 45.0e3;
-    const double t_chain = 4.5 / (n_slot < 2 * n_buf ? 2 : n_buf);   // tight slots: two heads in flight
+    double t_chain = 4.5 / n_buf;
+    if (n_slot < 2 * n_buf) {
+      // Tight slots: the exchange over the cluster is on the critical path of every head (d = 2)
+      // or of every head twice (d = 1).  Measured per head: 2.6 .. 3.3 us at 11 .. 16 CTAs with
+      // d = 2, 4.3 us at 10 CTAs with d = 1; a third more with 128 text rows on the lanes.
+      t_chain = (n_slot == 4 ? 1.8 + 0.09 * c : 3.0 + 0.13 * c) * (halves == 1 ? 1.3 : 1.0);
+    }
     const double t_head = t_stream > t_chain ? t_stream : t_chain;
     const double score = 1.0 / (static_cast<double>(waves) * t_head) - 1e-4 * c;   // prefer smaller clusters among equals
     if (score > best) {
       best = score;
       g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_stage = n_stage; g.n_buf = n_buf; g.ach = ach;
-      g.n_slot = n_slot;
+      g.n_slot = n_slot; g.resident = resident;
+      g.est_us = static_cast<float>(waves * r.H * t_head);
       g.smem_bytes = smem_bytes;
     }
   }
@@ -910,7 +923,7 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, c
   p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
   p.causal = r.causal;
   p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_stage = geo.n_stage;
-  p.n_buf = geo.n_buf; p.n_slot = geo.n_slot; p.tight = geo.n_slot < 2 * geo.n_buf;
+  p.n_buf = geo.n_buf; p.n_slot = geo.n_slot; p.tight = geo.n_slot < 2 * geo.n_buf ? geo.n_slot / 2 : 0;
   p.scale_log2e = r.scale_log2e;
   p.inv_heads = 1.0f / static_cast<float>(r.H);
 

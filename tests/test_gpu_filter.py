@@ -74,13 +74,21 @@ def test_filter_13b_batch64_sampled():
 
 
 def test_filter_falls_back_to_separate_launches_where_the_fused_geometry_does_not_fit():
-    # 2048 vision tokens with 96 text rows are outside the fused kernel's range: the call still does the whole step
+    # 4000 vision tokens with 100 text rows exceed 16 CTAs x 160 keys: the call still does the whole step
+    w = synth.WORKLOADS["c4_video"].with_(batch=1, n_vis=4000, n_txt=100, n_heads=2, hidden=256, budget=300)
+    run_chain_and_check(w, path="filter", expect_launches=4)
+
+
+def test_filter_video_runs_on_a_large_cluster_with_two_statistics_slots(monkeypatch):
+    # (the planner prefers the two-pass kernel for this shape: force the fused one)
+    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "fused")
     w = synth.WORKLOADS["c4_video"].with_(batch=2)
-    run_chain_and_check(w, sample=[1], path="filter", expect_launches=4)
+    run_chain_and_check(w, sample=[1], path="filter", expect_launches=1)
 
 
-def test_filter_next7b_runs_on_a_cluster_of_more_than_eight():
-    # 2944 keys per request need more than 8 CTAs x 320 keys: non-portable cluster size, four statistics slots
+def test_filter_next7b_runs_on_a_cluster_of_more_than_eight(monkeypatch):
+    # 2944 keys per request need more than 8 CTAs x 320 keys: non-portable cluster size, few statistics slots
+    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "fused")
     w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
     run_chain_and_check(w, sample=[1], path="filter", expect_launches=1)
 

@@ -123,12 +123,19 @@ def test_ragged_layer_llava7b_batch16_sampled():
     assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[0, 11]) == 1
 
 
-def test_ragged_layer_video_falls_back_to_the_two_pass_score():
+def test_ragged_layer_long_sequence_falls_back_to_the_two_pass_score():
+    w = synth.WORKLOADS["c4_video"].with_(batch=2, n_vis=4000, n_txt=100, n_heads=2, hidden=256, budget=300)
+    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True) == 4
+
+
+def test_ragged_layer_video_on_a_large_cluster(monkeypatch):
+    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "fused")
     w = synth.WORKLOADS["c4_video"].with_(batch=2)
-    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[1]) == 4
+    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[1]) == 1
 
 
-def test_ragged_layer_next7b_on_a_large_cluster():
+def test_ragged_layer_next7b_on_a_large_cluster(monkeypatch):
+    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "fused")
     w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
     assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[1]) == 1
 
