@@ -39,7 +39,8 @@ def _load():
     global _lib
     if _lib is None:
         _lib = ctypes.CDLL(build())
-        for name in ("mustdrop_oracle_attention", "mustdrop_oracle_score", "mustdrop_oracle_select",
+        for name in ("mustdrop_oracle_attention", "mustdrop_oracle_score", "mustdrop_oracle_score_per_head",
+                     "mustdrop_oracle_select",
                      "mustdrop_oracle_compact"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
@@ -85,6 +86,22 @@ def score(q_text: np.ndarray, k: np.ndarray, vis_start: int, n_vis: int, txt_sta
     if rc:
         raise ValueError("mustdrop_oracle_score rejected its arguments")
     return (G, I, a) if return_a else (G, I)
+
+
+def score_per_head(q_text: np.ndarray, k: np.ndarray, vis_start: int, n_vis: int, txt_start: int,
+                   causal: bool = True, scale: float = 0.0):
+    """The per-head reading of Eq. 10: I = head mean of the per-head maxima over text rows; G as in score()."""
+    q_text, k = _c(q_text, np.uint16), _c(k, np.uint16)
+    B, H, N, D = q_text.shape
+    L = k.shape[2]
+    assert k.shape == (B, H, L, D)
+    G = np.empty((B, n_vis), np.float32)
+    I = np.empty((B, n_vis), np.float32)
+    rc = _load().mustdrop_oracle_score_per_head(_p(q_text), _p(k), B, H, N, L, D, int(vis_start), int(n_vis),
+                                                int(txt_start), int(bool(causal)), ctypes.c_double(scale), _p(G), _p(I))
+    if rc:
+        raise ValueError("mustdrop_oracle_score_per_head rejected its arguments")
+    return G, I
 
 
 def select(G: np.ndarray, I: np.ndarray, seq_len: int, key_idx: Optional[np.ndarray] = None,

@@ -117,6 +117,43 @@ int mustdrop_oracle_score(const uint16_t *q_text, const uint16_t *k, int B, int 
     return 0;
 }
 
+/*
+ * The other reading of Eq. 10 over heads (the paper does not say how heads enter): the maximum
+ * over text tokens is taken per head and the maxima are averaged,
+ *   I[j] = (1/H) sum_h max_i p^h[i][vis_start + j],
+ * instead of the maximum of the head mean.  G (Eq. 8) is linear in the heads and is unchanged.
+ */
+int mustdrop_oracle_score_per_head(const uint16_t *q_text, const uint16_t *k, int B, int H, int N, int L, int D,
+                                   int vis_start, int M, int txt_start, int causal, double scale,
+                                   float *g_out, float *i_out)
+{
+    if (!q_text || !k || !g_out || !i_out) return -1;
+    if (B <= 0 || M <= 0 || vis_start < 0 || vis_start + M > txt_start || txt_start + N > L) return -1;
+    double *p = (double *)malloc(sizeof(double) * (size_t)H * N * L);
+    if (!p) return -1;
+    for (int b = 0; b < B; ++b) {
+        const uint16_t *qb = q_text + (size_t)b * H * N * D;
+        const uint16_t *kb = k + (size_t)b * H * L * D;
+        if (mustdrop_oracle_attention(qb, kb, H, N, L, D, txt_start, causal, scale, p)) { free(p); return -1; }
+        for (int j = 0; j < M; ++j) {
+            double g = 0.0, isum = 0.0;
+            for (int h = 0; h < H; ++h) {
+                double mx = -INFINITY;
+                for (int i = 0; i < N; ++i) {
+                    double v = p[((size_t)h * N + i) * L + vis_start + j];
+                    g += v;
+                    if (v > mx) mx = v;
+                }
+                isum += mx;
+            }
+            g_out[(size_t)b * M + j] = (float)(g / (double)H);
+            i_out[(size_t)b * M + j] = (float)(isum / (double)H);
+        }
+    }
+    free(p);
+    return 0;
+}
+
 /* ---- selection ------------------------------------------------------------------------- */
 
 enum { MODE_BUDGET = 0, MODE_THRESHOLD = 1 };

@@ -196,3 +196,25 @@ def test_planted_salient_keys_score_high():
     sal = d["salient_idx"][0]
     rest = np.setdiff1d(np.arange(w.n_vis), sal)
     assert G[0, sal].min() > np.median(G[0, rest]) * 1.5
+
+
+# ---- the per-head reading of Eq. 10 --------------------------------------------------------------
+
+def test_per_head_reading_coincides_with_one_head_and_dominates_otherwise():
+    w = synth.WORKLOADS["c1_tiny"].with_(batch=2, n_vis=40, n_txt=6, n_heads=1, hidden=128, n_salient=2, key_cnt=0, budget=8)
+    d = synth.make_batch(w, with_values=False)
+    G1, I1 = oracle.score(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start)
+    G2, I2 = oracle.score_per_head(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start)
+    assert np.array_equal(G1, G2) and np.array_equal(I1, I2)            # H = 1: one reading
+    w = w.with_(n_heads=4, hidden=512)
+    d = synth.make_batch(w, with_values=False)
+    G1, I1 = oracle.score(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start)
+    G2, I2 = oracle.score_per_head(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start)
+    assert np.allclose(G1, G2, rtol=1e-6)                                # G is linear in the heads
+    assert np.all(I2 >= I1 * (1 - 1e-6)) and np.any(I2 > I1 * 1.01)      # a mean of maxima is at least the maximum of the mean
+    # against the attention map itself: the definition written with numpy
+    for b in range(w.batch):
+        p = oracle.attention(d["q_text"][b], d["k"][b], w.txt_start)     # [H, N, L]
+        pv = p[:, :, w.vis_start:w.vis_start + w.n_vis]
+        assert np.allclose(I2[b], pv.max(axis=1).mean(axis=0), rtol=1e-6)
+        assert np.allclose(G2[b], pv.mean(axis=0).sum(axis=0), rtol=1e-6)
