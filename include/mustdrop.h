@@ -69,6 +69,14 @@ typedef enum {
  */
 #define MUSTDROP_FLAG_REBUILD_SEQUENCE 1
 
+/*
+ * MUSTDROP_FLAG_PER_HEAD_MAX: the other reading of Eq. 10 over attention heads, which the paper
+ * leaves open: i_out[b][j] = mean over heads of ( max over text tokens of p^h[i][vis_start + j] )
+ * instead of the maximum of the head-mean attention.  g_out (Eq. 8) is the same under both.
+ * Plans with this flag run the two-pass score kernel.
+ */
+#define MUSTDROP_FLAG_PER_HEAD_MAX 2
+
 typedef struct {
   int32_t batch;      /* B, independent requests */
   int32_t n_heads;    /* H */

@@ -54,6 +54,7 @@ class mustdrop_config_t(ctypes.Structure):
 
 
 MUSTDROP_FLAG_REBUILD_SEQUENCE = 1
+MUSTDROP_FLAG_PER_HEAD_MAX = 2
 
 
 class mustdrop_layer_io_t(ctypes.Structure):

@@ -39,7 +39,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   *workspace_bytes = 0;
   if (c->batch <= 0 || c->n_heads <= 0 || c->head_dim <= 0 || c->hidden <= 0 || c->seq_len <= 0 ||
       c->n_vis <= 0 || c->n_txt <= 0 || c->vis_start < 0 || c->txt_start < 0 || c->key_max < 0 ||
-      (c->flags & ~MUSTDROP_FLAG_REBUILD_SEQUENCE) != 0)
+      (c->flags & ~(MUSTDROP_FLAG_REBUILD_SEQUENCE | MUSTDROP_FLAG_PER_HEAD_MAX)) != 0)
     return MUSTDROP_ERR_INVALID_ARG;
   // the vision span precedes the text span and both lie inside the sequence
   if (static_cast<int64_t>(c->vis_start) + c->n_vis > c->txt_start ||
@@ -79,6 +79,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   r.key_max = c->key_max;
   r.cap = (c->mode == MUSTDROP_MODE_BUDGET) ? c->budget : c->n_vis;
   r.rebuild = (c->flags & MUSTDROP_FLAG_REBUILD_SEQUENCE) ? 1 : 0;
+  r.per_head_max = (c->flags & MUSTDROP_FLAG_PER_HEAD_MAX) ? 1 : 0;
   r.out_rows = r.rebuild ? c->vis_start + r.cap + c->n_txt : r.cap;
   r.gamma_default = c->gamma == 0.0f;
   r.alpha_default = c->alpha == 0.0f;
@@ -120,7 +121,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
     const char* want = std::getenv("MUSTDROP_SCORE_VARIANT");
     const char* cl = std::getenv("MUSTDROP_CLUSTER");
     const int forced_cluster = cl ? std::atoi(cl) : 0;
-    const bool allow_fused = !(want && std::strcmp(want, "two_pass") == 0);
+    const bool allow_fused = !(want && std::strcmp(want, "two_pass") == 0) && !r.per_head_max;
     if (allow_fused && plan_score_fused(r, p->sm_count, forced_cluster, &p->fused)) {
       p->score_variant = kScoreFusedCluster;
       // A fused plan that had to fall back to few statistics slots (sequences needing clusters of

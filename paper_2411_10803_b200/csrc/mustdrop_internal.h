@@ -47,6 +47,7 @@ struct FilterGeometry {
 struct Resolved {
   int32_t B, H, D, hidden, L, vis_start, M, txt_start, N;
   int32_t causal, mode, criteria, budget, key_max, cap;
+  int32_t per_head_max;   // Eq. 10 per head, then the head mean (two-pass kernel only)
   int32_t rebuild;        // outputs hold [prefix ; kept vision ; text] instead of the kept vision rows only
   int32_t out_rows;       // rows per request (and head) of hidden_out / k_out / v_out
   int32_t gamma_default, alpha_default;   // thresholds follow each request's own sizes (ragged batches)

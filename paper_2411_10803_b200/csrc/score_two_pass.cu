@@ -28,6 +28,7 @@ struct ScoreParams {
   float* i_out;             // [B,M]
   const int32_t* vis_cnt;   // [B] or null: vision tokens the request holds; its text keys follow them
   int32_t H, N, L, M, vis_start, txt_start, causal, n_warps;
+  int32_t per_head_max;     // 1: i_out = head mean of the per-head column maxima
   float scale_log2e, inv_heads;
   int64_t k_sb, k_sh, k_sl;
 };
@@ -188,6 +189,7 @@ __global__ void __launch_bounds__(256) accumulate_kernel(ScoreParams p) {
   __nv_bfloat16* stage0 = reinterpret_cast<__nv_bfloat16*>(smem_raw);
   __nv_bfloat16* stage1 = stage0 + stage_elems;
   float* red = reinterpret_cast<float*>(stage1 + stage_elems);  // [2][n_warps][64]
+  float* imax_s = red + 2 * p.n_warps * kTileKeys;              // [64] sum over heads of the per-head column maxima
   const int vt = blockIdx.x, b = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int n_threads = blockDim.x;
@@ -205,6 +207,7 @@ __global__ void __launch_bounds__(256) accumulate_kernel(ScoreParams p) {
     cp_async_commit();
   };
   stage_head(stage0, 0);
+  for (int col = threadIdx.x; col < kTileKeys; col += n_threads) imax_s[col] = 0.0f;
 
   const int row0 = warp * 16 + g, row1 = row0 + 8;
   float acc[8][4];
@@ -230,10 +233,31 @@ __global__ void __launch_bounds__(256) accumulate_kernel(ScoreParams p) {
     for (int nb = 0; nb < 8; ++nb) {
       float c[4];
       tile_block_logits(c, a, k_s, nb, lane);
-      acc[nb][0] += exp2f(c[0] * p.scale_log2e - st0.x) * st0.y;
-      acc[nb][1] += exp2f(c[1] * p.scale_log2e - st0.x) * st0.y;
-      acc[nb][2] += exp2f(c[2] * p.scale_log2e - st1.x) * st1.y;
-      acc[nb][3] += exp2f(c[3] * p.scale_log2e - st1.x) * st1.y;
+      const float p0 = exp2f(c[0] * p.scale_log2e - st0.x) * st0.y, p1 = exp2f(c[1] * p.scale_log2e - st0.x) * st0.y;
+      const float p2 = exp2f(c[2] * p.scale_log2e - st1.x) * st1.y, p3 = exp2f(c[3] * p.scale_log2e - st1.x) * st1.y;
+      acc[nb][0] += p0; acc[nb][1] += p1; acc[nb][2] += p2; acc[nb][3] += p3;
+      if (p.per_head_max) {
+        // this head's column maxima over the warp's 16 rows (rows at or beyond N do not take part)
+        float m0 = fmaxf(row0 < p.N ? p0 : -INFINITY, row1 < p.N ? p2 : -INFINITY);
+        float m1 = fmaxf(row0 < p.N ? p1 : -INFINITY, row1 < p.N ? p3 : -INFINITY);
+#pragma unroll
+        for (int d = 4; d <= 16; d <<= 1) {
+          m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, d));
+          m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, d));
+        }
+        if (g == 0) {
+          red[warp * kTileKeys + nb * 8 + 2 * t] = m0;
+          red[warp * kTileKeys + nb * 8 + 2 * t + 1] = m1;
+        }
+      }
+    }
+    if (p.per_head_max) {   // over the warps, then onto the running head sum
+      __syncthreads();
+      for (int col = threadIdx.x; col < kTileKeys; col += n_threads) {
+        float mx = -INFINITY;
+        for (int w = 0; w < p.n_warps; ++w) mx = fmaxf(mx, red[w * kTileKeys + col]);
+        imax_s[col] += mx;
+      }
     }
     __syncthreads();
   }
@@ -267,6 +291,7 @@ __global__ void __launch_bounds__(256) accumulate_kernel(ScoreParams p) {
       s += red[w * kTileKeys + col];
       mx = fmaxf(mx, red[(p.n_warps + w) * kTileKeys + col]);
     }
+    if (p.per_head_max) mx = imax_s[col];
     if (col >= valid_keys) s = mx = 0.0f;   // beyond the request's own tokens
     p.g_out[static_cast<int64_t>(b) * p.M + j_base + col] = s * p.inv_heads;
     p.i_out[static_cast<int64_t>(b) * p.M + j_base + col] = mx * p.inv_heads;
@@ -284,6 +309,7 @@ cudaError_t launch_score_two_pass(const mustdrop_plan& plan, const void* q_text,
   p.rowstats = static_cast<float2*>(rowstats);
   p.g_out = g_out; p.i_out = i_out;
   p.vis_cnt = vis_cnt;
+  p.per_head_max = r.per_head_max;
   p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
   p.causal = r.causal;
   p.n_warps = (r.N + 15) / 16;
@@ -294,7 +320,7 @@ cudaError_t launch_score_two_pass(const mustdrop_plan& plan, const void* q_text,
   const int threads = p.n_warps * 32;
   const size_t smem1 = sizeof(__nv_bfloat16) * static_cast<size_t>(n_rows + 2 * kTileKeys) * kRowStride;
   const size_t smem2 = sizeof(__nv_bfloat16) * 2 * static_cast<size_t>(n_rows + kTileKeys) * kRowStride +
-                       sizeof(float) * 2 * p.n_warps * kTileKeys;
+                       sizeof(float) * (2 * p.n_warps + 1) * kTileKeys;
   cudaError_t e = cudaFuncSetAttribute(rowstats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem1));
   if (e != cudaSuccess) return e;

@@ -374,3 +374,44 @@ def test_chain_is_deterministic():
     assert torch.equal(a[0], f.g) and torch.equal(a[1], f.i) and torch.equal(a[2], f.kept_idx)
     assert torch.equal(a[3], f.hidden_out)
     f.close()
+
+
+# ---- the per-head reading of Eq. 10 (MUSTDROP_FLAG_PER_HEAD_MAX) ------------------------------------
+
+@pytest.mark.parametrize("causal", [1, 0])
+@pytest.mark.parametrize("kw", [dict(), dict(batch=3, n_vis=333, n_txt=21, n_heads=5, hidden=640, vis_start=2),
+                                dict(batch=2, n_vis=130, n_txt=100, n_heads=2, hidden=256)])
+def test_score_per_head_max_matches_oracle(kw, causal):
+    w = small(**kw)
+    d = synth.make_batch(w, with_values=False)
+    f = md.Filter(md.config_for(w, causal=causal, flags=md.MUSTDROP_FLAG_PER_HEAD_MAX))
+    assert f.score_variant == "two_pass_mma"
+    f.score(to_dev_bf16(d["q_text"]), to_dev_bf16(d["k"]))
+    torch.cuda.synchronize()
+    G, I = oracle.score_per_head(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start, causal=bool(causal))
+    assert_scores_close(f.g.cpu().numpy(), G, "G")
+    assert_scores_close(f.i.cpu().numpy(), I, "I (per head)")
+    # and it is not the other reading
+    _, I_mean_first = oracle.score(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start, causal=bool(causal))
+    assert np.any(np.abs(f.i.cpu().numpy() - I_mean_first) > 1e-2 * I_mean_first)
+    f.close()
+
+
+def test_filter_call_with_per_head_max_selects_by_the_per_head_scores():
+    w = synth.WORKLOADS["c2_llava7b_b16"].with_(batch=3)
+    d = synth.make_batch(w)
+    f = md.Filter(md.config_for(w, flags=md.MUSTDROP_FLAG_PER_HEAD_MAX))
+    q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
+    ki, kc = key_args(w, d)
+    f.filter(q, k, v, hid, ki, kc, want_s=True)
+    torch.cuda.synchronize()
+    assert f.device_status() == (0, 0)
+    G, I = oracle.score_per_head(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start)
+    ref_idx, ref_cnt, ref_s, _ = oracle.select(G, I, w.seq_len, d["key_idx"], d["key_cnt"], budget=w.budget)
+    idx, cnt = f.kept_idx.cpu().numpy(), f.kept_cnt.cpu().numpy()
+    assert_kept_matches(idx, cnt, ref_idx, ref_cnt, ref_s, d["key_idx"], d["key_cnt"])
+    zh, zk, zv = (np.zeros_like(bf16_bits(t)) for t in (f.hidden_out, f.k_out, f.v_out))
+    eh, ek, ev = host_gather(idx, cnt, w.vis_start, d["hidden"], d["k"], d["v"], zh, zk, zv)
+    assert np.array_equal(bf16_bits(f.hidden_out), eh) and np.array_equal(bf16_bits(f.k_out), ek)
+    assert np.array_equal(bf16_bits(f.v_out), ev)
+    f.close()
