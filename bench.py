@@ -183,6 +183,26 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def quick_measure(torch, md, w, steps, dev):
+    """Step time of the one-call filter on another workload (device-resident inputs, back-to-back steps)."""
+    host = synth.make_batch(w)
+    t = {n: torch.from_numpy(host[n].view(np.int16)).to(dev).view(torch.bfloat16) for n in ("q_text", "k", "v", "hidden")}
+    ki, kc = (torch.from_numpy(host["key_idx"]).to(dev), torch.from_numpy(host["key_cnt"]).to(dev)) if w.key_cnt else (None, None)
+    f = md.Filter(md.config_for(w), device=dev)
+    stream = torch.cuda.current_stream()
+    ms = _time_steps(torch, stream, lambda: f.filter(t["q_text"], t["k"], t["v"], t["hidden"], ki, kc, stream=stream), steps, 5)
+    code, _ = f.device_status()
+    plan = f.description
+    f.close()
+    if code != 0:
+        raise RuntimeError("device status %d on %s" % (code, w.name))
+    bm = bytes_model(w)
+    peak, _ = measured_peak()
+    return {"workload": w.name, "batch": w.batch, "budget": w.budget, "ms_per_step": ms,
+            "tokens_per_s": w.batch * w.n_vis / (ms / 1e3), "headline_frac_of_peak": bm["headline"] / (ms / 1e3) / 1e9 / peak,
+            "plan": plan}
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -374,6 +394,15 @@ def run_ours(args, w):
                          "peak_kind": peak_kind, "algorithmic_bytes": dom_bytes, "ms": dom_ms},
             "clocks": clocks,
         }
+        if world == 1 and not args.no_sweep:
+            # the other listed configurations, for the record (not the benchmark line's metric)
+            also = []
+            b16 = synth.WORKLOADS["c2_llava7b_b16"]
+            for item in (b16.with_(budget=192), b16.with_(budget=128), b16.with_(budget=64),
+                         synth.WORKLOADS["c3_next7b"], synth.WORKLOADS["c4_video"], synth.WORKLOADS["c5_13b_b64"]):
+                if item.name != w.name or item.budget != w.budget:
+                    also.append(quick_measure(torch, md, item, 50, dev))
+            line["other_workloads"] = also
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
@@ -569,6 +598,7 @@ def main():
     ap.add_argument("--path", default="filter", choices=["filter", "staged"],
                     help="filter: the one-call entry point; staged: score, select and compact as three calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the short runs of the other listed configurations")
     ap.add_argument("--op", default="filter", choices=["filter", "layers", "cache_compact", "upstream"],
                     help="filter: the benchmark proper; layers / cache_compact: side measurements (1 GPU)")
     ap.add_argument("--layer-budgets", default="192,128,64", help="--op layers: keep budget of each pruning layer")
