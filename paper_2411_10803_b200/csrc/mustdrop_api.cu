@@ -340,9 +340,10 @@ int32_t mustdrop_plan_describe(const mustdrop_plan_t* plan, char* buf, size_t n)
   if (plan->score_variant == mustdrop::kScoreFusedCluster) {
     const mustdrop::FusedGeometry& g = plan->fused;
     len = std::snprintf(text, sizeof(text),
-                        "fused tcgen05 score: cluster %d, %d keys per CTA, %d stages, %d tensor-memory buffers, "
+                        "fused tcgen05 score: cluster %d, %d keys per CTA, %s %d/%d, %d tensor-memory buffers, "
                         "%d statistics slots, %d clusters resident; filter = %d launch(es)",
-                        g.cluster, g.tk, g.n_stage, g.n_buf, g.n_slot, g.resident, mustdrop_plan_filter_launches(plan));
+                        g.cluster, g.tk, g.split ? "query/key-half rings" : "stages", g.n_q, g.split ? g.n_k : 0, g.n_buf, g.n_slot,
+                        g.resident, mustdrop_plan_filter_launches(plan));
   } else {
     len = std::snprintf(text, sizeof(text), "two-pass mma.sync score; filter = %d launch(es)",
                         mustdrop_plan_filter_launches(plan));

@@ -28,7 +28,8 @@ struct FusedGeometry {
   int32_t cluster;    // CTAs per request
   int32_t tk;         // keys per CTA
   int32_t cpl;        // tensor-memory columns per lane and head (= tk / halves)
-  int32_t n_stage;    // shared-memory stages
+  int32_t n_q, n_k;   // whole stages: n_q of them (n_k unused); split: rings of n_q query tiles and n_k key half-tiles
+  int32_t split;      // 1: split rings
   int32_t n_buf;      // tensor-memory buffers
   int32_t n_slot;     // statistics slots: 2 x n_buf, or 2d (d = 2 or 1) with the exp warps held within d heads of the add warps
   int32_t ach;        // chunks of 16 columns per accumulating thread (kernel variant: 5 or 10)

@@ -42,7 +42,8 @@ constexpr int kMmaWarp = kTmaWarp + 1;            // warp 13; warps 14-15 only f
 constexpr int kThreads = 16 * 32;
 constexpr int kChunk = 16;                  // TMEM columns per tcgen05.ld / st
 constexpr int kMaxCluster = 16;               // beyond 8 the cluster size is non-portable (opt-in per kernel)
-constexpr int kMaxStages = 4;
+constexpr int kMaxQBufs = 4;                  // shared-memory ring of text-query tiles (one per head)
+constexpr int kMaxKBufs = 8;                  // shared-memory ring of key half-tiles (HALVES per head)
 constexpr int kMinBufs = 3;                 // tensor-memory buffers: MMA, exp and add stages in flight ...
 constexpr int kMaxBufs = 8;                 // ... more when the columns per head allow, to hide the per-head latency chain
 constexpr int kMaxSlots = 2 * kMaxBufs;     // statistics slots = 2 x buffers: a peer's exp warps run at most that far ahead of our add warps
@@ -57,7 +58,9 @@ struct FusedParams {
   void* workspace;
   const int32_t* vis_cnt;             // [B] or null: vision tokens the request holds; its text keys follow them
   int32_t H, N, L, M, vis_start, txt_start, causal;
-  int32_t cluster, tk, cpl, n_stage;  // CTAs per request, keys per CTA, columns per TMEM lane
+  int32_t cluster, tk, cpl;           // CTAs per request, keys per CTA, columns per TMEM lane
+  int32_t n_q, n_k;                   // whole stages: n_q of them; split: ring sizes of query tiles and key half-tiles
+  int32_t split;
   int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (2 * n_buf, or 4 when tight)
   int32_t tight;                      // d = 1 or 2: the exp warps start head h only when the add warps are done with head h - d (0: no such rule)
   float scale_log2e, inv_heads;
@@ -241,8 +244,10 @@ __device__ __forceinline__ void trace_stamp(void* workspace, int n_heads, int h,
 #endif
 
 struct __align__(8) Barriers {
-  uint64_t full[kMaxStages];     // TMA -> MMA: stage filled
-  uint64_t empty[kMaxStages];    // MMA -> TMA: stage consumed
+  uint64_t qfull[kMaxQBufs];     // TMA -> MMA: query tile of a head has landed
+  uint64_t qempty[kMaxQBufs];    // MMA -> TMA: query tile consumed
+  uint64_t full[kMaxKBufs];      // TMA -> MMA: key half-tile has landed
+  uint64_t empty[kMaxKBufs];     // MMA -> TMA: key half-tile consumed
   uint64_t tfull[kMaxBufs];      // MMA -> exp warps: logits of a head are in tensor memory
   uint64_t eready[kMaxBufs];     // exp -> add warps: exponentials of a head are in tensor memory
   uint64_t tempty[kMaxBufs];     // add warps -> MMA: tensor-memory buffer free
@@ -278,16 +283,26 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const uint32_t rank = cluster_cta_rank();
   const int b = blockIdx.x / p.cluster;
   MD_PIPE(p.workspace, 0, false, true);
+  // dynamic shared memory: [n_q query tiles][n_k key half-tiles][stats: n_slot x cluster x NROWS x EPR float2]
+  // A tile is two slabs of 64 elements (128 bytes per row, 128-byte swizzle), rows contiguous per slab.
+  // Two layouts of the staging area: whole stages (a head's query tile and all its keys, n_q of
+  // them, recycled together), or - where shared memory is short - a ring of n_q query tiles and a
+  // ring of n_k key half-tiles recycled on their own (p.split).
+  constexpr uint32_t q_bytes = NROWS * 256u;
+  const uint32_t kh_bytes = static_cast<uint32_t>(p.cpl) * 256u;
   const uint32_t stage_bytes = static_cast<uint32_t>(NROWS + p.tk) * 256u;
-  // dynamic shared memory: [stages][stats: n_slot x cluster x NROWS x EPR float2]
   const uint32_t stage_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  const uint32_t k_base = stage_base + static_cast<uint32_t>(p.n_q) * q_bytes;
   unsigned char* stage_ptr = smem_dyn + (stage_base - smem_u32(smem_dyn));
-  float2* stats = reinterpret_cast<float2*>(stage_ptr + static_cast<size_t>(p.n_stage) * stage_bytes);
+  const size_t staging = p.split ? static_cast<size_t>(p.n_q) * q_bytes + static_cast<size_t>(p.n_k) * kh_bytes
+                                 : static_cast<size_t>(p.n_q) * stage_bytes;
+  float2* stats = reinterpret_cast<float2*>(stage_ptr + staging);
   const uint32_t slot_pairs = static_cast<uint32_t>(p.cluster) * NROWS * EPR;   // pairs per slot
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
-    for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&bars.full[s]), 1); mbar_init(smem_u32(&bars.empty[s]), 1); }
+    for (int s = 0; s < kMaxQBufs; ++s) { mbar_init(smem_u32(&bars.qfull[s]), 1); mbar_init(smem_u32(&bars.qempty[s]), 1); }
+    for (int s = 0; s < kMaxKBufs; ++s) { mbar_init(smem_u32(&bars.full[s]), 1); mbar_init(smem_u32(&bars.empty[s]), 1); }
     for (int s = 0; s < kMaxBufs; ++s) {
       mbar_init(smem_u32(&bars.tfull[s]), 1);
       mbar_init(smem_u32(&bars.eready[s]), kExpWarps);
@@ -348,62 +363,143 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       // ---------------- TMA producer ----------------
       const int key0 = static_cast<int>(rank) * p.tk;
       const uint64_t stream_once = l2_evict_first_policy();
-      int issued = 0;
-      for (int h = 0; h < p.H; ++h) {
-        const int s = h % p.n_stage;
-        const uint32_t ph = static_cast<uint32_t>(h / p.n_stage) & 1u;
-        if (!mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag)) break;
-        const uint32_t full = smem_u32(&bars.full[s]);
-        const uint32_t q_dst = stage_base + s * stage_bytes;
-        const uint32_t k_dst = q_dst + NROWS * 256u;
-        mbar_expect_tx(full, stage_bytes);
-        MD_TRACE(h, 0);
-#pragma unroll
-        for (int slab = 0; slab < 2; ++slab) {
-          tma_load_4d(q_dst + slab * (NROWS * 128u), &q_map, slab * 64, 0, h, b, full);
-#pragma unroll
-          for (int hv = 0; hv < HALVES; ++hv)
-            tma_load_4d_hint(k_dst + slab * (p.tk * 128u) + hv * (p.cpl * 128u), &k_map, slab * 64, key0 + hv * p.cpl,
-                             h, b, full, stream_once);
+      if (p.split) {
+        int q_issued = 0, k_issued = 0;   // tiles started so far
+        bool ok = true;
+        for (int h = 0; h < p.H && ok; ++h) {
+          const int qi = h % p.n_q;
+          if (!mbar_wait(smem_u32(&bars.qempty[qi]), (static_cast<uint32_t>(h / p.n_q) & 1u) ^ 1u, abort_flag)) break;
+          const uint32_t qfull = smem_u32(&bars.qfull[qi]);
+          const uint32_t q_dst = stage_base + qi * q_bytes;
+          mbar_expect_tx(qfull, q_bytes);
+          MD_TRACE(h, 0);
+          tma_load_4d(q_dst, &q_map, 0, 0, h, b, qfull);
+          tma_load_4d(q_dst + NROWS * 128u, &q_map, 64, 0, h, b, qfull);
+          q_issued = h + 1;
+  #pragma unroll
+          for (int hv = 0; hv < HALVES; ++hv) {
+            const int ki = k_issued % p.n_k;
+            if (!mbar_wait(smem_u32(&bars.empty[ki]), (static_cast<uint32_t>(k_issued / p.n_k) & 1u) ^ 1u, abort_flag)) {
+              ok = false;
+              break;
+            }
+            const uint32_t full = smem_u32(&bars.full[ki]);
+            const uint32_t k_dst = k_base + ki * kh_bytes;
+            mbar_expect_tx(full, kh_bytes);
+            tma_load_4d_hint(k_dst, &k_map, 0, key0 + hv * p.cpl, h, b, full, stream_once);
+            tma_load_4d_hint(k_dst + p.cpl * 128u, &k_map, 64, key0 + hv * p.cpl, h, b, full, stream_once);
+            ++k_issued;
+          }
         }
-        issued = h + 1;
-      }
-      // Leave only when every copy this thread started has landed (bounded).
-      for (int h = (issued > p.n_stage ? issued - p.n_stage : 0); h < issued; ++h) {
-        const uint32_t bar = smem_u32(&bars.full[h % p.n_stage]);
-        const uint32_t ph = static_cast<uint32_t>(h / p.n_stage) & 1u;
-        const long long t0 = clock64();
-        while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles) {}
+        // Leave only when every copy this thread started has landed (bounded).
+        for (int x = (q_issued > p.n_q ? q_issued - p.n_q : 0); x < q_issued; ++x) {
+          const uint32_t bar = smem_u32(&bars.qfull[x % p.n_q]);
+          const uint32_t ph = static_cast<uint32_t>(x / p.n_q) & 1u;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles) {}
+        }
+        for (int x = (k_issued > p.n_k ? k_issued - p.n_k : 0); x < k_issued; ++x) {
+          const uint32_t bar = smem_u32(&bars.full[x % p.n_k]);
+          const uint32_t ph = static_cast<uint32_t>(x / p.n_k) & 1u;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles) {}
+        }
+      } else {
+        int issued = 0;
+        for (int h = 0; h < p.H; ++h) {
+          const int s = h % p.n_q;
+          const uint32_t ph = static_cast<uint32_t>(h / p.n_q) & 1u;
+          if (!mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag)) break;
+          const uint32_t full = smem_u32(&bars.full[s]);
+          const uint32_t q_dst = stage_base + s * stage_bytes;
+          const uint32_t k_dst = q_dst + NROWS * 256u;
+          mbar_expect_tx(full, stage_bytes);
+          MD_TRACE(h, 0);
+  #pragma unroll
+          for (int slab = 0; slab < 2; ++slab) {
+            tma_load_4d(q_dst + slab * (NROWS * 128u), &q_map, slab * 64, 0, h, b, full);
+  #pragma unroll
+            for (int hv = 0; hv < HALVES; ++hv)
+              tma_load_4d_hint(k_dst + slab * (p.tk * 128u) + hv * (p.cpl * 128u), &k_map, slab * 64, key0 + hv * p.cpl,
+                               h, b, full, stream_once);
+          }
+          issued = h + 1;
+        }
+        // Leave only when every copy this thread started has landed (bounded).
+        for (int h = (issued > p.n_q ? issued - p.n_q : 0); h < issued; ++h) {
+          const uint32_t bar = smem_u32(&bars.full[h % p.n_q]);
+          const uint32_t ph = static_cast<uint32_t>(h / p.n_q) & 1u;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles) {}
+        }
       }
     } else if (warp == kMmaWarp && lane == 0) {
       // ---------------- MMA issuer ----------------
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(p.cpl >> 3) << 17) |
                              (static_cast<uint32_t>(NROWS >> 4) << 24);
-      for (int h = 0; h < p.H; ++h) {
-        const int s = h % p.n_stage, buf = h % p.n_buf;
-        const uint32_t ph = static_cast<uint32_t>(h / p.n_stage) & 1u;
-        const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
-        if (!mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag)) break;
-        MD_TRACE(h, 1);
-        if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag)) break;
-        MD_TRACE(h, 2);
-        tc_fence_after();
-        const uint32_t q_src = stage_base + s * stage_bytes;
-        const uint32_t k_src = q_src + NROWS * 256u;
-#pragma unroll
-        for (int hv = 0; hv < HALVES; ++hv) {
-          // the second M=64 tile goes to the upper 16 lanes of every TMEM quadrant
-          const uint32_t d = tmem_base + static_cast<uint32_t>(buf * p.cpl) + (hv ? (16u << 16) : 0u);
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t slab = ks >> 2, koff = (ks & 3) * 32u;
-            const uint64_t ad = smem_desc(q_src + slab * (NROWS * 128u) + koff);
-            const uint64_t bd = smem_desc(k_src + slab * (p.tk * 128u) + hv * (p.cpl * 128u) + koff);
-            tc_mma(d, ad, bd, idesc, ks > 0 ? 1u : 0u);
+      if (p.split) {
+        int k_used = 0;
+        bool ok = true;
+        for (int h = 0; h < p.H && ok; ++h) {
+          const int qi = h % p.n_q, buf = h % p.n_buf;
+          const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
+          if (!mbar_wait(smem_u32(&bars.qfull[qi]), static_cast<uint32_t>(h / p.n_q) & 1u, abort_flag)) break;
+          MD_TRACE(h, 1);
+          if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag)) break;
+          MD_TRACE(h, 2);
+          const uint32_t q_src = stage_base + qi * q_bytes;
+  #pragma unroll
+          for (int hv = 0; hv < HALVES; ++hv) {
+            const int ki = k_used % p.n_k;
+            if (!mbar_wait(smem_u32(&bars.full[ki]), static_cast<uint32_t>(k_used / p.n_k) & 1u, abort_flag)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t k_src = k_base + ki * kh_bytes;
+            // the second M=64 tile goes to the upper 16 lanes of every TMEM quadrant
+            const uint32_t d = tmem_base + static_cast<uint32_t>(buf * p.cpl) + (hv ? (16u << 16) : 0u);
+  #pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint32_t slab = ks >> 2, koff = (ks & 3) * 32u;
+              const uint64_t ad = smem_desc(q_src + slab * (NROWS * 128u) + koff);
+              const uint64_t bd = smem_desc(k_src + slab * (p.cpl * 128u) + koff);
+              tc_mma(d, ad, bd, idesc, ks > 0 ? 1u : 0u);
+            }
+            tc_commit(smem_u32(&bars.empty[ki]));   // this half-tile may be refilled once its MMAs are done
+            ++k_used;
           }
+          if (!ok) break;
+          tc_commit(smem_u32(&bars.qempty[qi]));
+          tc_commit(smem_u32(&bars.tfull[buf]));
         }
-        tc_commit(smem_u32(&bars.empty[s]));
-        tc_commit(smem_u32(&bars.tfull[buf]));
+      } else {
+        for (int h = 0; h < p.H; ++h) {
+          const int s = h % p.n_q, buf = h % p.n_buf;
+          const uint32_t ph = static_cast<uint32_t>(h / p.n_q) & 1u;
+          const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
+          if (!mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag)) break;
+          MD_TRACE(h, 1);
+          if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag)) break;
+          MD_TRACE(h, 2);
+          tc_fence_after();
+          const uint32_t q_src = stage_base + s * stage_bytes;
+          const uint32_t k_src = q_src + NROWS * 256u;
+  #pragma unroll
+          for (int hv = 0; hv < HALVES; ++hv) {
+            // the second M=64 tile goes to the upper 16 lanes of every TMEM quadrant
+            const uint32_t d = tmem_base + static_cast<uint32_t>(buf * p.cpl) + (hv ? (16u << 16) : 0u);
+  #pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint32_t slab = ks >> 2, koff = (ks & 3) * 32u;
+              const uint64_t ad = smem_desc(q_src + slab * (NROWS * 128u) + koff);
+              const uint64_t bd = smem_desc(k_src + slab * (p.tk * 128u) + hv * (p.cpl * 128u) + koff);
+              tc_mma(d, ad, bd, idesc, ks > 0 ? 1u : 0u);
+            }
+          }
+          tc_commit(smem_u32(&bars.empty[s]));
+          tc_commit(smem_u32(&bars.tfull[buf]));
+        }
       }
     }
     if constexpr (FILTER) {
@@ -840,38 +936,51 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     const size_t stage = static_cast<size_t>(nrows + tk) * 256;
     const int ach = cpl <= 5 * kChunk ? 5 : 10;             // chunks per add thread (kernel variant)
     const int epr = kColGroups;                             // (max, sum) pairs per row and CTA
-    // As many tensor-memory buffers as the columns allow (3..8), fewer if their statistics
-    // slots (2 x buffers x cluster x rows x pairs x 8 bytes) would leave no room for 2 stages;
-    // if even three buffers' slots do not fit (large clusters), four slots with the exp warps
-    // held within two heads of the add warps.
+    // Shared memory.  Whole stages first (a head's query tile and keys recycled together): as many
+    // tensor-memory buffers as the columns allow (3..8), fewer if their statistics slots (2 x
+    // buffers x cluster x rows x pairs x 8 bytes) would leave no room for 2 stages; four stages
+    // are preferred over more buffers.  If even three buffers' slots do not fit (large clusters):
+    // 2d slots with the exp warps held within d heads of the add warps (d = 2, else 1) - and for
+    // those the split layout (two query tiles + a ring of key half-tiles, which needs less
+    // memory for the same look-ahead) is tried as well and taken when it allows a wider window.
+    const size_t q_tile = static_cast<size_t>(nrows) * 256, k_half = static_cast<size_t>(cpl) * 256;
+    const size_t avail = 227 * 1024 - 4096 /* static */ - 1024 /* alignment */;
+    auto slots_bytes = [&](int n_slot) { return static_cast<size_t>(n_slot) * c * nrows * epr * 8; };
     int n_buf = kTmemCols / cpl;
     if (n_buf > kMaxBufs) n_buf = kMaxBufs;
     if (n_buf < kMinBufs) continue;
     const int max_buf = n_buf;
     size_t extra = 0;
-    int n_stage = 0, n_slot = 0;
-    for (; n_buf >= kMinBufs; --n_buf) {
+    int n_q = 0, n_k = 0, n_slot = 0, split = 0;
+    for (; n_buf >= kMinBufs; --n_buf) {          // whole stages, full set of slots
       n_slot = 2 * n_buf;
-      extra = static_cast<size_t>(n_slot) * c * nrows * epr * 8;
-      const size_t reserved = 4096 /* static */ + 1024 /* alignment */ + extra;
-      if (reserved + 2 * stage > 227 * 1024) continue;
-      n_stage = static_cast<int>((227 * 1024 - reserved) / stage);
-      // a stage is held for a load latency plus an MMA (~2.3 us): prefer four stages over more buffers
-      if (n_stage >= kMaxStages || n_buf == kMinBufs) break;
+      extra = slots_bytes(n_slot);
+      if (extra + 2 * stage > avail) continue;
+      n_q = static_cast<int>((avail - extra) / stage);
+      if (n_q >= 4 || n_buf == kMinBufs) break;
     }
-    for (int d = 2; d >= 1 && n_stage < 2; --d) {   // tight: 2d slots, exp warps within d heads of the add warps
+    if (n_q < 2) {                                 // tight windows
       n_buf = max_buf;
-      n_slot = 2 * d;
-      extra = static_cast<size_t>(n_slot) * c * nrows * epr * 8;
-      const size_t reserved = 4096 + 1024 + extra;
-      n_stage = reserved + 2 * stage > 227 * 1024 ? 0 : static_cast<int>((227 * 1024 - reserved) / stage);
+      int best_d = 0;
+      for (int d = 2; d >= 1 && best_d == 0; --d) {
+        const size_t e = slots_bytes(2 * d);
+        if (e + 2 * stage <= avail) {              // whole stages
+          best_d = d; split = 0; extra = e; n_slot = 2 * d;
+          n_q = static_cast<int>((avail - e) / stage);
+        } else if (e + 2 * q_tile + (halves + 1) * k_half <= avail) {   // split rings
+          best_d = d; split = 1; extra = e; n_slot = 2 * d;
+          n_q = 2;
+          n_k = static_cast<int>((avail - e - 2 * q_tile) / k_half);
+          if (n_k > 4 * halves) n_k = 4 * halves;
+        }
+      }
+      if (best_d == 0) continue;
     }
-    if (n_stage < 2) continue;
-    if (n_stage > kMaxStages) n_stage = kMaxStages;
+    if (n_q > 4) n_q = 4;
     // Cost model (microseconds per head and CTA): streaming the stage at ~45 GB/s per SM, or the
     // MMA -> exp -> exchange -> add chain (~4.5 us) spread over the buffers, whichever is longer;
     // times the number of waves of CTAs.
-    size_t smem_bytes = stage * n_stage + 1024 + extra;
+    size_t smem_bytes = (split ? n_q * q_tile + n_k * k_half : n_q * stage) + 1024 + extra;
     // at least 116 KB, so that two CTAs (each wanting all of tensor memory) never share an SM
     if (smem_bytes < 116 * 1024) smem_bytes = 116 * 1024;
     int resident = max_resident_clusters(halves, ach, c, smem_bytes);
@@ -891,7 +1000,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     const double score = 1.0 / (static_cast<double>(waves) * t_head) - 1e-4 * c;   // prefer smaller clusters among equals
     if (score > best) {
       best = score;
-      g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_stage = n_stage; g.n_buf = n_buf; g.ach = ach;
+      g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_q = n_q; g.n_k = n_k; g.split = split; g.n_buf = n_buf; g.ach = ach;
       g.n_slot = n_slot; g.resident = resident;
       g.est_us = static_cast<float>(waves * r.H * t_head);
       g.smem_bytes = smem_bytes;
@@ -922,7 +1031,7 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, c
   p.vis_cnt = vis_cnt;
   p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
   p.causal = r.causal;
-  p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_stage = geo.n_stage;
+  p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_q = geo.n_q; p.n_k = geo.n_k; p.split = geo.split;
   p.n_buf = geo.n_buf; p.n_slot = geo.n_slot; p.tight = geo.n_slot < 2 * geo.n_buf ? geo.n_slot / 2 : 0;
   p.scale_log2e = r.scale_log2e;
   p.inv_heads = 1.0f / static_cast<float>(r.H);
