@@ -114,7 +114,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   (void)cudaGetLastError();
 
   // Score kernel: the fused single-pass kernel where its geometry covers the shape, else the
-  // two-pass kernel.  MUSTDROP_SCORE_VARIANT (two_pass | fused) and MUSTDROP_CLUSTER (1..16) are
+  // two-pass kernel.  MUSTDROP_SCORE_VARIANT (two_pass | fused | row_split) and MUSTDROP_CLUSTER (1..16) are
   // debugging overrides read here, once per plan.
   p->score_variant = kScoreTwoPassMma;
   {
@@ -122,23 +122,47 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
     const char* cl = std::getenv("MUSTDROP_CLUSTER");
     const int forced_cluster = cl ? std::atoi(cl) : 0;
     const bool allow_fused = !(want && std::strcmp(want, "two_pass") == 0) && !r.per_head_max;
-    if (allow_fused && plan_score_fused(r, p->sm_count, forced_cluster, &p->fused)) {
+    const bool force_split = want && std::strcmp(want, "row_split") == 0;
+    const double k_mb = 256.0e-6 * r.B * r.H * r.L;
+    const double two_pass_us = k_mb * (0.6 + 0.7 * r.N / 128.0);   // the two-pass kernel's measured rate
+    double chosen_us = two_pass_us;
+    p->row_split = 0;
+    if (allow_fused && !force_split && plan_score_fused(r, p->sm_count, forced_cluster, &p->fused)) {
       p->score_variant = kScoreFusedCluster;
+      chosen_us = p->fused.est_us;
       // A fused plan that had to fall back to few statistics slots (sequences needing clusters of
-      // more than 8 CTAs) can be slower than reading K twice: compare with the two-pass kernel's
-      // measured rate (about 0.6 + 0.7 * N / 128 us per MB of keys) unless the variant is forced.
+      // more than 8 CTAs) can be slower than reading K twice: compare with the two-pass kernel
+      // unless the variant is forced.
       const bool tight = p->fused.n_slot < 2 * p->fused.n_buf;
-      const double k_mb = 256.0e-6 * r.B * r.H * r.L;
-      const double two_pass_us = k_mb * (0.6 + 0.7 * r.N / 128.0);
-      if (tight && want == nullptr && forced_cluster == 0 && p->fused.est_us > two_pass_us)
+      if (tight && want == nullptr && forced_cluster == 0 && p->fused.est_us > two_pass_us) {
         p->score_variant = kScoreTwoPassMma;
+        chosen_us = two_pass_us;
+      }
+    }
+    // More than 64 text rows fill all 128 tensor-memory lanes with one key range, which halves the
+    // keys a CTA can take.  Alternative: two launches over the same keys, text rows 0..63 and the
+    // rest, each with the two-tile layout (twice the keys per CTA); the second adds its column
+    // sums to / takes the maximum with the first's.  Taken when estimated faster than the above.
+    if (allow_fused && r.N > 64) {
+      mustdrop::FusedGeometry ga, gb;
+      if (plan_score_fused(r, p->sm_count, forced_cluster, &ga, 0, 64) &&
+          plan_score_fused(r, p->sm_count, forced_cluster, &gb, 64, r.N - 64)) {
+        const bool together = r.B * (ga.cluster + gb.cluster) <= p->sm_count;   // both launches resident at once
+        const double split_us = together ? 1.15 * (ga.est_us > gb.est_us ? ga.est_us : gb.est_us) : ga.est_us + gb.est_us;
+        if (force_split || (want == nullptr && forced_cluster == 0 && split_us < chosen_us)) {
+          p->score_variant = kScoreFusedCluster;
+          p->row_split = 1;
+          p->fused = ga;
+          p->fused_b = gb;
+        }
+      }
     }
     // mustdrop_filter: one launch where the fused kernel covers the shape and a kept row fits its
     // shared-memory ring; MUSTDROP_FILTER=staged forces the three launches (debugging override).
     const char* fw = std::getenv("MUSTDROP_FILTER");
     p->filter_single = 0;
     if (p->score_variant == kScoreFusedCluster && !(fw && std::strcmp(fw, "staged") == 0) &&
-        plan_filter_single(r, p->fused, &p->filter))
+        plan_filter_single(r, p->row_split ? p->fused_b : p->fused, &p->filter))
       p->filter_single = 1;
   }
   size_t off = kWsStatusBytes;
@@ -287,8 +311,8 @@ mustdrop_status_t mustdrop_filter_layer(const mustdrop_plan_t* plan, const mustd
 
 int32_t mustdrop_plan_filter_launches(const mustdrop_plan_t* plan) {
   if (!valid_plan(plan)) return -1;
-  if (plan->filter_single) return 1;
-  return plan->score_variant == mustdrop::kScoreTwoPassMma ? 4 : 3;
+  if (plan->filter_single) return plan->row_split ? 2 : 1;
+  return plan->score_variant == mustdrop::kScoreTwoPassMma ? 4 : (plan->row_split ? 4 : 3);
 }
 
 mustdrop_status_t mustdrop_device_status(const mustdrop_plan_t* plan, const void* workspace, void* cuda_stream,
@@ -338,11 +362,11 @@ int32_t mustdrop_plan_describe(const mustdrop_plan_t* plan, char* buf, size_t n)
   char text[256];
   int len;
   if (plan->score_variant == mustdrop::kScoreFusedCluster) {
-    const mustdrop::FusedGeometry& g = plan->fused;
+    const mustdrop::FusedGeometry& g = plan->row_split ? plan->fused_b : plan->fused;
     len = std::snprintf(text, sizeof(text),
-                        "fused tcgen05 score: cluster %d, %d keys per CTA, %s %d/%d, %d tensor-memory buffers, "
+                        "fused tcgen05 score%s: cluster %d, %d keys per CTA, %s %d/%d, %d tensor-memory buffers, "
                         "%d statistics slots, %d clusters resident; filter = %d launch(es)",
-                        g.cluster, g.tk, g.split ? "query/key-half rings" : "stages", g.n_q, g.split ? g.n_k : 0, g.n_buf, g.n_slot,
+                        plan->row_split ? " (text rows in two launches; second launch)" : "", g.cluster, g.tk, g.split ? "query/key-half rings" : "stages", g.n_q, g.split ? g.n_k : 0, g.n_buf, g.n_slot,
                         g.resident, mustdrop_plan_filter_launches(plan));
   } else {
     len = std::snprintf(text, sizeof(text), "two-pass mma.sync score; filter = %d launch(es)",

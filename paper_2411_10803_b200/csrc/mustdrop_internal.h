@@ -33,6 +33,7 @@ struct FusedGeometry {
   int32_t n_buf;      // tensor-memory buffers
   int32_t n_slot;     // statistics slots: 2 x n_buf, or 2d (d = 2 or 1) with the exp warps held within d heads of the add warps
   int32_t ach;        // chunks of 16 columns per accumulating thread (kernel variant: 5 or 10)
+  int32_t row0, n_rows;   // the text rows this geometry's launch covers
   int32_t resident;   // clusters the device can hold at once (0: not asked)
   float est_us;       // the planner's estimate of the score time
   size_t smem_bytes;  // dynamic shared memory
@@ -80,6 +81,8 @@ struct mustdrop_plan {
   size_t ws_bytes;
   size_t ws_rowstats_off;   // float2 [B,H,N]: (row max in log2 units, 1 / row sum)
   mustdrop::FusedGeometry fused;
+  int32_t row_split;        // 1: the text rows are scored by two launches (fused: rows 0..63, fused_b: the rest)
+  mustdrop::FusedGeometry fused_b;
   int32_t filter_single;    // 1: mustdrop_filter is one launch of the fused kernel with its tail
   mustdrop::FilterGeometry filter;
 };
@@ -92,7 +95,8 @@ constexpr uint32_t kPlanMagic = 0x4d445250u;  // "MDRP"
 cudaError_t launch_score_two_pass(const mustdrop_plan& p, const void* q_text, const void* k,
                                   float* g_out, float* i_out, void* rowstats, cudaStream_t stream,
                                   const int32_t* vis_cnt = nullptr);
-bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out);
+bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out, int row0 = 0,
+                      int n_rows = 0);
 cudaError_t launch_score_fused(const mustdrop_plan& p, const void* q_text, const void* k, float* g_out,
                                float* i_out, void* workspace, cudaStream_t stream, const int32_t* vis_cnt = nullptr);
 bool plan_filter_single(const Resolved& r, const FusedGeometry& geo, FilterGeometry* out);

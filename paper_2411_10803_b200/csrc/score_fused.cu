@@ -58,6 +58,8 @@ struct FusedParams {
   void* workspace;
   const int32_t* vis_cnt;             // [B] or null: vision tokens the request holds; its text keys follow them
   int32_t H, N, L, M, vis_start, txt_start, causal;
+  int32_t n_txt;                      // all text rows of the request (N is this launch's share)
+  int32_t row0, combine;              // this launch covers text rows row0 .. row0 + N - 1; combine: add to / max with what g_out / i_out hold
   int32_t cluster, tk, cpl;           // CTAs per request, keys per CTA, columns per TMEM lane
   int32_t n_q, n_k;                   // whole stages: n_q of them; split: ring sizes of query tiles and key half-tiles
   int32_t split;
@@ -335,7 +337,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     pdl_wait();
     Mb = clamp_vis_cnt(p.vis_cnt[b], p.M);
     txt_start = p.vis_start + Mb;
-    Lb = txt_start + p.N;
+    Lb = txt_start + p.n_txt;
   }
 
   // End of the score part, executed by every thread: tensor memory freed, and no CTA goes on
@@ -519,7 +521,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const int total_chunks = p.cpl / kChunk;
     const int my_chunks = (total_chunks - g + kColGroups - 1) / kColGroups;   // chunks g, g+2, ... (uniform per warp)
     const int key_lane0 = static_cast<int>(rank) * p.tk + half * p.cpl;        // key of this lane's column 0
-    int lim = p.causal ? (txt_start + row + 1) : Lb;                           // keys below lim are visible
+    int lim = p.causal ? (txt_start + p.row0 + row + 1) : Lb;                  // keys below lim are visible
     lim = (lim < Lb ? lim : Lb) - key_lane0;                                   // ... as a column count of this lane
     const bool all_visible = lim >= p.cpl;
     const bool sender = (half == 0);           // with two halves, lanes s and s+16 share a row: the lower one sends
@@ -735,8 +737,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           mx = fmaxf(mx, v);
         }
         const bool present = j < Mb;    // beyond the request's own tokens: zeros
-        p.g_out[static_cast<size_t>(b) * p.M + j] = present ? s * p.inv_heads : 0.0f;
-        p.i_out[static_cast<size_t>(b) * p.M + j] = present ? mx * p.inv_heads : 0.0f;
+        float gv = present ? s * p.inv_heads : 0.0f, iv = present ? mx * p.inv_heads : 0.0f;
+        if (p.combine) {                // the text rows before row0 were scored by the launch before this one
+          gv += p.g_out[static_cast<size_t>(b) * p.M + j];
+          iv = fmaxf(iv, p.i_out[static_cast<size_t>(b) * p.M + j]);
+        }
+        p.g_out[static_cast<size_t>(b) * p.M + j] = gv;
+        p.i_out[static_cast<size_t>(b) * p.M + j] = iv;
       }
     }
     if constexpr (FILTER) {
@@ -920,8 +927,10 @@ int max_resident_clusters(int halves, int ach, int cluster, size_t smem_bytes) {
 }  // namespace
 
 // Geometry of the fused kernel for a problem; false when the shape is outside what it covers.
-bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out) {
-  const int halves = r.N <= 64 ? 2 : 1;
+// row0 / n_rows: the text rows the launch covers (n_rows = 0: all of them).
+bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out, int row0, int n_rows) {
+  if (n_rows <= 0) { row0 = 0; n_rows = r.N; }
+  const int halves = n_rows <= 64 ? 2 : 1;
   const int nrows = 128 / halves;
   const int max_cpl = 10 * kChunk;   // 160 columns per TMEM lane (add threads with 10 chunks)
   double best = -1.0;
@@ -1001,7 +1010,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     if (score > best) {
       best = score;
       g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_q = n_q; g.n_k = n_k; g.split = split; g.n_buf = n_buf; g.ach = ach;
-      g.n_slot = n_slot; g.resident = resident;
+      g.n_slot = n_slot; g.resident = resident; g.row0 = row0; g.n_rows = n_rows;
       g.est_us = static_cast<float>(waves * r.H * t_head);
       g.smem_bytes = smem_bytes;
     }
@@ -1014,14 +1023,16 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
 namespace {
 
 // Common launch of the score kernel, with (tail != nullptr) or without the selection / gather tail.
-cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, const void* k, float* g_out,
-                                float* i_out, void* workspace, const GatherMaps* maps, const FilterTail* tail,
-                                size_t smem_bytes, cudaStream_t stream, const int32_t* vis_cnt) {
+cudaError_t launch_fused_common(const mustdrop_plan& plan, const FusedGeometry& geo, bool combine, const void* q_text,
+                                const void* k, float* g_out, float* i_out, void* workspace, const GatherMaps* maps,
+                                const FilterTail* tail, size_t smem_bytes, cudaStream_t stream,
+                                const int32_t* vis_cnt) {
   const Resolved& r = plan.r;
-  const FusedGeometry& geo = plan.fused;
   const int nrows = 128 / geo.halves;
   CUtensorMap q_map, k_map;
-  if (!make_map(&q_map, q_text, r.N, r.H, r.B, 256, static_cast<uint64_t>(r.N) * 256,
+  // the launch's text rows: a window of geo.n_rows rows starting at geo.row0 of every head's N rows
+  const unsigned char* q_rows = static_cast<const unsigned char*>(q_text) + static_cast<size_t>(geo.row0) * 256;
+  if (!make_map(&q_map, q_rows, geo.n_rows, r.H, r.B, 256, static_cast<uint64_t>(r.N) * 256,
                 static_cast<uint64_t>(r.H) * r.N * 256, nrows) ||
       !make_map(&k_map, k, r.L, r.H, r.B, static_cast<uint64_t>(r.k_sl) * 2, static_cast<uint64_t>(r.k_sh) * 2,
                 static_cast<uint64_t>(r.k_sb) * 2, geo.cpl))
@@ -1029,8 +1040,9 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, c
   FusedParams p;
   p.g_out = g_out; p.i_out = i_out; p.workspace = workspace;
   p.vis_cnt = vis_cnt;
-  p.H = r.H; p.N = r.N; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
+  p.H = r.H; p.N = geo.n_rows; p.L = r.L; p.M = r.M; p.vis_start = r.vis_start; p.txt_start = r.txt_start;
   p.causal = r.causal;
+  p.n_txt = r.N; p.row0 = geo.row0; p.combine = combine ? 1 : 0;
   p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_q = geo.n_q; p.n_k = geo.n_k; p.split = geo.split;
   p.n_buf = geo.n_buf; p.n_slot = geo.n_slot; p.tight = geo.n_slot < 2 * geo.n_buf ? geo.n_slot / 2 : 0;
   p.scale_log2e = r.scale_log2e;
@@ -1067,8 +1079,12 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const void* q_text, c
 
 cudaError_t launch_score_fused(const mustdrop_plan& plan, const void* q_text, const void* k, float* g_out,
                                float* i_out, void* workspace, cudaStream_t stream, const int32_t* vis_cnt) {
-  return launch_fused_common(plan, q_text, k, g_out, i_out, workspace, nullptr, nullptr, plan.fused.smem_bytes, stream,
-                             vis_cnt);
+  cudaError_t e = launch_fused_common(plan, plan.fused, false, q_text, k, g_out, i_out, workspace, nullptr, nullptr,
+                                      plan.fused.smem_bytes, stream, vis_cnt);
+  if (e != cudaSuccess || !plan.row_split) return e;
+  // the remaining text rows: same keys again, results combined with the first launch's
+  return launch_fused_common(plan, plan.fused_b, true, q_text, k, g_out, i_out, workspace, nullptr, nullptr,
+                             plan.fused_b.smem_bytes, stream, vis_cnt);
 }
 
 // Shared-memory plan of the gather tail; false when a row does not fit the ring at least three times.
@@ -1127,8 +1143,15 @@ cudaError_t launch_filter_fused(const mustdrop_plan& plan, const void* q_text, c
   t.has_k = k_out != nullptr; t.has_v = v_out != nullptr;
   t.slot_bytes = plan.filter.slot_bytes; t.n_slot = plan.filter.n_slot;
   t.vis_start = r.vis_start;
-  return launch_fused_common(plan, q_text, k, g_out, i_out, workspace, &maps, &t, plan.filter.smem_bytes, stream,
-                             la.vis_cnt);
+  if (plan.row_split) {   // first the score of text rows 0..63 alone, then the rest with the tail
+    cudaError_t e = launch_fused_common(plan, plan.fused, false, q_text, k, g_out, i_out, workspace, nullptr, nullptr,
+                                        plan.fused.smem_bytes, stream, la.vis_cnt);
+    if (e != cudaSuccess) return e;
+    return launch_fused_common(plan, plan.fused_b, true, q_text, k, g_out, i_out, workspace, &maps, &t,
+                               plan.filter.smem_bytes, stream, la.vis_cnt);
+  }
+  return launch_fused_common(plan, plan.fused, false, q_text, k, g_out, i_out, workspace, &maps, &t,
+                             plan.filter.smem_bytes, stream, la.vis_cnt);
 }
 
 }  // namespace mustdrop

@@ -178,3 +178,42 @@ def test_filter_is_deterministic_and_repeatable_on_one_stream():
     for a, b in zip(first, now):
         assert torch.equal(a, b)
     f.close()
+
+
+# ---- more than 64 text rows scored by two launches over the same keys ---------------------------
+
+@pytest.mark.parametrize("n_txt,causal", [(65, 1), (96, 1), (128, 1), (100, 0)])
+def test_row_split_score_and_filter_match_oracle(n_txt, causal, monkeypatch):
+    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "row_split")
+    w = small(batch=3, n_vis=500, n_txt=n_txt, n_heads=3, hidden=384, key_cnt=7, budget=60, vis_start=1)
+    d = synth.make_batch(w)
+    f = md.Filter(md.config_for(w, causal=causal))
+    assert "two launches" in f.description and f.filter_launches == 2
+    q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
+    ki, kc = key_args(w, d)
+    # the score call alone (two launches, the second combining), then the whole step
+    f.score(q, k)
+    torch.cuda.synchronize()
+    G, I = oracle.score(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start, causal=bool(causal))
+    from parity_util import assert_scores_close
+    assert_scores_close(f.g.cpu().numpy(), G, "G")
+    assert_scores_close(f.i.cpu().numpy(), I, "I")
+    f.g.zero_(); f.i.zero_()
+    f.filter(q, k, v, hid, ki, kc, want_s=True)
+    torch.cuda.synchronize()
+    assert f.device_status() == (0, 0)
+    assert_scores_close(f.g.cpu().numpy(), G, "G")
+    assert_scores_close(f.i.cpu().numpy(), I, "I")
+    ref_idx, ref_cnt, ref_s, _ = oracle.select(G, I, w.seq_len, d["key_idx"], d["key_cnt"], budget=w.budget)
+    idx, cnt = f.kept_idx.cpu().numpy(), f.kept_cnt.cpu().numpy()
+    assert_kept_matches(idx, cnt, ref_idx, ref_cnt, ref_s, d["key_idx"], d["key_cnt"])
+    zh, zk, zv = (np.zeros_like(bf16_bits(t)) for t in (f.hidden_out, f.k_out, f.v_out))
+    eh, ek, ev = host_gather(idx, cnt, w.vis_start, d["hidden"], d["k"], d["v"], zh, zk, zv)
+    assert np.array_equal(bf16_bits(f.hidden_out), eh) and np.array_equal(bf16_bits(f.k_out), ek)
+    assert np.array_equal(bf16_bits(f.v_out), ev)
+    f.close()
+
+
+def test_video_workload_takes_the_row_split_plan_by_itself():
+    w = synth.WORKLOADS["c4_video"]
+    run_chain_and_check(w, sample=[3], path="filter", expect_launches=2)

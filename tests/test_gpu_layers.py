@@ -265,3 +265,11 @@ def test_cache_compact_reports_a_token_the_layer_does_not_hold_and_takes_one_ten
             for r, o in enumerate(s_few[b, :s_few_cnt[b]].tolist()):
                 if o in ids:
                     assert np.array_equal(out[y, b][:, vs + r], kc[y, b][:, vs + ids.index(o)])
+
+
+def test_ragged_layer_with_text_rows_in_two_launches(monkeypatch):
+    for n in ("MUSTDROP_CLUSTER", "MUSTDROP_FILTER"):
+        monkeypatch.delenv(n, raising=False)
+    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "row_split")
+    w = small(batch=3, n_vis=260, n_txt=90, n_heads=2, hidden=256, key_cnt=4, budget=40, vis_start=2)
+    assert run_ragged_layer(w, np.array([260, 40, 133], np.int32), True) == 2
