@@ -143,3 +143,19 @@ def test_upstream_calls_reject_bad_sizes_without_a_gpu():
     assert md.mustdrop_key_set(1, 16, 64, 5000, 64, 256, 256, None, None, 256, 256, stream=0) == md.MUSTDROP_ERR_UNSUPPORTED
     assert md.mustdrop_key_set(1, 16, 64, 576, 0, 256, 256, None, None, 256, 256, stream=0) == md.MUSTDROP_ERR_INVALID_ARG
     assert md.mustdrop_key_set(1, 16, 64, 576, 64, 256, 264, None, None, 256, 256, stream=0) == md.MUSTDROP_ERR_INVALID_ARG
+
+
+def test_plan_description_names_the_geometry_without_a_gpu():
+    # no device: the planner assumes 148 SMs and clusters of at most 8 CTAs
+    st, plan, _ = md.mustdrop_filter_plan(md.config_for(synth.WORKLOADS["c2_llava7b_b64"]))
+    assert st == md.MUSTDROP_OK
+    text = md.mustdrop_plan_describe(plan)
+    assert "cluster 2" in text and "320 keys per CTA" in text and "filter = 1 launch" in text
+    assert md.mustdrop_plan_filter_launches(plan) == 1
+    md.mustdrop_plan_destroy(plan)
+    st, plan, _ = md.mustdrop_filter_plan(md.config_for(synth.WORKLOADS["c2_llava7b_b64"],
+                                                        flags=md.MUSTDROP_FLAG_PER_HEAD_MAX))
+    assert st == md.MUSTDROP_OK and md.mustdrop_plan_score_variant(plan) == "two_pass_mma"
+    assert md.mustdrop_plan_filter_launches(plan) == 4
+    md.mustdrop_plan_destroy(plan)
+    assert md.mustdrop_plan_describe(0) == "" or md.mustdrop_plan_filter_launches(0) == -1
