@@ -131,7 +131,8 @@ mustdrop_status_t mustdrop_score(const mustdrop_plan_t *plan, const void *q_text
 
 /*
  * mustdrop_score for callers that cannot allocate device memory.  (The paper has no
- * counterpart: this is a packaging variant of the call above, with identical results.)
+ * counterpart: this is a packaging variant of the call above.  It always runs the two-pass
+ * kernel, so its results equal mustdrop_score's up to the rounding order of fp32 sums.)
  *
  * Who needs it: code running where cudaMalloc is not an option - inside an engine whose pool
  * allocator owns the whole device heap, in a plug-in that must leave the host application's
