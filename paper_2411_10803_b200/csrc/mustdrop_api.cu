@@ -145,8 +145,14 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
     // sums to / takes the maximum with the first's.  Taken when estimated faster than the above.
     if (allow_fused && r.N > 64) {
       mustdrop::FusedGeometry ga, gb;
-      if (plan_score_fused(r, p->sm_count, forced_cluster, &ga, 0, 64) &&
-          plan_score_fused(r, p->sm_count, forced_cluster, &gb, 64, r.N - 64)) {
+      // clusters small enough for both launches to be resident at once, if such a plan exists
+      const int fit = p->sm_count / (2 * r.B);
+      bool ok = fit >= 1 && plan_score_fused(r, p->sm_count, forced_cluster, &ga, 0, 64, fit) &&
+                plan_score_fused(r, p->sm_count, forced_cluster, &gb, 64, r.N - 64, fit);
+      if (!ok)
+        ok = plan_score_fused(r, p->sm_count, forced_cluster, &ga, 0, 64) &&
+             plan_score_fused(r, p->sm_count, forced_cluster, &gb, 64, r.N - 64);
+      if (ok) {
         const bool together = r.B * (ga.cluster + gb.cluster) <= p->sm_count;   // both launches resident at once
         const double split_us = together ? 1.15 * (ga.est_us > gb.est_us ? ga.est_us : gb.est_us) : ga.est_us + gb.est_us;
         if (force_split || (want == nullptr && forced_cluster == 0 && split_us < chosen_us)) {

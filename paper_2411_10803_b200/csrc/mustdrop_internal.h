@@ -96,7 +96,7 @@ cudaError_t launch_score_two_pass(const mustdrop_plan& p, const void* q_text, co
                                   float* g_out, float* i_out, void* rowstats, cudaStream_t stream,
                                   const int32_t* vis_cnt = nullptr);
 bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out, int row0 = 0,
-                      int n_rows = 0);
+                      int n_rows = 0, int max_cluster = 0);
 cudaError_t launch_score_fused(const mustdrop_plan& p, const void* q_text, const void* k, float* g_out,
                                float* i_out, void* workspace, cudaStream_t stream, const int32_t* vis_cnt = nullptr);
 bool plan_filter_single(const Resolved& r, const FusedGeometry& geo, FilterGeometry* out);

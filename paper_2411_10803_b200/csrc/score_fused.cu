@@ -927,8 +927,10 @@ int max_resident_clusters(int halves, int ach, int cluster, size_t smem_bytes) {
 }  // namespace
 
 // Geometry of the fused kernel for a problem; false when the shape is outside what it covers.
-// row0 / n_rows: the text rows the launch covers (n_rows = 0: all of them).
-bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out, int row0, int n_rows) {
+// row0 / n_rows: the text rows the launch covers (n_rows = 0: all of them); max_cluster: an upper
+// limit on the cluster size (0: none).
+bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out, int row0, int n_rows,
+                      int max_cluster) {
   if (n_rows <= 0) { row0 = 0; n_rows = r.N; }
   const int halves = n_rows <= 64 ? 2 : 1;
   const int nrows = 128 / halves;
@@ -937,6 +939,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
   FusedGeometry g{};
   for (int c = 1; c <= kMaxCluster; ++c) {
     if (forced_cluster > 0 && c != forced_cluster) continue;
+    if (max_cluster > 0 && c > max_cluster) continue;
     const int per_cta = (r.L + c - 1) / c;
     int cpl = (per_cta + halves - 1) / halves;
     cpl = (cpl + kChunk - 1) / kChunk * kChunk;
