@@ -1001,7 +1001,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     if (resident <= 0) continue;
     const long waves = (r.B + resident - 1) / resident;
     const double t_stream = static_cast<double>(stage) / 45.0e3;
-    double t_chain = 4.5 / n_buf;
+    double t_chain = 4.5 / n_buf + 0.02 * c;   // the statistics exchange grows with the cluster
     if (n_slot < 2 * n_buf) {
       // Tight slots: the exchange over the cluster is on the critical path of every head (d = 2)
       // or of every head twice (d = 1).  Measured per head: 2.6 .. 3.3 us at 11 .. 16 CTAs with
