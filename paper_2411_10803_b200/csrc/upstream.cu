@@ -240,30 +240,38 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
       q_s[d] = __bfloat162float(p.q_cls[(static_cast<size_t>(b) * p.H + h) * p.D + d]);
     __syncthreads();
     const uint4* kh = p.k + (static_cast<size_t>(b) * p.H + h) * M * dv;
+    // Coalesced rows: a group of `grp` lanes (the power of two >= D/8) reads one token's row as
+    // 16-byte vectors; a warp takes 32/grp consecutive tokens per step, two steps in flight.  Each
+    // lane keeps its eight query values in registers for the whole head.
+    int grp = 1;
+    while (grp < dv) grp <<= 1;
+    const int sub = lane % grp, tok_in_warp = lane / grp, per_warp = 32 / grp;
+    float qv[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) qv[e] = sub < dv ? q_s[sub * 8 + e] : 0.0f;
     float mx = -INFINITY;
-    for (int j = threadIdx.x; j < M; j += kThreads) {   // one token per thread: its row is D contiguous bf16
-      float dot = 0.0f;
-      const uint4* krow = kh + static_cast<size_t>(j) * dv;
-      for (int v0 = 0; v0 < dv; v0 += 4) {                 // four 16-byte loads in flight per thread
-        uint4 kv[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-          if (v0 + u < dv) kv[u] = krow[v0 + u];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (v0 + u < dv) {
-            const float4 qa = *reinterpret_cast<const float4*>(&q_s[(v0 + u) * 8]);
-            const float4 qb = *reinterpret_cast<const float4*>(&q_s[(v0 + u) * 8 + 4]);
-            dot = fmaf(bf16_lo(kv[u].x), qa.x, dot); dot = fmaf(bf16_hi(kv[u].x), qa.y, dot);
-            dot = fmaf(bf16_lo(kv[u].y), qa.z, dot); dot = fmaf(bf16_hi(kv[u].y), qa.w, dot);
-            dot = fmaf(bf16_lo(kv[u].z), qb.x, dot); dot = fmaf(bf16_hi(kv[u].z), qb.y, dot);
-            dot = fmaf(bf16_lo(kv[u].w), qb.z, dot); dot = fmaf(bf16_hi(kv[u].w), qb.w, dot);
-          }
-        }
+    const int step = kWarps * per_warp;
+    for (int base = warp * per_warp; base < M; base += 2 * step) {   // warp-uniform trip count
+      const int ja = base + tok_in_warp, jb = ja + step;
+      uint4 ka = make_uint4(0, 0, 0, 0), kb = make_uint4(0, 0, 0, 0);
+      if (ja < M && sub < dv) ka = kh[static_cast<size_t>(ja) * dv + sub];
+      if (jb < M && sub < dv) kb = kh[static_cast<size_t>(jb) * dv + sub];
+      float da = bf16_lo(ka.x) * qv[0], db = bf16_lo(kb.x) * qv[0];
+      da = fmaf(bf16_hi(ka.x), qv[1], da); db = fmaf(bf16_hi(kb.x), qv[1], db);
+      da = fmaf(bf16_lo(ka.y), qv[2], da); db = fmaf(bf16_lo(kb.y), qv[2], db);
+      da = fmaf(bf16_hi(ka.y), qv[3], da); db = fmaf(bf16_hi(kb.y), qv[3], db);
+      da = fmaf(bf16_lo(ka.z), qv[4], da); db = fmaf(bf16_lo(kb.z), qv[4], db);
+      da = fmaf(bf16_hi(ka.z), qv[5], da); db = fmaf(bf16_hi(kb.z), qv[5], db);
+      da = fmaf(bf16_lo(ka.w), qv[6], da); db = fmaf(bf16_lo(kb.w), qv[6], db);
+      da = fmaf(bf16_hi(ka.w), qv[7], da); db = fmaf(bf16_hi(kb.w), qv[7], db);
+      for (int d = grp >> 1; d >= 1; d >>= 1) {       // sum over the group's lanes (fixed tree)
+        da += __shfl_xor_sync(0xffffffffu, da, d);
+        db += __shfl_xor_sync(0xffffffffu, db, d);
       }
-      const float zz = dot * p.scale_log2e;
-      z[j] = zz;
-      mx = fmaxf(mx, zz);
+      if (sub == 0) {
+        if (ja < M) { const float zz = da * p.scale_log2e; z[ja] = zz; mx = fmaxf(mx, zz); }
+        if (jb < M) { const float zz = db * p.scale_log2e; z[jb] = zz; mx = fmaxf(mx, zz); }
+      }
     }
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
