@@ -159,3 +159,33 @@ def test_plan_description_names_the_geometry_without_a_gpu():
     assert md.mustdrop_plan_filter_launches(plan) == 4
     md.mustdrop_plan_destroy(plan)
     assert md.mustdrop_plan_describe(0) == "" or md.mustdrop_plan_filter_launches(0) == -1
+
+
+def test_filter_layer_rejects_bad_arguments_without_a_gpu():
+    w = synth.WORKLOADS["c1_tiny"]
+    st, plan, _ = md.mustdrop_filter_plan(md.config_for(w))
+    assert st == md.MUSTDROP_OK
+    good = dict(q_text=256, k=256, v=256, hidden=256, key_idx=256, key_cnt=256, g_out=256, i_out=256,
+                kept_idx=256, kept_cnt=256, hidden_out=256, k_out=256, v_out=256)
+
+    def call(workspace=256, **kw):
+        a = dict(good)
+        a.update(kw)
+        return md.mustdrop_filter_layer(plan, workspace, 0, **a)
+
+    assert call(q_text=None) == md.MUSTDROP_ERR_INVALID_ARG
+    assert call(kept_cnt=None) == md.MUSTDROP_ERR_INVALID_ARG
+    assert call(key_idx=None) == md.MUSTDROP_ERR_INVALID_ARG              # the plan has a key set
+    assert call(hidden_out=None) == md.MUSTDROP_ERR_INVALID_ARG           # source without destination
+    assert call(key_idx_out=256) == md.MUSTDROP_ERR_INVALID_ARG           # key_cnt_out missing
+    assert call(vis_cnt=264) == md.MUSTDROP_ERR_INVALID_ARG               # misaligned
+    assert call(workspace=None) == md.MUSTDROP_ERR_WORKSPACE
+    md.mustdrop_plan_destroy(plan)
+    # a ragged batch needs the text directly behind the image
+    st, plan, _ = md.mustdrop_filter_plan(md.config_for(w, txt_start=w.txt_start + 8, seq_len=w.seq_len + 8))
+    assert st == md.MUSTDROP_OK
+    assert md.mustdrop_filter_layer(plan, 256, 0, vis_cnt=256, **good) == md.MUSTDROP_ERR_INVALID_ARG
+    md.mustdrop_plan_destroy(plan)
+    import pytest as _pytest
+    with _pytest.raises(TypeError):
+        md.mustdrop_filter_layer(0, 256, 0, no_such_field=1)

@@ -273,3 +273,35 @@ def test_ragged_layer_with_text_rows_in_two_launches(monkeypatch):
     monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "row_split")
     w = small(batch=3, n_vis=260, n_txt=90, n_heads=2, hidden=256, key_cnt=4, budget=40, vis_start=2)
     assert run_ragged_layer(w, np.array([260, 40, 133], np.int32), True) == 2
+
+
+@pytest.mark.parametrize("path", ["one_launch", "two_pass"], indirect=True)
+def test_ragged_layer_threshold_mode_is_the_printed_rule_on_each_requests_own_sizes(path):
+    # Eq. 9 and Eq. 10 as printed, with gamma = 1 / (own tokens) and alpha = 2 / (own length)
+    w = small(batch=4, n_vis=280, n_txt=17, key_cnt=5)
+    d = synth.make_batch(w)
+    vis_cnt = np.array([280, 31, 150, 199], np.int32)
+    p = synth.pack_ragged(d, w, vis_cnt)
+    f = md.Filter(md.config_for(w, mode=md.MUSTDROP_MODE_THRESHOLD, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE))
+    q, k, v, hid = (to_dev_bf16(p[n]) for n in ("q_text", "k", "v", "hidden"))
+    f.filter_layer(q, k, v, hid, to_dev(p["key_idx"]), to_dev(p["key_cnt"]), vis_cnt=to_dev(vis_cnt), want_s=True)
+    torch.cuda.synchronize()
+    assert f.device_status() == (0, 0)
+    g, i = f.g.cpu().numpy(), f.i.cpu().numpy()
+    idx, cnt = f.kept_idx.cpu().numpy(), f.kept_cnt.cpu().numpy()
+    ho = bf16_bits(f.hidden_out)
+    vs, N = w.vis_start, w.n_txt
+    for b, m in enumerate(vis_cnt):
+        lb = vs + int(m) + N
+        G, I = oracle.score(p["q_text"][b:b + 1], p["k"][b:b + 1, :, :lb], vs, int(m), vs + int(m))
+        assert_scores_close(g[b:b + 1, :m], G, "G")
+        assert_scores_close(i[b:b + 1, :m], I, "I")
+        # the selection is a function of its fp32 inputs: the oracle's rule on the GPU's own scores
+        ref_idx, ref_cnt, _, _ = oracle.select(g[b:b + 1, :m].copy(), i[b:b + 1, :m].copy(), lb, p["key_idx"][b:b + 1],
+                                               p["key_cnt"][b:b + 1], mode=oracle.MODE_THRESHOLD)
+        n = int(ref_cnt[0])
+        assert cnt[b] == n and 0 < n <= m
+        assert np.array_equal(idx[b, :n], ref_idx[0, :n])
+        rows = np.concatenate([np.arange(vs), vs + idx[b, :n], vs + m + np.arange(N)])
+        assert np.array_equal(ho[b, :len(rows)], p["hidden"][b, rows])
+    f.close()
