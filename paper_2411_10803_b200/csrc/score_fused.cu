@@ -271,8 +271,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const FusedParams p, const __grid_constant__ GatherMaps gm, const FilterTail ft) {
   constexpr int NROWS = 128 / HALVES;            // text rows carried by the TMEM lanes
-  constexpr int ECH = (ACH + 1) / 2;             // chunks per exp thread
-  constexpr int EPR = kColGroups;                // (max, sum) pairs per text row and CTA: one per column group
+  // How the two exp warps of a lane quadrant share the work.  Wide tiles (ACH > 5): each takes
+  // every second chunk of columns of every head (one (max, sum) pair per warp).  Narrow tiles: the
+  // whole row of a head fits one thread's registers, so the two warps ALTERNATE heads - two heads
+  // are in the exp stage at a time, which hides the tensor-memory load / store latencies that
+  // bound that stage when a head is only a few chunks wide.
+  constexpr bool kAlt = ACH <= 5;
+  constexpr int ECH = kAlt ? ACH : (ACH + 1) / 2;   // chunks per exp thread
+  constexpr int EPR = kAlt ? 1 : kColGroups;        // (max, sum) pairs per text row and CTA
   constexpr bool kRealloc = ACH > 5;             // move registers from the other warpgroups to the add warps
 
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
@@ -307,7 +313,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     for (int s = 0; s < kMaxKBufs; ++s) { mbar_init(smem_u32(&bars.full[s]), 1); mbar_init(smem_u32(&bars.empty[s]), 1); }
     for (int s = 0; s < kMaxBufs; ++s) {
       mbar_init(smem_u32(&bars.tfull[s]), 1);
-      mbar_init(smem_u32(&bars.eready[s]), kExpWarps);
+      mbar_init(smem_u32(&bars.eready[s]), kAlt ? kExpWarps / kColGroups : kExpWarps);
       mbar_init(smem_u32(&bars.tempty[s]), kAddWarps);
     }
     for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), 1);
@@ -519,16 +525,18 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const int row = (HALVES == 2) ? (16 * q + (lane & 15)) : (32 * q + lane);
     const uint32_t lane_addr = static_cast<uint32_t>(32 * q) << 16;
     const int total_chunks = p.cpl / kChunk;
-    const int my_chunks = (total_chunks - g + kColGroups - 1) / kColGroups;   // chunks g, g+2, ... (uniform per warp)
+    // chunks g, g+2, ... of every head, or all chunks of every second head (uniform per warp)
+    const int my_chunks = kAlt ? total_chunks : (total_chunks - g + kColGroups - 1) / kColGroups;
+    auto chunk_of = [&](int t) { return kAlt ? t : g + t * kColGroups; };
     const int key_lane0 = static_cast<int>(rank) * p.tk + half * p.cpl;        // key of this lane's column 0
     int lim = p.causal ? (txt_start + p.row0 + row + 1) : Lb;                  // keys below lim are visible
     lim = (lim < Lb ? lim : Lb) - key_lane0;                                   // ... as a column count of this lane
     const bool all_visible = lim >= p.cpl;
     const bool sender = (half == 0);           // with two halves, lanes s and s+16 share a row: the lower one sends
-    const uint32_t pair_idx = (rank * NROWS + row) * EPR + g;                  // this thread's pair in a slot
+    const uint32_t pair_idx = (rank * NROWS + row) * EPR + (kAlt ? 0 : g);     // this thread's pair in a slot
 
     int last_buf = -1;
-    for (int h = 0; h < p.H; ++h) {
+    for (int h = kAlt ? g : 0; h < p.H; h += kAlt ? kColGroups : 1) {
       const int buf = h % p.n_buf;
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
       const int slot = h % p.n_slot;
@@ -543,8 +551,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           break;
       }
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag))) break;
-      if (threadIdx.x == 0) {
-        MD_TRACE(h, 3);
+      if (threadIdx.x == 0) MD_TRACE(h, 3);
+      if (lane == 0 && q == 0 && (kAlt || g == 0)) {
         // arm this head's statistics barrier with the bytes all CTAs will send
         mbar_expect_tx(smem_u32(&bars.sfull[slot]), slot_pairs * 8u);
       }
@@ -557,18 +565,18 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       float z[ECH][kChunk];
 #pragma unroll
       for (int t = 0; t < ECH; ++t)
-        if (t < my_chunks) tc_ld16(tbuf + kChunk * (g + t * kColGroups), z[t]);
-      if (h > 0 && !p.tight) {
+        if (t < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t), z[t]);
+      if (last_buf >= 0 && !p.tight) {   // the head this warp worked on before
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[(h - 1) % p.n_buf]));
+        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[last_buf]));
       }
       tc_wait_ld();
       if (!all_visible) {
 #pragma unroll
         for (int t = 0; t < ECH; ++t) {
-          const int nvis = lim - kChunk * (g + t * kColGroups);   // visible columns of this chunk
+          const int nvis = lim - kChunk * chunk_of(t);   // visible columns of this chunk
           if (nvis < kChunk) {
 #pragma unroll
             for (int j = 0; j < kChunk; ++j) z[t][j] = (j < nvis) ? z[t][j] : -INFINITY;
@@ -595,7 +603,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             z[t][j] = e;
             ls4[j & 3] += e;
           }
-          tc_st16(tbuf + kChunk * (g + t * kColGroups), z[t]);
+          tc_st16(tbuf + kChunk * chunk_of(t), z[t]);
         }
       float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
       if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
@@ -693,7 +701,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           if (c0 + 1 < ACH && c0 + 1 < total_chunks) tc_ld16(tbuf + kChunk * (c0 + 1), e[1]);
           tc_wait_ld();
           // chunk c was exponentiated by column group c & 1 (c0 is even)
-          const float f0 = f[0], f1 = f[1];
+          const float f0 = f[0], f1 = f[EPR - 1];
 #pragma unroll
           for (int j = 0; j < kChunk; ++j) acc[c0][j] = fmaf(e[0][j], f0, acc[c0][j]);
           if (c0 + 1 < ACH && c0 + 1 < total_chunks) {
