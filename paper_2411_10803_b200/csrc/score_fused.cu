@@ -972,12 +972,20 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     const int max_buf = n_buf;
     size_t extra = 0;
     int n_q = 0, n_k = 0, n_slot = 0, split = 0;
-    for (; n_buf >= kMinBufs; --n_buf) {          // whole stages, full set of slots
-      n_slot = 2 * n_buf;
-      extra = slots_bytes(n_slot);
-      if (extra + 2 * stage > avail) continue;
-      n_q = static_cast<int>((avail - extra) / stage);
-      if (n_q >= 4 || n_buf == kMinBufs) break;
+    {                                              // whole stages, full set of slots
+      // a stage is held for a load latency plus an MMA: as many stages as fit (up to four) first,
+      // then as many buffers as still fit (the MMA -> exp -> exchange -> add chain of ~4.6 us
+      // per head is spread over them)
+      int best_q = 0, best_buf = 0;
+      for (int nb = max_buf; nb >= kMinBufs; --nb) {
+        const size_t e = slots_bytes(2 * nb);
+        if (e + 2 * stage > avail) continue;
+        int q = static_cast<int>((avail - e) / stage);
+        if (q > 4) q = 4;
+        if (q > best_q) { best_q = q; best_buf = nb; }
+      }
+      n_q = best_q;
+      if (best_q >= 2) { n_buf = best_buf; n_slot = 2 * n_buf; extra = slots_bytes(n_slot); }
     }
     if (n_q < 2) {                                 // tight windows
       n_buf = max_buf;
@@ -1016,8 +1024,12 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
       // d = 2, 4.3 us at 10 CTAs with d = 1; a third more with 128 text rows on the lanes.
       t_chain = (n_slot == 4 ? 1.8 + 0.09 * c : 3.0 + 0.13 * c) * (halves == 1 ? 1.3 : 1.0);
     }
-    const double t_head = t_stream > t_chain ? t_stream : t_chain;
-    const double score = 1.0 / (static_cast<double>(waves) * t_head) - 1e-4 * c;   // prefer smaller clusters among equals
+    double t_head = t_stream > t_chain ? t_stream : t_chain;
+    if (t_head < 1.4) t_head = 1.4;   // the exp stage and its hand-overs take that long per head however narrow the tile
+    // among equals: larger clusters while even twice as many CTAs would leave SMs idle (a lone request
+    // gains from spreading its keys), else smaller ones (successive calls overlap better)
+    const double tie = (2 * r.B * c <= sm_count) ? 1e-4 * c : -1e-4 * c;
+    const double score = 1.0 / (static_cast<double>(waves) * t_head) + tie;
     if (score > best) {
       best = score;
       g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_q = n_q; g.n_k = n_k; g.split = split; g.n_buf = n_buf; g.ach = ach;
