@@ -37,8 +37,8 @@ FALLBACK_HBM_GBS = 6650.0
 # captures summarised under profiles/.  Keyed by (workload, budget, "filter" | "score", kernel
 # variant); anything else (or a kernel changed since its capture) reports null.
 NCU_TRAFFIC_BYTES = {
-    ("c2_llava7b_b64", 64, "filter", "fused_cluster_tcgen05"): 468273920 + 45074176,   # profiles/filter_kernel_c2_llava7b_b64.md
-    ("c2_llava7b_b64", 64, "score", "fused_cluster_tcgen05"): 369156096 + 3657472,     # profiles/score_fused_kernel_c2_llava7b_b64.md
+    ("c2_llava7b_b64", 64, "filter", "fused_cluster_tcgen05"): 468290816 + 43839488,   # profiles/filter_kernel_c2_llava7b_b64.md
+    ("c2_llava7b_b64", 64, "score", "fused_cluster_tcgen05"): 369175040 + 2975232,     # profiles/score_fused_kernel_c2_llava7b_b64.md
 }
 
 
