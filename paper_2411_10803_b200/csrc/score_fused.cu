@@ -955,7 +955,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     const int tk = cpl * halves;
     const size_t stage = static_cast<size_t>(nrows + tk) * 256;
     const int ach = cpl <= 5 * kChunk ? 5 : 10;             // chunks per add thread (kernel variant)
-    const int epr = kColGroups;                             // (max, sum) pairs per row and CTA
+    const int epr = ach <= 5 ? 1 : kColGroups;              // (max, sum) pairs per row and CTA (the kernel's EPR)
     // Shared memory.  Whole stages first (a head's query tile and keys recycled together): as many
     // tensor-memory buffers as the columns allow (3..8), fewer if their statistics slots (2 x
     // buffers x cluster x rows x pairs x 8 bytes) would leave no room for 2 stages; four stages
