@@ -3,9 +3,13 @@
 The vision-encoding stage (Local Spatial Merging, Key Retaining; Sec. 3.3) produces the
 tokens and the key set O that the prefill filter consumes; the decoding stage (output-aware
 cache policy, Sec. 3.5) consumes the filter's kept sets.  The paper leaves their constants and
-several details unstated, so every function here is a stated reading and is checked only
-against internal invariants: PARITY UNPINNED for ``local_spatial_merge``, ``key_set`` and
-``cache_policy``.  ``kv_cache_mb`` is pinned to the token/MB pairs of Tables 3 and 6.
+several details unstated, so every function here is a stated reading.  READING UNPINNED,
+ARITHMETIC PINNED for ``local_spatial_merge``, ``key_set`` / ``upper_fence`` and
+``cache_policy``: nothing the paper prints fixes the choice of similarity, weights, tau or
+fence, but the arithmetic of the reading taken is checked against values worked out by hand
+(windows with exactly known cosines, rank-one logits whose softmax is written with
+``math.exp``, quartiles that fall on and between elements).  ``kv_cache_mb`` is pinned to the
+token/MB pairs of Tables 3 and 6.
 """
 from __future__ import annotations
 
@@ -53,6 +57,14 @@ def local_spatial_merge(tokens: np.ndarray, grid: int, window: int = 2, tau: flo
     return out + (np.asarray(all_sims),) if return_sims else out
 
 
+def upper_fence(a: np.ndarray) -> float:
+    """The adaptive threshold mu of Eq. 7, read as Tukey's upper fence of the values a:
+    Q3 + 1.5 (Q3 - Q1), the quartiles interpolated linearly between order statistics (the
+    quartile of n values sits at position (n - 1) p of the sorted list)."""
+    q1, q3 = np.quantile(np.asarray(a, np.float64), [0.25, 0.75])
+    return float(q3 + 1.5 * (q3 - q1))
+
+
 def key_set(q_cls: np.ndarray, k: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     """Key Retaining (Sec. 3.3, Eq. 6-7).
 
@@ -67,8 +79,7 @@ def key_set(q_cls: np.ndarray, k: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     p = np.exp(z)
     p /= p.sum(axis=1, keepdims=True)
     a = p.mean(axis=0)
-    q1, q3 = np.quantile(a, [0.25, 0.75])
-    mu = q3 + 1.5 * (q3 - q1)
+    mu = upper_fence(a)
     return np.nonzero(a > mu)[0].astype(np.int32), a
 
 
