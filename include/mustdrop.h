@@ -16,14 +16,21 @@
  *     mustdrop_device_status.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *     Calls enqueue work and return; issuing score, select, compact in that order on one
- *     stream is the whole protocol.
+ *     stream is the whole protocol.  Every kernel waits for the work that precedes it in the
+ *     stream before it reads an input or writes an output (only its set-up overlaps the end of
+ *     its predecessor), so inputs may come from the kernel enqueued just before the call.
  *   - Host-detectable problems return a non-OK status and launch nothing.  Conditions only
  *     the device can see (a key index outside [0, n_vis)) are recorded in a status word in
  *     the workspace and never trap.
  *   - Sequence layout (Sec. 3.1, "Prefilling"): the n_vis vision tokens occupy positions
  *     [vis_start, vis_start+n_vis), the n_txt text tokens [txt_start, txt_start+n_txt),
  *     vis_start+n_vis <= txt_start, txt_start+n_txt <= seq_len.
- *   - A plan is immutable; concurrent calls are safe when they use distinct workspaces.
+ *   - A plan's configuration is immutable.  Calls from several host threads are safe when they
+ *     use distinct workspaces (launch attributes of the kernels are set once per device, and the
+ *     plan's cache of encoded tensor maps is guarded by a lock).
+ *   - A request whose result is invalid because a bounded wait inside the one-launch filter
+ *     kernel ran out gets kept_cnt[b] = -1 (and MUSTDROP_ERR_TIMEOUT in the device status word);
+ *     its other outputs are unspecified.
  */
 #ifndef MUSTDROP_H_
 #define MUSTDROP_H_
@@ -62,7 +69,8 @@ typedef enum {
  * MUSTDROP_FLAG_REBUILD_SEQUENCE: the compacted outputs hold the request's whole next sequence
  * instead of the kept vision rows only: the vis_start prefix rows, the kept vision rows, then
  * the n_txt text rows, packed without a gap - the input layout of the next pruning layer
- * (Sec. 3.4 filters "from the shallow layers" on, every layer on what the last one kept).
+ * (the paper's overview has the filter applied gradually at several layers, each on what the
+ * layer before it kept).
  * Outputs then have vis_start + cap + n_txt rows per request (and head); rows behind a
  * request's own end are left untouched.  Requires txt_start == vis_start + n_vis and
  * seq_len == txt_start + n_txt.
@@ -73,9 +81,19 @@ typedef enum {
  * MUSTDROP_FLAG_PER_HEAD_MAX: the other reading of Eq. 10 over attention heads, which the paper
  * leaves open: i_out[b][j] = mean over heads of ( max over text tokens of p^h[i][vis_start + j] )
  * instead of the maximum of the head-mean attention.  g_out (Eq. 8) is the same under both.
- * Plans with this flag run the two-pass score kernel.
  */
 #define MUSTDROP_FLAG_PER_HEAD_MAX 2
+
+/*
+ * MUSTDROP_FLAG_INPUTS_READY: a promise by the caller that q_text and k were completely written,
+ * and visible to the device, before the kernel that PRECEDES this call in the stream started
+ * (e.g. they were produced several kernels earlier, or uploaded and synchronised).  The score
+ * part then starts streaming keys without waiting for that predecessor to finish, so the
+ * beginning of one call overlaps the end of the call before it.  Without the flag (the default)
+ * nothing is read before all earlier work in the stream has completed.  Outputs are always
+ * written after that wait.  Ignored when vis_cnt is given to mustdrop_filter_layer.
+ */
+#define MUSTDROP_FLAG_INPUTS_READY 4
 
 typedef struct {
   int32_t batch;      /* B, independent requests */
@@ -101,7 +119,20 @@ typedef struct {
   int64_t k_stride_b, k_stride_h, k_stride_l;       /* K      [B,H,L,D] */
   int64_t v_stride_b, v_stride_h, v_stride_l;       /* V      [B,H,L,D] */
   int64_t hid_stride_b, hid_stride_l;               /* hidden [B,L,hidden] */
+  /* Debugging overrides of the planner, for tests and sweeps.  All 0 in normal use. */
+  int32_t debug_score_variant;  /* mustdrop_debug_variant_t: force a score kernel */
+  int32_t debug_cluster;        /* 1..16: force the fused kernel's cluster size */
+  int32_t debug_filter_staged;  /* 1: mustdrop_filter enqueues the separate kernels even where one launch would do */
+  int32_t debug_wait_cycles;    /* > 0: waits between the warp roles of the fused kernel give up after this many
+                                   SM clock cycles instead of ~0.1 s (used to exercise the time-out path) */
 } mustdrop_config_t;
+
+typedef enum {
+  MUSTDROP_DEBUG_VARIANT_AUTO = 0,
+  MUSTDROP_DEBUG_VARIANT_TWO_PASS = 1,   /* the general-shape two-pass kernel */
+  MUSTDROP_DEBUG_VARIANT_FUSED = 2,      /* the one-pass tcgen05 kernel, whatever the cost model says */
+  MUSTDROP_DEBUG_VARIANT_ROW_SPLIT = 3   /* the one-pass kernel with the text rows scored by two launches */
+} mustdrop_debug_variant_t;
 
 /*
  * Validate a configuration and build a plan (host only; nothing is launched).
@@ -185,7 +216,8 @@ mustdrop_status_t mustdrop_select(const mustdrop_plan_t *plan, const float *g, c
  * hidden_out [B,cap,hidden], k_out, v_out [B,H,cap,D].  Rows r >= kept_cnt[b] are left
  * untouched.  Any of the three (source, destination) pairs may be NULL together to skip it.
  * An index outside [0, n_vis) is skipped and, when workspace is not NULL, recorded in its
- * device status word.
+ * device status word.  A kept_cnt[b] above cap is clamped to cap; a negative one (a request
+ * marked invalid) copies nothing for that request; both are recorded the same way.
  */
 mustdrop_status_t mustdrop_compact(const mustdrop_plan_t *plan, const int32_t *kept_idx,
                                    const int32_t *kept_cnt, const void *hidden, const void *k,

@@ -50,11 +50,17 @@ class mustdrop_config_t(ctypes.Structure):
         ("k_stride_b", ctypes.c_int64), ("k_stride_h", ctypes.c_int64), ("k_stride_l", ctypes.c_int64),
         ("v_stride_b", ctypes.c_int64), ("v_stride_h", ctypes.c_int64), ("v_stride_l", ctypes.c_int64),
         ("hid_stride_b", ctypes.c_int64), ("hid_stride_l", ctypes.c_int64),
+        ("debug_score_variant", ctypes.c_int32), ("debug_cluster", ctypes.c_int32),
+        ("debug_filter_staged", ctypes.c_int32), ("debug_wait_cycles", ctypes.c_int32),
     ]
 
 
 MUSTDROP_FLAG_REBUILD_SEQUENCE = 1
 MUSTDROP_FLAG_PER_HEAD_MAX = 2
+MUSTDROP_FLAG_INPUTS_READY = 4
+
+MUSTDROP_DEBUG_VARIANT_AUTO, MUSTDROP_DEBUG_VARIANT_TWO_PASS = 0, 1
+MUSTDROP_DEBUG_VARIANT_FUSED, MUSTDROP_DEBUG_VARIANT_ROW_SPLIT = 2, 3
 
 
 class mustdrop_layer_io_t(ctypes.Structure):
@@ -169,6 +175,10 @@ class Config:
     v_stride_l: int = 0
     hid_stride_b: int = 0
     hid_stride_l: int = 0
+    debug_score_variant: int = 0
+    debug_cluster: int = 0
+    debug_filter_staged: int = 0
+    debug_wait_cycles: int = 0
 
     def to_c(self) -> mustdrop_config_t:
         c = mustdrop_config_t()

@@ -50,7 +50,13 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
   pdl_launch_dependents();
   pdl_wait();   // kept_idx / kept_cnt come from the previous kernel in the stream
   if (p.src[which] == nullptr) return;
-  const int n_kept = min(p.kept_cnt[b], p.cap);
+  // a count outside [0, cap] is not trusted: clamped, and recorded (a negative one marks a request
+  // whose selection failed: nothing of it is copied)
+  const int cnt_raw = p.kept_cnt[b];
+  const int n_kept = min(max(cnt_raw, 0), p.cap);
+  if (cnt_raw != n_kept && threadIdx.x == 0 && r == 0)
+    record_status(p.workspace, MUSTDROP_ERR_BAD_KEY_INDEX, b * 65536 + 65535);
+  if (cnt_raw < 0) return;
   int64_t row;        // source row
   int out_row = r;    // destination row
   if (!p.rebuild || (r >= p.vis_start && r < p.vis_start + p.cap)) {

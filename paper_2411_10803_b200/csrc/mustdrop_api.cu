@@ -4,7 +4,10 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
+#include <set>
+#include <utility>
 
 #include "mustdrop_internal.h"
 
@@ -27,6 +30,32 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 namespace mustdrop {
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int32_t>(e); }
+
+cudaError_t ensure_kernel_attributes(const void* kernel, bool nonportable_cluster) {
+  static std::mutex mu;
+  static std::set<std::pair<const void*, int>> done;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(mu);
+  const auto key = std::make_pair(kernel, dev);
+  if (done.count(key)) return cudaSuccess;
+  cudaFuncAttributes fa;
+  e = cudaFuncGetAttributes(&fa, kernel);
+  if (e != cudaSuccess) return e;
+  int optin = 0;
+  e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           optin - static_cast<int>(fa.sharedSizeBytes));
+  if (e != cudaSuccess) return e;
+  if (nonportable_cluster) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+  }
+  done.insert(key);
+  return cudaSuccess;
+}
 }  // namespace mustdrop
 
 extern "C" {
@@ -39,7 +68,10 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   *workspace_bytes = 0;
   if (c->batch <= 0 || c->n_heads <= 0 || c->head_dim <= 0 || c->hidden <= 0 || c->seq_len <= 0 ||
       c->n_vis <= 0 || c->n_txt <= 0 || c->vis_start < 0 || c->txt_start < 0 || c->key_max < 0 ||
-      (c->flags & ~(MUSTDROP_FLAG_REBUILD_SEQUENCE | MUSTDROP_FLAG_PER_HEAD_MAX)) != 0)
+      (c->flags & ~(MUSTDROP_FLAG_REBUILD_SEQUENCE | MUSTDROP_FLAG_PER_HEAD_MAX | MUSTDROP_FLAG_INPUTS_READY)) != 0)
+    return MUSTDROP_ERR_INVALID_ARG;
+  if (c->debug_score_variant < MUSTDROP_DEBUG_VARIANT_AUTO || c->debug_score_variant > MUSTDROP_DEBUG_VARIANT_ROW_SPLIT ||
+      c->debug_cluster < 0 || c->debug_cluster > 16 || (c->debug_filter_staged & ~1) != 0 || c->debug_wait_cycles < 0)
     return MUSTDROP_ERR_INVALID_ARG;
   // the vision span precedes the text span and both lie inside the sequence
   if (static_cast<int64_t>(c->vis_start) + c->n_vis > c->txt_start ||
@@ -80,6 +112,8 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   r.cap = (c->mode == MUSTDROP_MODE_BUDGET) ? c->budget : c->n_vis;
   r.rebuild = (c->flags & MUSTDROP_FLAG_REBUILD_SEQUENCE) ? 1 : 0;
   r.per_head_max = (c->flags & MUSTDROP_FLAG_PER_HEAD_MAX) ? 1 : 0;
+  r.inputs_ready = (c->flags & MUSTDROP_FLAG_INPUTS_READY) ? 1 : 0;
+  r.wait_cycles = c->debug_wait_cycles;
   r.out_rows = r.rebuild ? c->vis_start + r.cap + c->n_txt : r.cap;
   r.gamma_default = c->gamma == 0.0f;
   r.alpha_default = c->alpha == 0.0f;
@@ -114,15 +148,13 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   (void)cudaGetLastError();
 
   // Score kernel: the fused single-pass kernel where its geometry covers the shape, else the
-  // two-pass kernel.  MUSTDROP_SCORE_VARIANT (two_pass | fused | row_split) and MUSTDROP_CLUSTER (1..16) are
-  // debugging overrides read here, once per plan.
+  // two-pass kernel.  The configuration's debug_score_variant / debug_cluster override the choice.
   p->score_variant = kScoreTwoPassMma;
   {
-    const char* want = std::getenv("MUSTDROP_SCORE_VARIANT");
-    const char* cl = std::getenv("MUSTDROP_CLUSTER");
-    const int forced_cluster = cl ? std::atoi(cl) : 0;
-    const bool allow_fused = !(want && std::strcmp(want, "two_pass") == 0) && !r.per_head_max;
-    const bool force_split = want && std::strcmp(want, "row_split") == 0;
+    const bool want = c->debug_score_variant != MUSTDROP_DEBUG_VARIANT_AUTO;   // a variant is forced
+    const int forced_cluster = c->debug_cluster;
+    const bool allow_fused = c->debug_score_variant != MUSTDROP_DEBUG_VARIANT_TWO_PASS && !r.per_head_max;
+    const bool force_split = c->debug_score_variant == MUSTDROP_DEBUG_VARIANT_ROW_SPLIT;
     const double k_mb = 256.0e-6 * r.B * r.H * r.L;
     const double two_pass_us = k_mb * (0.6 + 0.7 * r.N / 128.0);   // the two-pass kernel's measured rate
     double chosen_us = two_pass_us;
@@ -134,7 +166,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
       // more than 8 CTAs) can be slower than reading K twice: compare with the two-pass kernel
       // unless the variant is forced.
       const bool tight = p->fused.n_slot < 2 * p->fused.n_buf;
-      if (tight && want == nullptr && forced_cluster == 0 && p->fused.est_us > two_pass_us) {
+      if (tight && !want && forced_cluster == 0 && p->fused.est_us > two_pass_us) {
         p->score_variant = kScoreTwoPassMma;
         chosen_us = two_pass_us;
       }
@@ -155,7 +187,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
       if (ok) {
         const bool together = r.B * (ga.cluster + gb.cluster) <= p->sm_count;   // both launches resident at once
         const double split_us = together ? 1.15 * (ga.est_us > gb.est_us ? ga.est_us : gb.est_us) : ga.est_us + gb.est_us;
-        if (force_split || (want == nullptr && forced_cluster == 0 && split_us < chosen_us)) {
+        if (force_split || (!want && forced_cluster == 0 && split_us < chosen_us)) {
           p->score_variant = kScoreFusedCluster;
           p->row_split = 1;
           p->fused = ga;
@@ -164,10 +196,9 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
       }
     }
     // mustdrop_filter: one launch where the fused kernel covers the shape and a kept row fits its
-    // shared-memory ring; MUSTDROP_FILTER=staged forces the three launches (debugging override).
-    const char* fw = std::getenv("MUSTDROP_FILTER");
+    // shared-memory ring; debug_filter_staged forces the separate launches.
     p->filter_single = 0;
-    if (p->score_variant == kScoreFusedCluster && !(fw && std::strcmp(fw, "staged") == 0) &&
+    if (p->score_variant == kScoreFusedCluster && !c->debug_filter_staged &&
         plan_filter_single(r, p->row_split ? p->fused_b : p->fused, &p->filter))
       p->filter_single = 1;
   }
@@ -175,6 +206,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   p->ws_rowstats_off = off;
   off += round_up(sizeof(float) * 2 * static_cast<size_t>(r.B) * r.H * r.N, 256);
   p->ws_bytes = off;
+  p->map_cache = map_cache_create();
   *workspace_bytes = p->ws_bytes;
   *plan_out = p;
   return MUSTDROP_OK;
@@ -184,6 +216,7 @@ mustdrop_status_t mustdrop_plan_destroy(mustdrop_plan_t* plan) {
   if (plan == nullptr) return MUSTDROP_OK;
   if (!valid_plan(plan)) return MUSTDROP_ERR_INVALID_ARG;
   plan->magic = 0;
+  mustdrop::map_cache_destroy(plan->map_cache);
   delete plan;
   return MUSTDROP_OK;
 }

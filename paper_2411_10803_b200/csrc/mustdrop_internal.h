@@ -49,7 +49,9 @@ struct FilterGeometry {
 struct Resolved {
   int32_t B, H, D, hidden, L, vis_start, M, txt_start, N;
   int32_t causal, mode, criteria, budget, key_max, cap;
-  int32_t per_head_max;   // Eq. 10 per head, then the head mean (two-pass kernel only)
+  int32_t per_head_max;   // Eq. 10 per head, then the head mean
+  int32_t inputs_ready;   // the caller promises q_text / k were complete before the stream's previous kernel began
+  int32_t wait_cycles;    // > 0: the fused kernel's role waits give up after this many cycles (debugging)
   int32_t rebuild;        // outputs hold [prefix ; kept vision ; text] instead of the kept vision rows only
   int32_t out_rows;       // rows per request (and head) of hidden_out / k_out / v_out
   int32_t gamma_default, alpha_default;   // thresholds follow each request's own sizes (ragged batches)
@@ -69,6 +71,11 @@ struct LayerArgs {
 // Number of vision tokens of request b: the plan's n_vis, or vis_cnt[b] clamped to [1, n_vis].
 __host__ __device__ inline int32_t clamp_vis_cnt(int32_t v, int32_t M) { return v < 1 ? 1 : (v > M ? M : v); }
 
+// Encoded tensor maps of recent calls (defined with the fused kernel's launch code).
+struct MapCache;
+MapCache* map_cache_create();
+void map_cache_destroy(MapCache* c);
+
 }  // namespace mustdrop
 
 struct mustdrop_plan {
@@ -85,6 +92,7 @@ struct mustdrop_plan {
   mustdrop::FusedGeometry fused_b;
   int32_t filter_single;    // 1: mustdrop_filter is one launch of the fused kernel with its tail
   mustdrop::FilterGeometry filter;
+  mustdrop::MapCache* map_cache;   // guarded by its own lock; null: every call encodes its maps
 };
 
 namespace mustdrop {
@@ -111,6 +119,12 @@ cudaError_t launch_select(const mustdrop_plan& p, const float* g, const float* i
 cudaError_t launch_compact(const mustdrop_plan& p, const int32_t* kept_idx, const int32_t* kept_cnt,
                            const void* hidden, const void* k, const void* v, void* hidden_out, void* k_out,
                            void* v_out, void* workspace, cudaStream_t stream, const int32_t* vis_cnt = nullptr);
+
+// Launch attributes of a kernel, set ONCE per device and never changed afterwards (so that host
+// threads with different plans cannot interleave a set with a launch): the largest dynamic shared
+// memory the device grants next to the kernel's static part and, if asked, the opt-in to clusters
+// of more than 8 CTAs.
+cudaError_t ensure_kernel_attributes(const void* kernel, bool nonportable_cluster);
 
 // Remember the cudaError_t of a failed runtime call for mustdrop_last_cuda_error (per thread).
 void set_last_cuda_error(cudaError_t e);

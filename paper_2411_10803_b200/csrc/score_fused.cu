@@ -26,6 +26,10 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstring>
+#include <mutex>
+#include <new>
+
 #include "mustdrop_internal.h"
 #include "select_body.cuh"
 
@@ -65,6 +69,8 @@ struct FusedParams {
   int32_t split;
   int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (2 * n_buf, or 4 when tight)
   int32_t tight;                      // d = 1 or 2: the exp warps start head h only when the add warps are done with head h - d (0: no such rule)
+  int32_t early_inputs;               // 1: q_text / k may be read before the stream's earlier work has completed (caller's promise)
+  long long wait_cycles;              // clock cycles after which a wait between the warp roles gives up
   float scale_log2e, inv_heads;
 };
 
@@ -110,11 +116,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (and raises the CTA's abort flag) when the wait ran out or the
 // CTA has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (*abort_flag != 0 || clock64() - t0 > kWaitCycles) {
+    if (*abort_flag != 0 || clock64() - t0 > limit) {
       *abort_flag = 1;
       return false;
     }
@@ -132,6 +138,12 @@ __device__ __forceinline__ void st_async_f32x2(uint32_t addr, float a, float b, 
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];" ::"r"(addr),
                "f"(a), "f"(b), "r"(bar)
                : "memory");
+}
+// Barrier over all threads of the CTA, counted per thread: warps whose lanes took different
+// roles (one lane drives the copies or the MMAs, the others only wait) may arrive diverged.
+__device__ __forceinline__ void cta_sync() { asm volatile("barrier.sync 0, %0;" ::"n"(kThreads) : "memory"); }
+__device__ __forceinline__ void st_remote_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -284,9 +296,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
   __shared__ Barriers bars;
   __shared__ uint32_t tmem_base_holder;
-  __shared__ int abort_flag_s;
+  __shared__ int abort_flag_s;          // this CTA gave up a wait
+  __shared__ int cluster_abort_s;       // some CTA of the cluster did (written by that CTA before the exit barrier)
 
   volatile int* abort_flag = &abort_flag_s;
+  const long long wait_limit = p.wait_cycles;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_cta_rank();
   const int b = blockIdx.x / p.cluster;
@@ -309,6 +323,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
+    cluster_abort_s = 0;
     for (int s = 0; s < kMaxQBufs; ++s) { mbar_init(smem_u32(&bars.qfull[s]), 1); mbar_init(smem_u32(&bars.qempty[s]), 1); }
     for (int s = 0; s < kMaxKBufs; ++s) { mbar_init(smem_u32(&bars.full[s]), 1); mbar_init(smem_u32(&bars.empty[s]), 1); }
     for (int s = 0; s < kMaxBufs; ++s) {
@@ -331,9 +346,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   __syncthreads();
   cluster_sync_all();   // every CTA's barriers are initialised before any remote store counts on them
   tc_fence_after();
-  // Let the next kernel in the stream begin its prologue.  This kernel only reads q_text and k,
-  // which no kernel of the library writes, so it does not wait for its predecessors here; the add
-  // warps wait just before they store g_out / i_out, which an earlier select may still be reading.
+  // Let the next kernel in the stream begin its prologue.  Everything up to here touched no
+  // global data; the copy thread waits for the stream's earlier work before its first load (its
+  // inputs may come from the kernel just before this one), the other roles before their stores.
   pdl_launch_dependents();
   const uint32_t tmem_base = tmem_base_holder;
   // This request's own sequence.  In a ragged batch the token count comes from an earlier
@@ -353,15 +368,34 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   // every role keeps the register count setmaxnreg gave it; no second setmaxnreg is needed.)
   __shared__ int32_t kept_total_s;
   auto common_exit = [&]() {
+    __syncwarp();   // a warp whose lane 0 had a role of its own is whole again before the aligned instructions below
     tc_fence_before();
-    __syncthreads();
-    if (threadIdx.x == 0 && *abort_flag != 0) record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
+    cta_sync();
+    if (threadIdx.x == 0 && *abort_flag != 0) {
+      record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
+      for (int c = 0; c < p.cluster; ++c) st_remote_u32(map_to_cta(smem_u32(&cluster_abort_s), c), 1u);
+    }
     if (warp == kMmaWarp) {
       tc_fence_after();
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
-    cluster_sync_all();
+    cluster_sync_all();   // (release / acquire: a peer's flag store above is visible behind it)
     MD_PIPE(p.workspace, 0, true, false);
+  };
+  // After common_exit: did any CTA of the cluster give up?  (Stable by then: same answer in every thread.)
+  auto cluster_gave_up = [&]() { return *reinterpret_cast<volatile int*>(&cluster_abort_s) != 0; };
+  // The way out after a give-up, taken by every thread of every CTA of the cluster.  A peer's
+  // asynchronous statistics stores may still be on their way into this CTA's shared memory: give
+  // them time to land and meet once more, so that no CTA's shared memory goes away under them.
+  auto leave_after_give_up = [&](int32_t* kept_cnt) {
+    if (kept_cnt != nullptr && rank == 0 && threadIdx.x == 0) {
+      pdl_wait();
+      kept_cnt[b] = -1;   // this request's result is invalid
+    }
+    const long long t0 = clock64();
+    while (clock64() - t0 < 40000) {}
+    __syncwarp();
+    cluster_sync_all();
   };
   int32_t* const kept_list = reinterpret_cast<int32_t*>(stage_ptr);   // filter tail: the request's kept indices
 
@@ -371,12 +405,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       // ---------------- TMA producer ----------------
       const int key0 = static_cast<int>(rank) * p.tk;
       const uint64_t stream_once = l2_evict_first_policy();
+      if (!p.early_inputs) pdl_wait();   // q_text / k may be the output of the kernel just before this one
       if (p.split) {
         int q_issued = 0, k_issued = 0;   // tiles started so far
         bool ok = true;
         for (int h = 0; h < p.H && ok; ++h) {
           const int qi = h % p.n_q;
-          if (!mbar_wait(smem_u32(&bars.qempty[qi]), (static_cast<uint32_t>(h / p.n_q) & 1u) ^ 1u, abort_flag)) break;
+          if (!mbar_wait(smem_u32(&bars.qempty[qi]), (static_cast<uint32_t>(h / p.n_q) & 1u) ^ 1u, abort_flag, wait_limit)) break;
           const uint32_t qfull = smem_u32(&bars.qfull[qi]);
           const uint32_t q_dst = stage_base + qi * q_bytes;
           mbar_expect_tx(qfull, q_bytes);
@@ -387,7 +422,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   #pragma unroll
           for (int hv = 0; hv < HALVES; ++hv) {
             const int ki = k_issued % p.n_k;
-            if (!mbar_wait(smem_u32(&bars.empty[ki]), (static_cast<uint32_t>(k_issued / p.n_k) & 1u) ^ 1u, abort_flag)) {
+            if (!mbar_wait(smem_u32(&bars.empty[ki]), (static_cast<uint32_t>(k_issued / p.n_k) & 1u) ^ 1u, abort_flag, wait_limit)) {
               ok = false;
               break;
             }
@@ -417,7 +452,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         for (int h = 0; h < p.H; ++h) {
           const int s = h % p.n_q;
           const uint32_t ph = static_cast<uint32_t>(h / p.n_q) & 1u;
-          if (!mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag)) break;
+          if (!mbar_wait(smem_u32(&bars.empty[s]), ph ^ 1u, abort_flag, wait_limit)) break;
           const uint32_t full = smem_u32(&bars.full[s]);
           const uint32_t q_dst = stage_base + s * stage_bytes;
           const uint32_t k_dst = q_dst + NROWS * 256u;
@@ -445,21 +480,22 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       // ---------------- MMA issuer ----------------
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(p.cpl >> 3) << 17) |
                              (static_cast<uint32_t>(NROWS >> 4) << 24);
+      int committed = -1;   // last head whose MMAs were committed to its tfull barrier
       if (p.split) {
         int k_used = 0;
         bool ok = true;
         for (int h = 0; h < p.H && ok; ++h) {
           const int qi = h % p.n_q, buf = h % p.n_buf;
           const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
-          if (!mbar_wait(smem_u32(&bars.qfull[qi]), static_cast<uint32_t>(h / p.n_q) & 1u, abort_flag)) break;
+          if (!mbar_wait(smem_u32(&bars.qfull[qi]), static_cast<uint32_t>(h / p.n_q) & 1u, abort_flag, wait_limit)) break;
           MD_TRACE(h, 1);
-          if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag)) break;
+          if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag, wait_limit)) break;
           MD_TRACE(h, 2);
           const uint32_t q_src = stage_base + qi * q_bytes;
   #pragma unroll
           for (int hv = 0; hv < HALVES; ++hv) {
             const int ki = k_used % p.n_k;
-            if (!mbar_wait(smem_u32(&bars.full[ki]), static_cast<uint32_t>(k_used / p.n_k) & 1u, abort_flag)) {
+            if (!mbar_wait(smem_u32(&bars.full[ki]), static_cast<uint32_t>(k_used / p.n_k) & 1u, abort_flag, wait_limit)) {
               ok = false;
               break;
             }
@@ -480,15 +516,16 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           if (!ok) break;
           tc_commit(smem_u32(&bars.qempty[qi]));
           tc_commit(smem_u32(&bars.tfull[buf]));
+          committed = h;
         }
       } else {
         for (int h = 0; h < p.H; ++h) {
           const int s = h % p.n_q, buf = h % p.n_buf;
           const uint32_t ph = static_cast<uint32_t>(h / p.n_q) & 1u;
           const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
-          if (!mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag)) break;
+          if (!mbar_wait(smem_u32(&bars.full[s]), ph, abort_flag, wait_limit)) break;
           MD_TRACE(h, 1);
-          if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag)) break;
+          if (!mbar_wait(smem_u32(&bars.tempty[buf]), bph ^ 1u, abort_flag, wait_limit)) break;
           MD_TRACE(h, 2);
           tc_fence_after();
           const uint32_t q_src = stage_base + s * stage_bytes;
@@ -507,14 +544,22 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           }
           tc_commit(smem_u32(&bars.empty[s]));
           tc_commit(smem_u32(&bars.tfull[buf]));
+          committed = h;
         }
+      }
+      if (*abort_flag != 0 && committed >= 0) {
+        // gave up: leave only when the MMAs already issued have finished writing tensor memory (bounded)
+        const uint32_t bar = smem_u32(&bars.tfull[committed % p.n_buf]);
+        const uint32_t ph = static_cast<uint32_t>(committed / p.n_buf) & 1u;
+        const long long t0 = clock64();
+        while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles) {}
       }
     }
     if constexpr (FILTER) {
       // filter tail, TMA / MMA warps: nothing to do but to meet the others
-      __syncwarp();
       common_exit();
-      if (*abort_flag == 0) __syncthreads();   // (the flag no longer changes: same decision in every thread)
+      if (cluster_gave_up()) { leave_after_give_up(ft.sel.kept_cnt); return; }
+      cta_sync();   // pairs with the barrier after the selection
       return;
     }
   } else if (warp < kExpWarps) {
@@ -547,10 +592,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         // done with h - 2d), so 2d slots are enough whatever the number of buffers.
         const int u = h - p.tight;
         if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tempty[u % p.n_buf]),
-                                               static_cast<uint32_t>(u / p.n_buf) & 1u, abort_flag)))
+                                               static_cast<uint32_t>(u / p.n_buf) & 1u, abort_flag, wait_limit)))
           break;
       }
-      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag, wait_limit))) break;
       if (threadIdx.x == 0) MD_TRACE(h, 3);
       if (lane == 0 && q == 0 && (kAlt || g == 0)) {
         // arm this head's statistics barrier with the bytes all CTAs will send
@@ -634,8 +679,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       // inputs, fixed order: identical lists); rank 0 stores the list.
       __shared__ SelectShared sel_sh;
       common_exit();
+      if (cluster_gave_up()) { leave_after_give_up(ft.sel.kept_cnt); return; }
       pdl_wait();   // the outputs written below may still be read by an earlier kernel in the stream
-      if (*abort_flag != 0) return;
       const int tid = threadIdx.x;
       select_clear(sel_sh, tid);
       const bool writer = rank == 0;
@@ -645,7 +690,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       else if (own <= 4) select_request<4, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
       else if (own <= 8) select_request<8, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
       else select_request<16, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-      __syncthreads();   // the list is complete: the copy thread may start
+      cta_sync();   // the list is complete: the copy thread may start
       return;
     }
   } else {
@@ -670,7 +715,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
       const int slot = h % p.n_slot;
       const uint32_t sph = static_cast<uint32_t>(h / p.n_slot) & 1u;
-      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag, wait_limit))) break;
       if (tid_a == 0) MD_TRACE(h, 5);
       // statistics of this row over the whole key range: every CTA's pairs
       const float2* srow = stats + slot * slot_pairs + row * EPR;
@@ -689,7 +734,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       float f[EPR];                            // factor of each of this CTA's pairs
 #pragma unroll
       for (int x = 0; x < EPR; ++x) f[x] = ex2(srow[rank * NROWS * EPR + x].x - m) * inv_l;
-      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.eready[buf]), bph, abort_flag))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.eready[buf]), bph, abort_flag, wait_limit))) break;
       if (tid_a == 0) MD_TRACE(h, 6);
       tc_fence_after();
       const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
@@ -718,7 +763,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 
     // head mean -> column sum (Eq. 8) and column max (Eq. 10) over the text rows
     mbar_arrive(smem_u32(&bars.fin));
-    if (__all_sync(0xffffffffu, h == p.H && mbar_wait(smem_u32(&bars.fin), 0u, abort_flag))) {
+    if (__all_sync(0xffffffffu, h == p.H && mbar_wait(smem_u32(&bars.fin), 0u, abort_flag, wait_limit))) {
       // all TMA copies have landed and all MMAs have read them: the staging area is free
       float* mat = reinterpret_cast<float*>(stage_ptr);
       const int ld = p.tk | 1;
@@ -733,7 +778,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         }
       }
       mbar_arrive(smem_u32(&bars.fin));
-      const bool staged = mbar_wait(smem_u32(&bars.fin), 1u, abort_flag);
+      const bool staged = mbar_wait(smem_u32(&bars.fin), 1u, abort_flag, wait_limit);
       pdl_wait();
       for (int c = tid_a; staged && c < p.tk; c += kAddThreads) {
         const int j = static_cast<int>(rank) * p.tk + c - p.vis_start;   // vision-relative index
@@ -757,9 +802,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     if constexpr (FILTER) {
       // filter tail, add warps: row r of the compacted outputs is copied by CTA r mod cluster
       common_exit();
+      if (cluster_gave_up()) { leave_after_give_up(ft.sel.kept_cnt); return; }
       pdl_wait();
-      if (*abort_flag != 0) return;
-      __syncthreads();   // the exp warps have finished the selection
+      cta_sync();   // the exp warps have finished the selection
       if (warp == kExpWarps && lane == 0) {
         // One thread drives the copies: rows are loaded into a ring of shared-memory slots by bulk
         // copies that count on the slot's mbarrier, and stored from there by bulk copies tracked in
@@ -810,7 +855,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           const int c = i - ahead;
           if (c >= 0) {
             const int slot = c % S;
-            if (!mbar_wait(smem_u32(&bars.gfull[slot]), static_cast<uint32_t>(c / S) & 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(smem_u32(&bars.gfull[slot]), static_cast<uint32_t>(c / S) & 1u, abort_flag, kWaitCycles)) { ok = false; break; }
             const int r = dst_row(static_cast<int>(rank) + c * C);
             uint32_t src = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
             if (ft.hidden_bytes > 0) {
@@ -828,6 +873,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         if (!ok) {
           // gave up: still leave only when every load this thread started has landed (bounded)
           record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
+          ft.sel.kept_cnt[b] = -1;   // some of this request's rows were not copied
           for (int i = (loaded > S ? loaded - S : 0); i < loaded; ++i) {
             const uint32_t bar = smem_u32(&bars.gfull[i % S]);
             const long long t0 = clock64();
@@ -841,6 +887,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   }
 
   common_exit();   // (score-only kernel; the filter kernel's roles have left above)
+  if (cluster_gave_up()) leave_after_give_up(nullptr);
 }
 
 // ---- host side ------------------------------------------------------------------------------------
@@ -889,6 +936,25 @@ bool make_gather_map(CUtensorMap* map, const void* base, uint64_t d1, uint64_t d
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+}  // namespace
+
+// Encoded tensor maps of recent calls, kept with the plan: a steady-state call with pointers it
+// has seen before (a serving loop cycles through a few buffer sets) encodes nothing.
+struct MapCache {
+  struct ScoreEntry { const void* q; const void* k; int geo; CUtensorMap q_map, k_map; };
+  struct GatherEntry { const void* k; const void* v; const void* k_out; const void* v_out; GatherMaps maps; };
+  static constexpr int kEntries = 16;
+  std::mutex mu;
+  ScoreEntry score[kEntries];
+  GatherEntry gather[kEntries];
+  int n_score = 0, n_gather = 0, next_score = 0, next_gather = 0;
+};
+
+MapCache* map_cache_create() { return new (std::nothrow) MapCache(); }
+void map_cache_destroy(MapCache* c) { delete c; }
+
+namespace {
+
 using FusedKernel = void (*)(const CUtensorMap, const CUtensorMap, const FusedParams, const GatherMaps, const FilterTail);
 
 FusedKernel pick_kernel(int halves, int ach, bool filter = false) {
@@ -903,13 +969,7 @@ FusedKernel pick_kernel(int halves, int ach, bool filter = false) {
 // SMs / cluster); 0 when it cannot be asked (no device) or the shape cannot launch.
 int max_resident_clusters(int halves, int ach, int cluster, size_t smem_bytes) {
   FusedKernel kernel = pick_kernel(halves, ach);
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes)) !=
-      cudaSuccess) {
-    (void)cudaGetLastError();
-    return 0;
-  }
-  if (cluster > 8 &&
-      cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+  if (ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), true) != cudaSuccess) {
     (void)cudaGetLastError();
     return 0;
   }
@@ -1055,11 +1115,31 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const FusedGeometry& 
   CUtensorMap q_map, k_map;
   // the launch's text rows: a window of geo.n_rows rows starting at geo.row0 of every head's N rows
   const unsigned char* q_rows = static_cast<const unsigned char*>(q_text) + static_cast<size_t>(geo.row0) * 256;
-  if (!make_map(&q_map, q_rows, geo.n_rows, r.H, r.B, 256, static_cast<uint64_t>(r.N) * 256,
-                static_cast<uint64_t>(r.H) * r.N * 256, nrows) ||
-      !make_map(&k_map, k, r.L, r.H, r.B, static_cast<uint64_t>(r.k_sl) * 2, static_cast<uint64_t>(r.k_sh) * 2,
-                static_cast<uint64_t>(r.k_sb) * 2, geo.cpl))
-    return cudaErrorInvalidValue;
+  const int geo_id = (&geo == &plan.fused_b) ? 1 : 0;
+  bool cached = false;
+  if (MapCache* mc = plan.map_cache) {
+    std::lock_guard<std::mutex> lock(mc->mu);
+    for (int x = 0; x < mc->n_score && !cached; ++x)
+      if (mc->score[x].q == q_rows && mc->score[x].k == k && mc->score[x].geo == geo_id) {
+        q_map = mc->score[x].q_map;
+        k_map = mc->score[x].k_map;
+        cached = true;
+      }
+  }
+  if (!cached) {
+    if (!make_map(&q_map, q_rows, geo.n_rows, r.H, r.B, 256, static_cast<uint64_t>(r.N) * 256,
+                  static_cast<uint64_t>(r.H) * r.N * 256, nrows) ||
+        !make_map(&k_map, k, r.L, r.H, r.B, static_cast<uint64_t>(r.k_sl) * 2, static_cast<uint64_t>(r.k_sh) * 2,
+                  static_cast<uint64_t>(r.k_sb) * 2, geo.cpl))
+      return cudaErrorInvalidValue;
+    if (MapCache* mc = plan.map_cache) {
+      std::lock_guard<std::mutex> lock(mc->mu);
+      MapCache::ScoreEntry& en = mc->score[mc->next_score];
+      en.q = q_rows; en.k = k; en.geo = geo_id; en.q_map = q_map; en.k_map = k_map;
+      mc->next_score = (mc->next_score + 1) % MapCache::kEntries;
+      if (mc->n_score < MapCache::kEntries) ++mc->n_score;
+    }
+  }
   FusedParams p;
   p.g_out = g_out; p.i_out = i_out; p.workspace = workspace;
   p.vis_cnt = vis_cnt;
@@ -1068,17 +1148,14 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const FusedGeometry& 
   p.n_txt = r.N; p.row0 = geo.row0; p.combine = combine ? 1 : 0;
   p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_q = geo.n_q; p.n_k = geo.n_k; p.split = geo.split;
   p.n_buf = geo.n_buf; p.n_slot = geo.n_slot; p.tight = geo.n_slot < 2 * geo.n_buf ? geo.n_slot / 2 : 0;
+  p.early_inputs = (r.inputs_ready && vis_cnt == nullptr) ? 1 : 0;
+  p.wait_cycles = r.wait_cycles > 0 ? r.wait_cycles : kWaitCycles;
   p.scale_log2e = r.scale_log2e;
   p.inv_heads = 1.0f / static_cast<float>(r.H);
 
   FusedKernel kernel = pick_kernel(geo.halves, geo.ach, tail != nullptr);
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem_bytes));
+  cudaError_t e = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), true);
   if (e != cudaSuccess) return e;
-  if (geo.cluster > 8) {
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-    if (e != cudaSuccess) return e;
-  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(r.B * geo.cluster));
   cfg.blockDim = dim3(kThreads);
@@ -1137,16 +1214,38 @@ cudaError_t launch_filter_fused(const mustdrop_plan& plan, const void* q_text, c
   const Resolved& r = plan.r;
   GatherMaps maps = {};
   const uint64_t out_s1 = 256, out_s2 = static_cast<uint64_t>(r.out_rows) * 256, out_s3 = static_cast<uint64_t>(r.H) * out_s2;
-  if (k_out != nullptr &&
-      (!make_gather_map(&maps.k_src, k, r.L, r.H, r.B, static_cast<uint64_t>(r.k_sl) * 2,
-                        static_cast<uint64_t>(r.k_sh) * 2, static_cast<uint64_t>(r.k_sb) * 2) ||
-       !make_gather_map(&maps.k_dst, k_out, r.out_rows, r.H, r.B, out_s1, out_s2, out_s3)))
-    return cudaErrorInvalidValue;
-  if (v_out != nullptr &&
-      (!make_gather_map(&maps.v_src, v, r.L, r.H, r.B, static_cast<uint64_t>(r.v_sl) * 2,
-                        static_cast<uint64_t>(r.v_sh) * 2, static_cast<uint64_t>(r.v_sb) * 2) ||
-       !make_gather_map(&maps.v_dst, v_out, r.out_rows, r.H, r.B, out_s1, out_s2, out_s3)))
-    return cudaErrorInvalidValue;
+  const void* const gk = k_out != nullptr ? k : nullptr;   // the sources matter only where their output is given
+  const void* const gv = v_out != nullptr ? v : nullptr;
+  bool cached = false;
+  if (MapCache* mc = plan.map_cache) {
+    std::lock_guard<std::mutex> lock(mc->mu);
+    for (int x = 0; x < mc->n_gather && !cached; ++x) {
+      const MapCache::GatherEntry& en = mc->gather[x];
+      if (en.k == gk && en.v == gv && en.k_out == k_out && en.v_out == v_out) {
+        maps = en.maps;
+        cached = true;
+      }
+    }
+  }
+  if (!cached) {
+    if (k_out != nullptr &&
+        (!make_gather_map(&maps.k_src, k, r.L, r.H, r.B, static_cast<uint64_t>(r.k_sl) * 2,
+                          static_cast<uint64_t>(r.k_sh) * 2, static_cast<uint64_t>(r.k_sb) * 2) ||
+         !make_gather_map(&maps.k_dst, k_out, r.out_rows, r.H, r.B, out_s1, out_s2, out_s3)))
+      return cudaErrorInvalidValue;
+    if (v_out != nullptr &&
+        (!make_gather_map(&maps.v_src, v, r.L, r.H, r.B, static_cast<uint64_t>(r.v_sl) * 2,
+                          static_cast<uint64_t>(r.v_sh) * 2, static_cast<uint64_t>(r.v_sb) * 2) ||
+         !make_gather_map(&maps.v_dst, v_out, r.out_rows, r.H, r.B, out_s1, out_s2, out_s3)))
+      return cudaErrorInvalidValue;
+    if (MapCache* mc = plan.map_cache) {
+      std::lock_guard<std::mutex> lock(mc->mu);
+      MapCache::GatherEntry& en = mc->gather[mc->next_gather];
+      en.k = gk; en.v = gv; en.k_out = k_out; en.v_out = v_out; en.maps = maps;
+      mc->next_gather = (mc->next_gather + 1) % MapCache::kEntries;
+      if (mc->n_gather < MapCache::kEntries) ++mc->n_gather;
+    }
+  }
   FilterTail t = {};
   t.sel.g = g_out; t.sel.i = i_out; t.sel.key_idx = key_idx; t.sel.key_cnt = key_cnt;
   t.sel.kept_idx = kept_idx; t.sel.kept_cnt = kept_cnt; t.sel.s_out = s_out; t.sel.workspace = workspace;

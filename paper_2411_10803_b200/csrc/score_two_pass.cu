@@ -321,11 +321,9 @@ cudaError_t launch_score_two_pass(const mustdrop_plan& plan, const void* q_text,
   const size_t smem1 = sizeof(__nv_bfloat16) * static_cast<size_t>(n_rows + 2 * kTileKeys) * kRowStride;
   const size_t smem2 = sizeof(__nv_bfloat16) * 2 * static_cast<size_t>(n_rows + kTileKeys) * kRowStride +
                        sizeof(float) * (2 * p.n_warps + 1) * kTileKeys;
-  cudaError_t e = cudaFuncSetAttribute(rowstats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem1));
+  cudaError_t e = ensure_kernel_attributes(reinterpret_cast<const void*>(rowstats_kernel), false);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(accumulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(smem2));
+  e = ensure_kernel_attributes(reinterpret_cast<const void*>(accumulate_kernel), false);
   if (e != cudaSuccess) return e;
   rowstats_kernel<<<dim3(r.H, r.B), threads, smem1, stream>>>(p);
   e = cudaGetLastError();

@@ -43,6 +43,15 @@ __device__ __forceinline__ uint32_t cluster_size() {
 __device__ __forceinline__ void cluster_barrier() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The two halves of the barrier.  Shared memory of another CTA may only be touched once that CTA
+// is known to have started: every kernel arrives in its prologue and waits before its first
+// remote store, so the wait costs nothing unless a peer really is late.
+__device__ __forceinline__ void cluster_arrive() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 // Address of a shared-memory object of this CTA, as seen in CTA `rank` of the cluster.
 __device__ __forceinline__ uint32_t peer_addr(const void* local, uint32_t rank) {
   uint32_t r;
@@ -92,6 +101,8 @@ __global__ void __launch_bounds__(kThreads) spatial_merge_kernel(MergeParams p) 
   const int C = static_cast<int>(cluster_size()), rank = static_cast<int>(cluster_rank());
   const int b = blockIdx.x / C, g = p.grid, gw = g / 2, n_win = gw * gw, n_slot = g * g;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  cluster_arrive();          // "this CTA runs": peers wait for it before their first remote store
+  bool peers_started = false;
   pdl_launch_dependents();
   pdl_wait();
   const uint4* in = p.tokens + static_cast<size_t>(b) * n_slot * p.vecs;
@@ -127,6 +138,10 @@ __global__ void __launch_bounds__(kThreads) spatial_merge_kernel(MergeParams p) 
     n0 = warp_sum(n0); n1 = warp_sum(n1); n2 = warp_sum(n2); n3 = warp_sum(n3);
     d01 = warp_sum(d01); d02 = warp_sum(d02); d03 = warp_sum(d03);
     d12 = warp_sum(d12); d13 = warp_sum(d13); d23 = warp_sum(d23);
+    if (!peers_started) {   // (warp-uniform) every CTA of the cluster has started: its shared memory exists
+      cluster_wait();
+      peers_started = true;
+    }
     if (lane == 0) {
       const float tiny = 1e-30f;
       const float l0 = fmaxf(sqrtf(n0), tiny), l1 = fmaxf(sqrtf(n1), tiny), l2 = fmaxf(sqrtf(n2), tiny),
@@ -139,6 +154,7 @@ __global__ void __launch_bounds__(kThreads) spatial_merge_kernel(MergeParams p) 
       if (p.window_sim != nullptr) p.window_sim[static_cast<size_t>(b) * n_win + w] = sim;
     }
   }
+  if (!peers_started) cluster_wait();   // a warp without a window: complete the prologue's barrier
   cluster_barrier();   // every flag has arrived in every CTA; no remote store after this point
 
   // 2. which slots emit a token (all slots of an unmerged window, the first slot of a merged
@@ -229,6 +245,7 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
   const int C = static_cast<int>(cluster_size()), rank = static_cast<int>(cluster_rank());
   const int b = blockIdx.x / C, M = p.M, dv = p.D / 8;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  cluster_arrive();          // "this CTA runs": peers wait for it before their first remote store
   pdl_launch_dependents();
   pdl_wait();
   for (int j = threadIdx.x; j < M; j += kThreads) a[j] = 0.0f;
@@ -297,6 +314,7 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
     for (int j = threadIdx.x; j < M; j += kThreads) a[j] = fmaf(z[j], f, a[j]);
   }
   // every CTA hands its partial sums to every CTA; each adds them in rank order (same result everywhere)
+  cluster_wait();            // every CTA of the cluster has started: its shared memory exists
   for (int c = 0; c < C; ++c)
     for (int j = threadIdx.x; j < M; j += kThreads)
       asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr(&slab[static_cast<size_t>(rank) * M + j], c)), "f"(a[j])
@@ -434,8 +452,7 @@ extern "C" mustdrop_status_t mustdrop_key_set(int32_t batch, int32_t n_heads, in
   int cluster = 8;
   while (cluster > n_heads) cluster >>= 1;           // 1, 2, 4 or 8 CTAs, at most one per head
   const size_t smem = static_cast<size_t>(cluster) * n_tokens * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(key_set_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(8 * kMaxSlots * sizeof(float)));
+  cudaError_t e = ensure_kernel_attributes(reinterpret_cast<const void*>(key_set_kernel), false);
   if (e != cudaSuccess) return finish(e);
   return finish(launch_cluster(key_set_kernel, batch, cluster, smem, static_cast<cudaStream_t>(cuda_stream), p));
 }

@@ -4,12 +4,43 @@ Rules: importance scores within 2e-3 relative (fp32 accumulation from bf16 input
 indices bit-exact, except that tokens whose oracle scores lie within 1e-3 relative of the
 oracle's cut score may swap; compacted tensors byte-identical.
 """
+import concurrent.futures
+import functools
+import os
+
 import numpy as np
 import torch
+
+import oracle
+from paper_2411_10803_b200 import binding as md
+from paper_2411_10803_b200 import synth
 
 SCORE_RTOL = 2e-3
 SCORE_ATOL = 1e-10
 TIE_RTOL = 1e-3
+
+
+# Debugging overrides of the planner (the debug_* fields of the configuration) that a test's
+# fixtures want in every configuration the test builds.
+DEBUG = {}
+
+VARIANT_CODES = {"two_pass": md.MUSTDROP_DEBUG_VARIANT_TWO_PASS, "fused": md.MUSTDROP_DEBUG_VARIANT_FUSED,
+                 "row_split": md.MUSTDROP_DEBUG_VARIANT_ROW_SPLIT}
+
+
+def force(monkeypatch, variant=None, cluster=None, staged=None):
+    """Force a score kernel variant / a cluster size / the separate launches for the rest of the test."""
+    if variant is not None:
+        monkeypatch.setitem(DEBUG, "debug_score_variant", VARIANT_CODES[variant])
+    if cluster:
+        monkeypatch.setitem(DEBUG, "debug_cluster", int(cluster))
+    if staged is not None:
+        monkeypatch.setitem(DEBUG, "debug_filter_staged", 1 if staged else 0)
+
+
+def cfg(w, **kw):
+    """Configuration of a workload with the test's debugging overrides."""
+    return md.config_for(w, **{**DEBUG, **kw})
 
 
 def to_dev_bf16(bits: np.ndarray) -> torch.Tensor:
@@ -74,3 +105,26 @@ def host_gather(kept_idx, kept_cnt, vis_start, hidden, k, v, fill_h, fill_k, fil
         ko[b, :, :c] = k[b][:, rows]
         vo[b, :, :c] = v[b][:, rows]
     return ho, ko, vo
+
+
+def oracle_scores_all_requests(d, w, per_head=False):
+    """The oracle's G, I for EVERY request of a batch: the plain single-threaded C routine, one call
+    per request, the calls spread over the host's cores (ctypes releases the interpreter lock)."""
+    fn = oracle.score_per_head if per_head else oracle.score
+
+    def one(b):
+        return fn(d["q_text"][b:b + 1], d["k"][b:b + 1], w.vis_start, w.n_vis, w.txt_start)
+
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(32, os.cpu_count() or 1)) as pool:
+        parts = list(pool.map(one, range(w.batch)))
+    return np.concatenate([p[0] for p in parts]), np.concatenate([p[1] for p in parts])
+
+
+@functools.lru_cache(maxsize=1)
+def full_config_reference(name):
+    """Inputs of a named workload and the oracle's scores for all its requests (the workload last
+    asked for is kept: the tests that share it run next to each other)."""
+    w = synth.WORKLOADS[name]
+    d = synth.make_batch(w)
+    G, I = oracle_scores_all_requests(d, w)
+    return w, d, G, I

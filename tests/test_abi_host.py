@@ -63,7 +63,11 @@ def test_valid_plan_and_workspace_size():
     (dict(gamma=-1.0), md.MUSTDROP_ERR_INVALID_ARG),
     (dict(alpha=float("nan")), md.MUSTDROP_ERR_INVALID_ARG),
     (dict(scale=float("inf")), md.MUSTDROP_ERR_INVALID_ARG),
-    (dict(flags=4), md.MUSTDROP_ERR_INVALID_ARG),                 # unknown flag bit
+    (dict(flags=8), md.MUSTDROP_ERR_INVALID_ARG),                 # unknown flag bit
+    (dict(debug_score_variant=4), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(debug_cluster=17), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(debug_filter_staged=2), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(debug_wait_cycles=-1), md.MUSTDROP_ERR_INVALID_ARG),
     (dict(flags=1, seq_len=700), md.MUSTDROP_ERR_INVALID_ARG),    # rebuild needs the text directly behind the image
     (dict(k_stride_l=-8), md.MUSTDROP_ERR_INVALID_ARG),
     (dict(k_stride_l=64), md.MUSTDROP_ERR_INVALID_ARG),           # rows would overlap

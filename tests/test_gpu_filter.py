@@ -9,7 +9,7 @@ from paper_2411_10803_b200 import binding as md
 from paper_2411_10803_b200 import build as md_build
 from paper_2411_10803_b200 import synth
 
-from parity_util import assert_kept_matches, bf16_bits, host_gather, to_dev, to_dev_bf16
+from parity_util import assert_kept_matches, bf16_bits, cfg, force, host_gather, to_dev, to_dev_bf16
 from test_gpu_parity import key_args, run_chain_and_check, small
 
 pytestmark = pytest.mark.gpu
@@ -23,12 +23,7 @@ def _built():
 
 @pytest.fixture
 def cluster(request, monkeypatch):
-    monkeypatch.delenv("MUSTDROP_SCORE_VARIANT", raising=False)
-    monkeypatch.delenv("MUSTDROP_FILTER", raising=False)
-    if request.param:
-        monkeypatch.setenv("MUSTDROP_CLUSTER", str(request.param))
-    else:
-        monkeypatch.delenv("MUSTDROP_CLUSTER", raising=False)
+    force(monkeypatch, cluster=request.param)
     return request.param
 
 
@@ -37,7 +32,7 @@ def test_filter_tiny_reference_config_is_one_launch():
 
 
 def _skip_unless_fused(w):
-    f = md.Filter(md.config_for(w))
+    f = md.Filter(cfg(w))
     fused = f.score_variant == "fused_cluster_tcgen05"
     f.close()
     if not fused:
@@ -59,18 +54,14 @@ def test_filter_fewer_kept_rows_than_ctas(cluster):
     run_chain_and_check(w, path="filter", expect_launches=1)
 
 
-@pytest.mark.parametrize("budget", [192, 64])
-def test_filter_llava7b_batch16(budget):
-    run_chain_and_check(synth.WORKLOADS["c2_llava7b_b16"].with_(budget=budget), sample=[0, 9], path="filter",
-                        expect_launches=1)
-
-
-def test_filter_llava7b_batch64_sampled():
-    run_chain_and_check(synth.WORKLOADS["c2_llava7b_b64"], sample=[0, 31, 63], path="filter", expect_launches=1)
-
-
-def test_filter_13b_batch64_sampled():
-    run_chain_and_check(synth.WORKLOADS["c5_13b_b64"], sample=[17], path="filter", expect_launches=1)
+def test_full_size_plans_are_single_launches():
+    # (every request of these workloads is compared with the oracle, on this path too, by
+    # test_full_config_every_request_matches_oracle)
+    for name, launches in (("c2_llava7b_b16", 1), ("c2_llava7b_b64", 1), ("c3_next7b", 1), ("c5_13b_b64", 1),
+                           ("c4_video", 2)):
+        f = md.Filter(cfg(synth.WORKLOADS[name]))
+        assert f.filter_launches == launches, name
+        f.close()
 
 
 def test_filter_falls_back_to_separate_launches_where_the_fused_geometry_does_not_fit():
@@ -81,16 +72,16 @@ def test_filter_falls_back_to_separate_launches_where_the_fused_geometry_does_no
 
 def test_filter_video_runs_on_a_large_cluster_with_two_statistics_slots(monkeypatch):
     # (the planner prefers the two-pass kernel for this shape: force the fused one)
-    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "fused")
+    force(monkeypatch, variant="fused")
     w = synth.WORKLOADS["c4_video"].with_(batch=2)
-    run_chain_and_check(w, sample=[1], path="filter", expect_launches=1)
+    run_chain_and_check(w, path="filter", expect_launches=1)
 
 
 def test_filter_next7b_runs_on_a_cluster_of_more_than_eight(monkeypatch):
     # 2944 keys per request need more than 8 CTAs x 320 keys: non-portable cluster size, few statistics slots
-    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "fused")
+    force(monkeypatch, variant="fused")
     w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
-    run_chain_and_check(w, sample=[1], path="filter", expect_launches=1)
+    run_chain_and_check(w, path="filter", expect_launches=1)
 
 
 def _run_both(w, monkeypatch, cfg_kw=None, drop=()):
@@ -100,11 +91,8 @@ def _run_both(w, monkeypatch, cfg_kw=None, drop=()):
     ki, kc = key_args(w, d)
     out = []
     for staged in (False, True):
-        if staged:
-            monkeypatch.setenv("MUSTDROP_FILTER", "staged")
-        else:
-            monkeypatch.delenv("MUSTDROP_FILTER", raising=False)
-        f = md.Filter(md.config_for(w, **(cfg_kw or {})))
+        force(monkeypatch, staged=staged)
+        f = md.Filter(cfg(w, **(cfg_kw or {})))
         assert f.filter_launches == (3 if staged else 1)
         f.filter(q, k, None if "v" in drop else v, None if "hidden" in drop else hid, ki, kc, want_s=True)
         torch.cuda.synchronize()
@@ -165,7 +153,7 @@ def test_filter_without_a_key_set_and_keep_all():
 def test_filter_is_deterministic_and_repeatable_on_one_stream():
     w = synth.WORKLOADS["c2_llava7b_b16"].with_(batch=6)
     d = synth.make_batch(w)
-    f = md.Filter(md.config_for(w))
+    f = md.Filter(cfg(w))
     q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
     ki, kc = key_args(w, d)
     f.filter(q, k, v, hid, ki, kc)
@@ -184,10 +172,10 @@ def test_filter_is_deterministic_and_repeatable_on_one_stream():
 
 @pytest.mark.parametrize("n_txt,causal", [(65, 1), (96, 1), (128, 1), (100, 0)])
 def test_row_split_score_and_filter_match_oracle(n_txt, causal, monkeypatch):
-    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "row_split")
+    force(monkeypatch, variant="row_split")
     w = small(batch=3, n_vis=500, n_txt=n_txt, n_heads=3, hidden=384, key_cnt=7, budget=60, vis_start=1)
     d = synth.make_batch(w)
-    f = md.Filter(md.config_for(w, causal=causal))
+    f = md.Filter(cfg(w, causal=causal))
     assert "two launches" in f.description and f.filter_launches == 2
     q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
     ki, kc = key_args(w, d)
@@ -214,6 +202,64 @@ def test_row_split_score_and_filter_match_oracle(n_txt, causal, monkeypatch):
     f.close()
 
 
-def test_video_workload_takes_the_row_split_plan_by_itself():
-    w = synth.WORKLOADS["c4_video"]
-    run_chain_and_check(w, sample=[3], path="filter", expect_launches=2)
+# ---- bounded waits: a wait that runs out is reported, not a hang ---------------------------------
+
+@pytest.mark.parametrize("cluster", [0, 3], indirect=True)
+def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_unaffected(cluster):
+    """The configuration's debug_wait_cycles shortens the waits between the kernel's warp roles to
+    a few cycles, so the first wait for a copy from global memory runs out: the kernel must come
+    back by itself, report MUSTDROP_ERR_TIMEOUT, mark every request invalid (kept_cnt = -1) and
+    leave the device usable - the same step with normal waits, run right behind it on the same
+    stream, gives the oracle's result."""
+    w = small(batch=3, n_vis=333, n_txt=21, n_heads=3, hidden=384, key_cnt=9, budget=40, vis_start=2)
+    d = synth.make_batch(w)
+    q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
+    ki, kc = key_args(w, d)
+    bad = md.Filter(cfg(w, debug_wait_cycles=64))
+    assert bad.filter_launches == 1
+    bad.kept_cnt.fill_(7)
+    bad.filter(q, k, v, hid, ki, kc)
+    good = md.Filter(cfg(w))
+    good.filter(q, k, v, hid, ki, kc, want_s=True)
+    torch.cuda.synchronize()
+    code, _ = bad.device_status()
+    assert code == md.MUSTDROP_ERR_TIMEOUT
+    assert (bad.kept_cnt.cpu().numpy() == -1).all()
+    assert good.device_status() == (0, 0)
+    G, I = oracle.score(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start)
+    ref_idx, ref_cnt, ref_s, _ = oracle.select(G, I, w.seq_len, d["key_idx"], d["key_cnt"], budget=w.budget)
+    idx, cnt = good.kept_idx.cpu().numpy(), good.kept_cnt.cpu().numpy()
+    assert_kept_matches(idx, cnt, ref_idx, ref_cnt, ref_s, d["key_idx"], d["key_cnt"])
+    rh, rk, rv = oracle.compact(idx, cnt, w.vis_start, d["hidden"], d["k"], d["v"])
+    assert np.array_equal(bf16_bits(good.hidden_out), rh) and np.array_equal(bf16_bits(good.k_out), rk)
+    assert np.array_equal(bf16_bits(good.v_out), rv)
+    # the score-only call gives up the same way (status word only: it has no kept_cnt)
+    bad.workspace.zero_()
+    bad.score(q, k)
+    torch.cuda.synchronize()
+    assert bad.device_status()[0] == md.MUSTDROP_ERR_TIMEOUT
+    bad.close()
+    good.close()
+
+
+def test_compact_skips_a_request_marked_invalid():
+    """kept_cnt = -1 (a request whose selection failed) and a count beyond the capacity: nothing is
+    written for the first, the second is clamped; both are recorded; nothing lands outside the outputs."""
+    w = small(batch=3, n_vis=50, n_txt=6, n_heads=2, hidden=256, key_cnt=0, budget=8, vis_start=1)
+    d = synth.make_batch(w)
+    f = md.Filter(cfg(w, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE))
+    kept = np.tile(np.arange(8, dtype=np.int32), (3, 1))
+    cnt = np.array([-1, 8, 99], np.int32)
+    for t in (f.hidden_out, f.k_out, f.v_out):
+        t.fill_(-3.0)                                            # canary value in every output row
+    f.compact(to_dev_bf16(d["hidden"]), to_dev_bf16(d["k"]), to_dev_bf16(d["v"]), to_dev(kept), to_dev(cnt))
+    torch.cuda.synchronize()
+    canary = bf16_bits(torch.full((1,), -3.0, dtype=torch.bfloat16, device="cuda"))[0]
+    ho, ko = bf16_bits(f.hidden_out), bf16_bits(f.k_out)
+    assert (ho[0] == canary).all() and (ko[0] == canary).all()   # the invalid request: untouched
+    rows = np.concatenate([np.arange(1), 1 + kept[1], 1 + 50 + np.arange(6)])
+    for b in (1, 2):                                             # 99 is clamped to the capacity of 8
+        assert np.array_equal(ho[b, :len(rows)], d["hidden"][b, rows])
+        assert np.array_equal(ko[b][:, :len(rows)], d["k"][b][:, rows])
+    assert f.device_status()[0] == md.MUSTDROP_ERR_BAD_KEY_INDEX
+    f.close()

@@ -10,7 +10,7 @@ from paper_2411_10803_b200 import binding as md
 from paper_2411_10803_b200 import build as md_build
 from paper_2411_10803_b200 import synth
 
-from parity_util import assert_kept_matches, assert_scores_close, bf16_bits, to_dev, to_dev_bf16
+from parity_util import assert_kept_matches, assert_scores_close, bf16_bits, cfg, force, to_dev, to_dev_bf16
 
 pytestmark = pytest.mark.gpu
 TINY = synth.WORKLOADS["c1_tiny"]
@@ -26,12 +26,10 @@ def _built():
 
 @pytest.fixture
 def path(request, monkeypatch):
-    for n in ("MUSTDROP_SCORE_VARIANT", "MUSTDROP_CLUSTER", "MUSTDROP_FILTER"):
-        monkeypatch.delenv(n, raising=False)
     if request.param == "three_launches":
-        monkeypatch.setenv("MUSTDROP_FILTER", "staged")
+        force(monkeypatch, staged=True)
     elif request.param == "two_pass":
-        monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "two_pass")
+        force(monkeypatch, variant="two_pass")
     return request.param
 
 
@@ -41,10 +39,9 @@ def small(**kw):
     return TINY.with_(**base)
 
 
-def check_layer(f, w, p, ref, rebuild, sample=None):
-    """Compare one layer's GPU results (in Filter f) with the oracle's dict `ref`; p = the inputs."""
-    sample = range(w.batch) if sample is None else sample
-    sel = np.array(list(sample))
+def check_layer(f, w, p, ref, rebuild):
+    """Compare one layer's GPU results (in Filter f) with the oracle's dict `ref`, every request; p = the inputs."""
+    sel = np.arange(w.batch)
     g, i = f.g.cpu().numpy(), f.i.cpu().numpy()
     idx, cnt = f.kept_idx.cpu().numpy(), f.kept_cnt.cpu().numpy()
     orig = f.orig_out.cpu().numpy()
@@ -81,24 +78,24 @@ def check_layer(f, w, p, ref, rebuild, sample=None):
     return swapped
 
 
-def run_ragged_layer(w, vis_cnt, rebuild, sample=None, with_orig=False):
+def run_ragged_layer(w, vis_cnt, rebuild, with_orig=False):
     d = synth.make_batch(w)
     p = synth.pack_ragged(d, w, vis_cnt)
     if with_orig:
         p["orig_idx"] = (np.arange(w.n_vis, dtype=np.int32)[None, :] * 3 + 1).repeat(w.batch, 0)
-    f = md.Filter(md.config_for(w, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE if rebuild else 0))
+    f = md.Filter(cfg(w, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE if rebuild else 0))
     q, k, v, hid = (to_dev_bf16(p[n]) for n in ("q_text", "k", "v", "hidden"))
     ki, kc = (to_dev(p["key_idx"]), to_dev(p["key_cnt"])) if w.key_cnt else (None, None)
     f.filter_layer(q, k, v, hid, ki, kc, vis_cnt=to_dev(p["vis_cnt"]),
                    orig_idx=to_dev(p["orig_idx"]) if with_orig else None, want_s=True)
     torch.cuda.synchronize()
     assert f.device_status() == (0, 0)
-    sel = list(range(w.batch)) if sample is None else sample
+    sel = list(range(w.batch))
     ref = layers.filter_layer_ragged(p["q_text"][sel], p["k"][sel], p["v"][sel], p["hidden"][sel], w.vis_start,
                                      p["vis_cnt"][sel], w.budget, p["key_idx"][sel] if w.key_cnt else None,
                                      p["key_cnt"][sel] if w.key_cnt else None,
                                      orig_idx=p["orig_idx"][sel] if with_orig else None, rebuild=rebuild)
-    check_layer(f, w, p, ref, rebuild, sel)
+    check_layer(f, w, p, ref, rebuild)
     launches = f.filter_launches
     f.close()
     return launches
@@ -118,9 +115,9 @@ def test_ragged_layer_without_key_set_many_text_rows(path):
     run_ragged_layer(w, np.array([200, 30, 97], np.int32), True)
 
 
-def test_ragged_layer_llava7b_batch16_sampled():
+def test_ragged_layer_llava7b_batch16():
     w = synth.WORKLOADS["c2_llava7b_b16"]
-    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[0, 11]) == 1
+    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True) == 1
 
 
 def test_ragged_layer_long_sequence_falls_back_to_the_two_pass_score():
@@ -129,15 +126,15 @@ def test_ragged_layer_long_sequence_falls_back_to_the_two_pass_score():
 
 
 def test_ragged_layer_video_on_a_large_cluster(monkeypatch):
-    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "fused")
+    force(monkeypatch, variant="fused")
     w = synth.WORKLOADS["c4_video"].with_(batch=2)
-    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[1]) == 1
+    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True) == 1
 
 
 def test_ragged_layer_next7b_on_a_large_cluster(monkeypatch):
-    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "fused")
+    force(monkeypatch, variant="fused")
     w = synth.WORKLOADS["c3_next7b"].with_(batch=2)
-    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True, sample=[1]) == 1
+    assert run_ragged_layer(w, synth.draw_vis_cnt(w), True) == 1
 
 
 @pytest.mark.parametrize("path", ["one_launch", "two_pass"], indirect=True)
@@ -164,7 +161,7 @@ def test_chain_of_three_layers_matches_oracle(path):
     filters, dev = [], []
     for l, (cap, kp) in enumerate(zip(caps, budgets)):
         wl = w.with_(n_vis=cap, budget=kp)
-        filters.append(md.Filter(md.config_for(wl, key_max=5, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE)))
+        filters.append(md.Filter(cfg(wl, key_max=5, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE)))
         dev.append([to_dev_bf16(tensors[l][n]) for n in ("q_text", "k", "v", "hidden")])
     ki, kc, vc, orig = to_dev(key_idx), to_dev(key_cnt), to_dev(vis_cnt0), None
     for l, f in enumerate(filters):
@@ -268,9 +265,7 @@ def test_cache_compact_reports_a_token_the_layer_does_not_hold_and_takes_one_ten
 
 
 def test_ragged_layer_with_text_rows_in_two_launches(monkeypatch):
-    for n in ("MUSTDROP_CLUSTER", "MUSTDROP_FILTER"):
-        monkeypatch.delenv(n, raising=False)
-    monkeypatch.setenv("MUSTDROP_SCORE_VARIANT", "row_split")
+    force(monkeypatch, variant="row_split")
     w = small(batch=3, n_vis=260, n_txt=90, n_heads=2, hidden=256, key_cnt=4, budget=40, vis_start=2)
     assert run_ragged_layer(w, np.array([260, 40, 133], np.int32), True) == 2
 
@@ -282,7 +277,7 @@ def test_ragged_layer_threshold_mode_is_the_printed_rule_on_each_requests_own_si
     d = synth.make_batch(w)
     vis_cnt = np.array([280, 31, 150, 199], np.int32)
     p = synth.pack_ragged(d, w, vis_cnt)
-    f = md.Filter(md.config_for(w, mode=md.MUSTDROP_MODE_THRESHOLD, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE))
+    f = md.Filter(cfg(w, mode=md.MUSTDROP_MODE_THRESHOLD, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE))
     q, k, v, hid = (to_dev_bf16(p[n]) for n in ("q_text", "k", "v", "hidden"))
     f.filter_layer(q, k, v, hid, to_dev(p["key_idx"]), to_dev(p["key_cnt"]), vis_cnt=to_dev(vis_cnt), want_s=True)
     torch.cuda.synchronize()

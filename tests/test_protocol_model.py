@@ -1,0 +1,63 @@
+"""The barrier protocol of the fused score kernel on a host model (threads as warp roles, one
+cluster): it completes for the geometries the planner produces, its slot and buffer counts are
+exactly enough, and a role that skips an arrive ends in a time-out in every CTA - no hang."""
+import pytest
+
+from protocol_model import OK, TIMEOUT, Cluster
+
+GEOMETRIES = [
+    dict(C=1, n_q=2, n_buf=3),
+    dict(C=2, n_q=2, n_buf=3),                       # the 7B batch-64 plan
+    dict(C=4, n_q=4, n_buf=6),
+    dict(C=5, n_q=2, n_buf=3),
+    dict(C=8, n_q=3, n_buf=8),
+    dict(C=10, n_q=2, n_buf=3, n_slot=4, tight=2),   # large clusters: few slots, the exp role held near the add role
+    dict(C=12, n_q=2, n_buf=3, n_slot=2, tight=1),
+]
+
+
+@pytest.mark.parametrize("geo", GEOMETRIES, ids=lambda g: "C%d_q%d_b%d_s%s" % (g["C"], g["n_q"], g["n_buf"], g.get("n_slot", "2b")))
+def test_protocol_completes_and_keeps_its_invariants(geo):
+    cl = Cluster(H=13, limit=5.0, **geo)
+    assert cl.run(), "a role never came back"
+    assert cl.errors == []
+    for c in cl.ctas:
+        assert c.status == OK and c.added == list(range(13))
+    assert cl.kept_cnt == 13
+
+
+@pytest.mark.parametrize("slow", [(0, "add"), (1, "exp"), (0, "tma"), (1, "mma")])
+def test_protocol_tolerates_a_slow_role(slow):
+    # one role of one CTA is much slower than its peers: they run ahead as far as the barriers allow
+    cl = Cluster(C=3, H=10, n_q=2, n_buf=3, limit=5.0, jitter={slow: 0.01})
+    assert cl.run() and cl.errors == []
+    assert all(c.added == list(range(10)) for c in cl.ctas) and cl.kept_cnt == 10
+
+
+def test_fewer_slots_than_the_protocol_needs_is_caught_by_the_model():
+    # 2 x buffers slots are needed without the tight rule: with fewer, a fast peer overwrites an unread pair
+    cl = Cluster(C=2, H=16, n_q=4, n_buf=4, n_slot=4, tight=0, limit=0.3, jitter={(0, "add"): 0.01})
+    cl.run()
+    assert cl.errors and cl.cluster_abort and cl.kept_cnt == -1
+
+
+FAULTS = [
+    (1, "tma", 3, "full"),      # a copy that never completes
+    (0, "mma", 2, "tfull"),     # the MMA role does not hand the logits over
+    (1, "mma", 4, "empty"),     # a stage is never released
+    (0, "exp", 5, "eready"),    # the exponentials are never handed over
+    (1, "exp", 1, "stats"),     # one CTA's statistics never arrive anywhere
+    (0, "add", 3, "tempty"),    # a buffer is never freed
+]
+
+
+@pytest.mark.parametrize("tight", [0, 2])
+@pytest.mark.parametrize("fault", FAULTS, ids=lambda f: "cta%d_%s_h%d_%s" % f)
+def test_a_skipped_arrive_times_out_everywhere(fault, tight):
+    geo = dict(C=3, n_q=2, n_buf=3, n_slot=4, tight=2) if tight else dict(C=2, n_q=2, n_buf=3)
+    cl = Cluster(H=12, limit=0.2, fault=fault, **geo)
+    assert cl.run(join_limit=10.0), "a role hung instead of giving up"
+    assert cl.errors == []                                   # the invariants held up to the give-up
+    assert all(c.status == TIMEOUT for c in cl.ctas)         # every CTA of the cluster reports the time-out
+    assert cl.cluster_abort and cl.kept_cnt == -1            # and the request is marked invalid
+    assert all(len(c.added) < 12 for c in cl.ctas)

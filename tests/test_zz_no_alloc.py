@@ -1,8 +1,10 @@
 """mustdrop_score_static: the score call for callers that cannot allocate device memory
 (an engine whose pool owns the device heap, a plug-in that must not touch its host's
 allocator).  Its scratch is a fixed array inside the library, so it takes no workspace; its
-results must equal those of mustdrop_score.  Checked on two calls in a row, because every
-call reuses the same array and must not depend on what the previous call left there.
+results must equal those of mustdrop_score, and both must agree with the CPU oracle.  Checked
+on two calls in a row, because every call reuses the same array and must not depend on what
+the previous call left there; the device's free memory must read the same before and after
+the second call (the first one may still load the library's code onto the device).
 
 Collected last on purpose: a run that stops at the first failure has then already run every
 other test.
@@ -11,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2411_10803_b200 import binding as md
 from paper_2411_10803_b200 import build as md_build
 from paper_2411_10803_b200 import synth
@@ -37,10 +40,17 @@ def test_static_scratch_score_matches_the_workspace_call_twice_in_a_row():
         g_ref, i_ref = f.score(q, k)
         g = torch.full_like(g_ref, float("nan"))
         i = torch.full_like(i_ref, float("nan"))
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         st = md.mustdrop_score_static(f.plan, q, k, g, i)
         assert st == md.MUSTDROP_OK, md.mustdrop_status_string(st)
         torch.cuda.synchronize()
+        free_after = torch.cuda.mem_get_info()[0]
+        if call > 0:
+            assert free_after == free_before, "the call changed the device's free memory"
         assert _close(g, g_ref) and _close(i, i_ref), "call %d differs from mustdrop_score" % call
+        G, I = oracle.score(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start)
+        assert _close(g, torch.from_numpy(G)) and _close(i, torch.from_numpy(I)), "call %d differs from the oracle" % call
         f.close()
 
 
