@@ -153,7 +153,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   {
     const bool want = c->debug_score_variant != MUSTDROP_DEBUG_VARIANT_AUTO;   // a variant is forced
     const int forced_cluster = c->debug_cluster;
-    const bool allow_fused = c->debug_score_variant != MUSTDROP_DEBUG_VARIANT_TWO_PASS && !r.per_head_max;
+    const bool allow_fused = c->debug_score_variant != MUSTDROP_DEBUG_VARIANT_TWO_PASS;
     const bool force_split = c->debug_score_variant == MUSTDROP_DEBUG_VARIANT_ROW_SPLIT;
     const double k_mb = 256.0e-6 * r.B * r.H * r.L;
     const double two_pass_us = k_mb * (0.6 + 0.7 * r.N / 128.0);   // the two-pass kernel's measured rate
@@ -175,7 +175,9 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
     // keys a CTA can take.  Alternative: two launches over the same keys, text rows 0..63 and the
     // rest, each with the two-tile layout (twice the keys per CTA); the second adds its column
     // sums to / takes the maximum with the first's.  Taken when estimated faster than the above.
-    if (allow_fused && r.N > 64) {
+    // (Not with the per-head reading of Eq. 10: its maxima run over ALL text rows of a head before
+    // the head mean, which two launches over disjoint rows cannot combine afterwards.)
+    if (allow_fused && r.N > 64 && !r.per_head_max) {
       mustdrop::FusedGeometry ga, gb;
       // clusters small enough for both launches to be resident at once, if such a plan exists
       const int fit = p->sm_count / (2 * r.B);

@@ -69,6 +69,7 @@ struct FusedParams {
   int32_t split;
   int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (2 * n_buf, or 4 when tight)
   int32_t tight;                      // d = 1 or 2: the exp warps start head h only when the add warps are done with head h - d (0: no such rule)
+  int32_t per_head;                   // 1: i_out = head mean of the per-head maxima over the text rows (PH instantiations)
   int32_t early_inputs;               // 1: q_text / k may be read before the stream's earlier work has completed (caller's promise)
   long long wait_cycles;              // clock cycles after which a wait between the warp roles gives up
   float scale_log2e, inv_heads;
@@ -267,6 +268,7 @@ struct __align__(8) Barriers {
   uint64_t tempty[kMaxBufs];     // add warps -> MMA: tensor-memory buffer free
   uint64_t sfull[kMaxSlots];    // all CTAs' (max, sum) pairs of a head have arrived
   uint64_t fin;                  // add warps meet before / after staging the head sums
+  uint64_t ph;                   // add warps meet once per head (per-head maxima of Eq. 10)
   uint64_t gfull[kMaxGatherSlots];   // filter tail: a gathered row has landed in its slot
 };
 
@@ -278,7 +280,9 @@ struct GatherMaps {
 // HALVES: 2 = two M=64 tiles per head (N <= 64), 1 = one M=128 tile.
 // ACH: chunks (of 16 columns) an add thread may own; an exp thread owns up to (ACH+1)/2.
 // FILTER: after the scores, the cluster also selects the request's tokens and gathers them.
-template <int HALVES, int ACH, bool FILTER>
+// PH: the other reading of Eq. 10 - per head the column maximum over the text rows, then the head
+//     mean - computed by the add warps from the same normalised probabilities (G is unchanged).
+template <int HALVES, int ACH, bool FILTER, bool PH>
 __global__ void __launch_bounds__(kThreads, 1)
 score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const FusedParams p, const __grid_constant__ GatherMaps gm, const FilterTail ft) {
@@ -320,6 +324,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                                  : static_cast<size_t>(p.n_q) * stage_bytes;
   float2* stats = reinterpret_cast<float2*>(stage_ptr + staging);
   const uint32_t slot_pairs = static_cast<uint32_t>(p.cluster) * NROWS * EPR;   // pairs per slot
+  // PH only: [2][4 add warps][tk] per-head column maxima of each warp's text rows, double-buffered over heads
+  float* const ph_stage = reinterpret_cast<float*>(stats + static_cast<size_t>(p.n_slot) * slot_pairs);
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
@@ -333,6 +339,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     }
     for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), 1);
     mbar_init(smem_u32(&bars.fin), kAddThreads);
+    mbar_init(smem_u32(&bars.ph), kAddThreads);
     for (int s = 0; s < kMaxGatherSlots; ++s) mbar_init(smem_u32(&bars.gfull[s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -708,6 +715,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     for (int c = 0; c < ACH; ++c)
 #pragma unroll
       for (int j = 0; j < kChunk; ++j) acc[c][j] = 0.0f;
+    // PH: this thread's keys tid_a, tid_a + 128, ... of the CTA: running sum over heads of the per-head maxima
+    constexpr int PHK = (ACH * kChunk * HALVES + kAddThreads - 1) / kAddThreads;
+    float ph_acc[PHK];
+#pragma unroll
+    for (int x = 0; x < PHK; ++x) ph_acc[x] = 0.0f;
+    const unsigned grp_mask = (HALVES == 2) ? (half ? 0xffff0000u : 0x0000ffffu) : 0xffffffffu;   // lanes sharing a key range
+    const bool real_row = row < p.N;     // lanes beyond the text rows carry padding
 
     int h = 0;
     for (; h < p.H; ++h) {
@@ -753,6 +767,37 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 #pragma unroll
             for (int j = 0; j < kChunk; ++j) acc[c0 + 1][j] = fmaf(e[1][j], f1, acc[c0 + 1][j]);
           }
+          if constexpr (PH) {
+            // column maxima over this warp's text rows: probabilities are >= 0, so their bit
+            // patterns order like unsigned integers and one warp reduction per column does it;
+            // lane j of the group keeps column j's result and stores it for the other warps
+            float* const dst = ph_stage + ((h & 1) * kAddWarps + q) * p.tk + half * p.cpl + (lane & 15);
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+              if (c0 + x < ACH && c0 + x < total_chunks) {
+                const float fx = real_row ? (x ? f1 : f0) : 0.0f;
+                unsigned mine = 0u;
+#pragma unroll
+                for (int j = 0; j < kChunk; ++j) {
+                  const unsigned m = __reduce_max_sync(grp_mask, __float_as_uint(e[x][j] * fx));
+                  mine = ((lane & 15) == j) ? m : mine;
+                }
+                if (HALVES == 2 || lane < 16) dst[kChunk * (c0 + x)] = __uint_as_float(mine);
+              }
+            }
+          }
+        }
+      }
+      if constexpr (PH) {
+        // the four warps' maxima of this head meet; each thread adds the maximum of its keys
+        mbar_arrive(smem_u32(&bars.ph));
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.ph), static_cast<uint32_t>(h) & 1u, abort_flag, wait_limit))) break;
+        const float* const src = ph_stage + (h & 1) * kAddWarps * p.tk;
+#pragma unroll
+        for (int x = 0; x < PHK; ++x) {
+          const int key = tid_a + x * kAddThreads;
+          if (key < p.tk)
+            ph_acc[x] += fmaxf(fmaxf(src[key], src[p.tk + key]), fmaxf(src[2 * p.tk + key], src[3 * p.tk + key]));
         }
       }
       tc_fence_before();
@@ -780,7 +825,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       mbar_arrive(smem_u32(&bars.fin));
       const bool staged = mbar_wait(smem_u32(&bars.fin), 1u, abort_flag, wait_limit);
       pdl_wait();
-      for (int c = tid_a; staged && c < p.tk; c += kAddThreads) {
+      for (int c = tid_a, x = 0; staged && c < p.tk; c += kAddThreads, ++x) {
         const int j = static_cast<int>(rank) * p.tk + c - p.vis_start;   // vision-relative index
         if (j < 0 || j >= p.M) continue;
         float s = 0.0f, mx = -INFINITY;
@@ -788,6 +833,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           const float v = mat[r * ld + c];
           s += v;
           mx = fmaxf(mx, v);
+        }
+        if constexpr (PH) {
+          mx = 0.0f;   // (x < PHK always; a compile-time unrolled pick keeps ph_acc in registers)
+#pragma unroll
+          for (int y = 0; y < PHK; ++y) mx = (y == x) ? ph_acc[y] : mx;
         }
         const bool present = j < Mb;    // beyond the request's own tokens: zeros
         float gv = present ? s * p.inv_heads : 0.0f, iv = present ? mx * p.inv_heads : 0.0f;
@@ -957,18 +1007,21 @@ namespace {
 
 using FusedKernel = void (*)(const CUtensorMap, const CUtensorMap, const FusedParams, const GatherMaps, const FilterTail);
 
-FusedKernel pick_kernel(int halves, int ach, bool filter = false) {
-  if (filter)
-    return halves == 2 ? (ach > 5 ? score_fused_kernel<2, 10, true> : score_fused_kernel<2, 5, true>)
-                       : (ach > 5 ? score_fused_kernel<1, 10, true> : score_fused_kernel<1, 5, true>);
-  return halves == 2 ? (ach > 5 ? score_fused_kernel<2, 10, false> : score_fused_kernel<2, 5, false>)
-                     : (ach > 5 ? score_fused_kernel<1, 10, false> : score_fused_kernel<1, 5, false>);
+template <bool FILTER, bool PH>
+FusedKernel pick_shape(int halves, int ach) {
+  return halves == 2 ? (ach > 5 ? score_fused_kernel<2, 10, FILTER, PH> : score_fused_kernel<2, 5, FILTER, PH>)
+                     : (ach > 5 ? score_fused_kernel<1, 10, FILTER, PH> : score_fused_kernel<1, 5, FILTER, PH>);
+}
+
+FusedKernel pick_kernel(int halves, int ach, bool filter = false, bool per_head = false) {
+  if (filter) return per_head ? pick_shape<true, true>(halves, ach) : pick_shape<true, false>(halves, ach);
+  return per_head ? pick_shape<false, true>(halves, ach) : pick_shape<false, false>(halves, ach);
 }
 
 // Clusters of `cluster` CTAs that can be resident at once (GPC boundaries make this less than
 // SMs / cluster); 0 when it cannot be asked (no device) or the shape cannot launch.
-int max_resident_clusters(int halves, int ach, int cluster, size_t smem_bytes) {
-  FusedKernel kernel = pick_kernel(halves, ach);
+int max_resident_clusters(int halves, int ach, int cluster, size_t smem_bytes, bool per_head) {
+  FusedKernel kernel = pick_kernel(halves, ach, false, per_head);
   if (ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), true) != cudaSuccess) {
     (void)cudaGetLastError();
     return 0;
@@ -1024,7 +1077,9 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     // those the split layout (two query tiles + a ring of key half-tiles, which needs less
     // memory for the same look-ahead) is tried as well and taken when it allows a wider window.
     const size_t q_tile = static_cast<size_t>(nrows) * 256, k_half = static_cast<size_t>(cpl) * 256;
-    const size_t avail = 227 * 1024 - 4096 /* static */ - 1024 /* alignment */;
+    // the per-head reading of Eq. 10 stages each add warp's column maxima: 2 heads x 4 warps x tk floats
+    const size_t ph_bytes = r.per_head_max ? static_cast<size_t>(2 * kAddWarps) * tk * sizeof(float) : 0;
+    const size_t avail = 227 * 1024 - 4096 /* static */ - 1024 /* alignment */ - ph_bytes;
     auto slots_bytes = [&](int n_slot) { return static_cast<size_t>(n_slot) * c * nrows * epr * 8; };
     int n_buf = kTmemCols / cpl;
     if (n_buf > kMaxBufs) n_buf = kMaxBufs;
@@ -1068,10 +1123,10 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     // Cost model (microseconds per head and CTA): streaming the stage at ~45 GB/s per SM, or the
     // MMA -> exp -> exchange -> add chain (~4.5 us) spread over the buffers, whichever is longer;
     // times the number of waves of CTAs.
-    size_t smem_bytes = (split ? n_q * q_tile + n_k * k_half : n_q * stage) + 1024 + extra;
+    size_t smem_bytes = (split ? n_q * q_tile + n_k * k_half : n_q * stage) + 1024 + extra + ph_bytes;
     // at least 116 KB, so that two CTAs (each wanting all of tensor memory) never share an SM
     if (smem_bytes < 116 * 1024) smem_bytes = 116 * 1024;
-    int resident = max_resident_clusters(halves, ach, c, smem_bytes);
+    int resident = max_resident_clusters(halves, ach, c, smem_bytes, r.per_head_max != 0);
     if (resident <= 0 && c <= 8) resident = sm_count / c;    // no device to ask: ignore GPC boundaries
     // (a cluster of more than 8 CTAs is used only where the device says it can hold one)
     if (resident <= 0) continue;
@@ -1148,12 +1203,13 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const FusedGeometry& 
   p.n_txt = r.N; p.row0 = geo.row0; p.combine = combine ? 1 : 0;
   p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_q = geo.n_q; p.n_k = geo.n_k; p.split = geo.split;
   p.n_buf = geo.n_buf; p.n_slot = geo.n_slot; p.tight = geo.n_slot < 2 * geo.n_buf ? geo.n_slot / 2 : 0;
+  p.per_head = r.per_head_max;
   p.early_inputs = (r.inputs_ready && vis_cnt == nullptr) ? 1 : 0;
   p.wait_cycles = r.wait_cycles > 0 ? r.wait_cycles : kWaitCycles;
   p.scale_log2e = r.scale_log2e;
   p.inv_heads = 1.0f / static_cast<float>(r.H);
 
-  FusedKernel kernel = pick_kernel(geo.halves, geo.ach, tail != nullptr);
+  FusedKernel kernel = pick_kernel(geo.halves, geo.ach, tail != nullptr, r.per_head_max != 0);
   cudaError_t e = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), true);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};

@@ -376,22 +376,50 @@ def test_chain_is_deterministic():
 
 # ---- the per-head reading of Eq. 10 (MUSTDROP_FLAG_PER_HEAD_MAX) ------------------------------------
 
+@pytest.mark.parametrize("variant", VARIANTS, indirect=True)
 @pytest.mark.parametrize("causal", [1, 0])
 @pytest.mark.parametrize("kw", [dict(), dict(batch=3, n_vis=333, n_txt=21, n_heads=5, hidden=640, vis_start=2),
-                                dict(batch=2, n_vis=130, n_txt=100, n_heads=2, hidden=256)])
-def test_score_per_head_max_matches_oracle(kw, causal):
+                                dict(batch=2, n_vis=130, n_txt=100, n_heads=2, hidden=256),
+                                dict(batch=2, n_vis=700, n_txt=64, n_heads=4, hidden=512)])
+def test_score_per_head_max_matches_oracle(kw, causal, variant):
     w = small(**kw)
     d = synth.make_batch(w, with_values=False)
     f = md.Filter(cfg(w, causal=causal, flags=md.MUSTDROP_FLAG_PER_HEAD_MAX))
-    assert f.score_variant == "two_pass_mma"
+    check_variant(f, variant)
+    if variant == "auto":
+        assert f.score_variant == "fused_cluster_tcgen05"      # the flag runs on the one-pass kernel
     f.score(to_dev_bf16(d["q_text"]), to_dev_bf16(d["k"]))
     torch.cuda.synchronize()
+    assert f.device_status() == (0, 0)
     G, I = oracle.score_per_head(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start, causal=bool(causal))
     assert_scores_close(f.g.cpu().numpy(), G, "G")
     assert_scores_close(f.i.cpu().numpy(), I, "I (per head)")
     # and it is not the other reading
     _, I_mean_first = oracle.score(d["q_text"], d["k"], w.vis_start, w.n_vis, w.txt_start, causal=bool(causal))
-    assert np.any(np.abs(f.i.cpu().numpy() - I_mean_first) > 1e-2 * I_mean_first)
+    if w.n_heads > 1:
+        assert np.any(np.abs(f.i.cpu().numpy() - I_mean_first) > 1e-2 * I_mean_first)
+    f.close()
+
+
+def test_per_head_max_at_the_batch64_shape_runs_the_one_launch_filter():
+    w = synth.WORKLOADS["c2_llava7b_b64"].with_(batch=8)
+    d = synth.make_batch(w)
+    f = md.Filter(cfg(w, flags=md.MUSTDROP_FLAG_PER_HEAD_MAX))
+    assert f.score_variant == "fused_cluster_tcgen05" and f.filter_launches == 1
+    q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
+    ki, kc = key_args(w, d)
+    f.filter(q, k, v, hid, ki, kc, want_s=True)
+    torch.cuda.synchronize()
+    assert f.device_status() == (0, 0)
+    G, I = oracle_scores_all_requests(d, w, per_head=True)
+    assert_scores_close(f.g.cpu().numpy(), G, "G")
+    assert_scores_close(f.i.cpu().numpy(), I, "I (per head)")
+    ref_idx, ref_cnt, ref_s, _ = oracle.select(G, I, w.seq_len, d["key_idx"], d["key_cnt"], budget=w.budget)
+    idx, cnt = f.kept_idx.cpu().numpy(), f.kept_cnt.cpu().numpy()
+    assert_kept_matches(idx, cnt, ref_idx, ref_cnt, ref_s, d["key_idx"], d["key_cnt"])
+    rh, rk, rv = oracle.compact(idx, cnt, w.vis_start, d["hidden"], d["k"], d["v"])
+    assert np.array_equal(bf16_bits(f.hidden_out), rh) and np.array_equal(bf16_bits(f.k_out), rk)
+    assert np.array_equal(bf16_bits(f.v_out), rv)
     f.close()
 
 
