@@ -159,6 +159,12 @@ def test_plan_description_names_the_geometry_without_a_gpu():
     md.mustdrop_plan_destroy(plan)
     st, plan, _ = md.mustdrop_filter_plan(md.config_for(synth.WORKLOADS["c2_llava7b_b64"],
                                                         flags=md.MUSTDROP_FLAG_PER_HEAD_MAX))
+    # the per-head reading of Eq. 10 runs on the same one-launch kernel
+    assert st == md.MUSTDROP_OK and md.mustdrop_plan_score_variant(plan) == "fused_cluster_tcgen05"
+    assert md.mustdrop_plan_filter_launches(plan) == 1
+    md.mustdrop_plan_destroy(plan)
+    st, plan, _ = md.mustdrop_filter_plan(md.config_for(synth.WORKLOADS["c2_llava7b_b64"],
+                                                        debug_score_variant=md.MUSTDROP_DEBUG_VARIANT_TWO_PASS))
     assert st == md.MUSTDROP_OK and md.mustdrop_plan_score_variant(plan) == "two_pass_mma"
     assert md.mustdrop_plan_filter_launches(plan) == 4
     md.mustdrop_plan_destroy(plan)
