@@ -309,6 +309,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const uint32_t rank = cluster_cta_rank();
   const int b = blockIdx.x / p.cluster;
   MD_PIPE(p.workspace, 0, false, true);
+  if (threadIdx.x == 0) MD_TRACE(0, 8);    // (CTA-level stamps use the event slots 8.. of head 0) kernel entry
   // dynamic shared memory: [n_q query tiles][n_k key half-tiles][stats: n_slot x cluster x NROWS x EPR float2]
   // A tile is two slabs of 64 elements (128 bytes per row, 128-byte swizzle), rows contiguous per slab.
   // Two layouts of the staging area: whole stages (a head's query tile and all its keys, n_q of
@@ -357,6 +358,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   // global data; the copy thread waits for the stream's earlier work before its first load (its
   // inputs may come from the kernel just before this one), the other roles before their stores.
   pdl_launch_dependents();
+  if (threadIdx.x == 0) MD_TRACE(0, 9);    // prologue done
   const uint32_t tmem_base = tmem_base_holder;
   // This request's own sequence.  In a ragged batch the token count comes from an earlier
   // kernel in the stream (the previous layer's selection), so it is read after the wait.
@@ -387,6 +389,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
     cluster_sync_all();   // (release / acquire: a peer's flag store above is visible behind it)
+    if (threadIdx.x == 0) MD_TRACE(0, 11);   // score part left
     MD_PIPE(p.workspace, 0, true, false);
   };
   // After common_exit: did any CTA of the cluster give up?  (Stable by then: same answer in every thread.)
@@ -612,6 +615,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
       const uint32_t slot_addr = smem_u32(&stats[slot * slot_pairs + pair_idx]);
       const uint32_t bar_addr = smem_u32(&bars.sfull[slot]);
+#ifdef MUSTDROP_EXP_BATCHED
       // All of this thread's logits of the head are loaded at once; while they are in flight the
       // previous head is handed to the add warps (its exponentials have been stored by now).
       float z[ECH][kChunk];
@@ -659,6 +663,78 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         }
       float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
       if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
+#else
+      // The thread's chunks stream through two register sets: while chunk t is worked on, chunk
+      // t + 1 is already on its way from tensor memory, and the exponentials of chunk t - 1 are on
+      // their way back.  The stabiliser is the maximum of the thread's FIRST chunk (shared by the two
+      // lanes of a row): any value within a few dozen powers of two of the row maximum serves, because
+      // every CTA sends the stabiliser it used along with its sum.  Should a later chunk exceed it
+      // by more than 2^kRescale (extreme logits), the warp rescales what it has already stored.
+      constexpr float kRescale = 32.0f;
+      float z[2][kChunk];
+      tc_ld16(tbuf + kChunk * chunk_of(0), z[0]);
+      if (last_buf >= 0 && !p.tight) {   // the head this warp worked on before: hand it to the add warps
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[last_buf]));
+      }
+      float mx = -INFINITY, sub = 0.0f;
+      float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+      for (int t = 0; t < ECH; ++t) {
+        if (t < my_chunks) {   // (warp-uniform)
+          tc_wait_ld();
+          if (t + 1 < ECH && t + 1 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 1), z[(t + 1) & 1]);
+          float(&zc)[kChunk] = z[t & 1];
+          if (!all_visible) {
+            const int nvis = lim - kChunk * chunk_of(t);   // visible columns of this chunk
+            if (nvis < kChunk) {
+#pragma unroll
+              for (int j = 0; j < kChunk; ++j) zc[j] = (j < nvis) ? zc[j] : -INFINITY;
+            }
+          }
+          float c4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) c4[j & 3] = fmaxf(c4[j & 3], zc[j]);
+          const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3])) * p.scale_log2e;   // scale > 0 keeps the order
+          if (t == 0) {
+            mx = cm;
+            if (HALVES == 2) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));   // one stabiliser per row
+            sub = (mx == -INFINITY) ? 0.0f : mx;   // (first chunk all masked: so are the later ones)
+          } else if (__any_sync(0xffffffffu, cm - sub > kRescale)) {
+            // rare: move the stabiliser up and rescale the chunks already stored (all lanes take part:
+            // the tensor-memory instructions are warp-wide; lanes whose stabiliser stays multiply by 1)
+            float up = fmaxf(mx, cm);
+            if (HALVES == 2) up = fmaxf(up, __shfl_xor_sync(0xffffffffu, up, 16));
+            const float fac = (up == mx) ? 1.0f : ex2(sub - up);
+            tc_wait_st();
+#pragma unroll
+            for (int u = 0; u < t; ++u) {
+              float old[kChunk];
+              tc_ld16(tbuf + kChunk * chunk_of(u), old);
+              tc_wait_ld();
+#pragma unroll
+              for (int j = 0; j < kChunk; ++j) old[j] *= fac;
+              tc_st16(tbuf + kChunk * chunk_of(u), old);
+            }
+#pragma unroll
+            for (int x = 0; x < 4; ++x) ls4[x] *= fac;
+            mx = up;
+            sub = up;
+          }
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) {
+            const float e = ex2(fmaf(zc[j], p.scale_log2e, -sub));
+            zc[j] = e;
+            ls4[j & 3] += e;
+          }
+          tc_st16(tbuf + kChunk * chunk_of(t), zc);
+        }
+      }
+      float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+      if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
+#endif
       if (sender) {
         for (int c = 0; c < p.cluster; ++c)
           st_async_f32x2(map_to_cta(slot_addr, c), mx, lsum, map_to_cta(bar_addr, c));
@@ -697,6 +773,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       else if (own <= 4) select_request<4, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
       else if (own <= 8) select_request<8, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
       else select_request<16, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      if (threadIdx.x == 0) MD_TRACE(0, 12);   // selection done
       cta_sync();   // the list is complete: the copy thread may start
       return;
     }
@@ -848,6 +925,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         p.g_out[static_cast<size_t>(b) * p.M + j] = gv;
         p.i_out[static_cast<size_t>(b) * p.M + j] = iv;
       }
+      if (tid_a == 0) MD_TRACE(0, 10);     // scores stored
     }
     if constexpr (FILTER) {
       // filter tail, add warps: row r of the compacted outputs is copied by CTA r mod cluster
@@ -931,6 +1009,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           }
         }
         bulk_wait_all();   // the stores have been written before the CTA (and its shared memory) goes away
+        MD_TRACE(0, 13);   // gather done
       }
       return;
     }

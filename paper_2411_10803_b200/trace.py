@@ -6,6 +6,9 @@ first 4096 bytes.  Runs the score call on a synthetic workload and prints, for a
 each stage of each head happened and the mean duration of the stages.
 
     python -m paper_2411_10803_b200.trace [workload]        # default c2_llava7b_b16
+    python -m paper_2411_10803_b200.trace [workload] filter # the one-launch filter call: also the
+                                                            # CTA-level stamps (entry, prologue,
+                                                            # scores stored, selection, gather)
 """
 from __future__ import annotations
 
@@ -23,6 +26,7 @@ from . import build as md_build
 from . import synth
 
 EVENTS = ["tma_issue", "mma_full", "mma_tempty", "exp_start", "exp_done", "add_sfull", "add_eready", "add_done"]
+CTA_EVENTS = ["entry", "prologue_done", "scores_stored", "score_part_left", "selection_done", "gather_done"]   # slots 8.. of head 0
 
 
 def build_trace_library(out_dir: str) -> str:
@@ -39,13 +43,15 @@ def main(argv) -> int:
     if not torch.cuda.is_available():
         raise RuntimeError("the trace needs a CUDA device")
     w = synth.WORKLOADS[argv[1] if len(argv) > 1 else "c2_llava7b_b16"]
+    whole = len(argv) > 2 and argv[2] == "filter"
     with tempfile.TemporaryDirectory() as tmp:
         L = ctypes.CDLL(build_trace_library(tmp))
         vp = ctypes.c_void_p
         L.mustdrop_filter_plan.argtypes = [ctypes.c_void_p, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
         L.mustdrop_score.argtypes = [vp] * 7
+        L.mustdrop_filter.argtypes = [vp] * 17
         L.mustdrop_plan_describe.argtypes = [vp, ctypes.c_char_p, ctypes.c_size_t]
-        host = synth.make_batch(w, with_values=False)
+        host = synth.make_batch(w, with_values=whole)
         q = torch.from_numpy(host["q_text"].view(np.int16)).cuda()
         k = torch.from_numpy(host["k"].view(np.int16)).cuda()
         g = torch.empty((w.batch, w.n_vis), dtype=torch.float32, device="cuda")
@@ -60,8 +66,25 @@ def main(argv) -> int:
         n_cta = w.batch * 16
         ws = torch.zeros(4096 + n_cta * w.n_heads * 16 * 8, dtype=torch.uint8, device="cuda")
         stream = torch.cuda.current_stream().cuda_stream
+        if whole:
+            v = torch.from_numpy(host["v"].view(np.int16)).cuda()
+            hid = torch.from_numpy(host["hidden"].view(np.int16)).cuda()
+            ki, kc = torch.from_numpy(host["key_idx"]).cuda(), torch.from_numpy(host["key_cnt"]).cuda()
+            kept = torch.zeros((w.batch, w.budget), dtype=torch.int32, device="cuda")
+            cnt = torch.zeros((w.batch,), dtype=torch.int32, device="cuda")
+            ho = torch.zeros((w.batch, w.budget, w.hidden), dtype=torch.int16, device="cuda")
+            ko = torch.zeros((w.batch, w.n_heads, w.budget, 128), dtype=torch.int16, device="cuda")
+            vo = torch.zeros_like(ko)
         for _ in range(3):
-            L.mustdrop_score(plan, q.data_ptr(), k.data_ptr(), g.data_ptr(), i.data_ptr(), ws.data_ptr(), stream)
+            if whole:
+                st = L.mustdrop_filter(plan, q.data_ptr(), k.data_ptr(), v.data_ptr(), hid.data_ptr(),
+                                       ki.data_ptr() if w.key_cnt else None, kc.data_ptr() if w.key_cnt else None,
+                                       g.data_ptr(), i.data_ptr(), None, kept.data_ptr(), cnt.data_ptr(), ho.data_ptr(),
+                                       ko.data_ptr(), vo.data_ptr(), ws.data_ptr(), stream)
+            else:
+                st = L.mustdrop_score(plan, q.data_ptr(), k.data_ptr(), g.data_ptr(), i.data_ptr(), ws.data_ptr(), stream)
+            if st != 0:
+                raise RuntimeError("call refused: %d" % st)
             torch.cuda.synchronize()
         t = ws[4096:].cpu().numpy().view(np.uint64).reshape(n_cta, w.n_heads, 16).astype(np.float64)
     used = [c for c in range(n_cta) if t[c, 0, 0] > 0]
@@ -69,6 +92,18 @@ def main(argv) -> int:
         print("no stamps: the plan does not use the fused kernel")
         return 1
     print("CTAs with stamps:", len(used), "(stamps of even heads only where the exp warps alternate heads)")
+    # CTA-level phases, relative to the earliest kernel entry of the grid
+    entry0 = min(t[c, 0, 8] for c in used)
+    names = CTA_EVENTS if whole else CTA_EVENTS[:4]
+    rel = np.array([[(t[c, 0, 8 + e] - entry0) / 1e3 for e in range(len(names))] for c in used])
+    first_tma = np.array([(t[c, 0, 0] - entry0) / 1e3 for c in used])
+    first_full = np.array([(t[c, 0, 1] - entry0) / 1e3 for c in used])
+    last_add = np.array([(t[c, (w.n_heads - 1) // 2 * 2, 7] - entry0) / 1e3 for c in used])
+    print("phases (us after the first CTA's entry; min / median / max over CTAs):")
+    for n, col in [(names[0], rel[:, 0]), (names[1], rel[:, 1]), ("first_tma_issue", first_tma), ("first_stage_full", first_full),
+                   ("last_even_head_added", last_add)] + [(names[e], rel[:, e]) for e in range(2, len(names))]:
+        col = col[col > -1e6]
+        print("  %-22s %8.2f %8.2f %8.2f" % (n, col.min(), np.median(col), col.max()))
     for c in used[:2] + used[-1:]:
         t0 = t[c, 0, 0]
         print("CTA", c)

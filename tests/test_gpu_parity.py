@@ -140,6 +140,37 @@ def test_score_extreme_logits_do_not_overflow(variant):
     f.close()
 
 
+@pytest.mark.parametrize("variant", ["auto", "fused:1", "fused:2", "fused:5", "fused:12"], indirect=True)
+@pytest.mark.parametrize("n_txt", [20, 100])
+def test_score_with_logits_that_grow_along_the_keys(n_txt, variant):
+    """Later keys carry ever larger logits, so the stabiliser an exp warp takes from the first
+    columns it sees falls short by far more than 2^32 and the already stored exponentials have to
+    be rescaled (several times per row)."""
+    w = small(batch=2, n_vis=700, n_txt=n_txt, n_heads=2, hidden=256, n_salient=0)
+    d = synth.make_batch(w, with_values=False)
+    q = synth.bf16_bits_to_f32(d["q_text"])
+    k = synth.bf16_bits_to_f32(d["k"])
+    u = q.mean(axis=2, keepdims=True)                                    # [B,H,1,D] mean text query
+    u /= np.linalg.norm(u, axis=-1, keepdims=True)
+    ramp = np.linspace(0.0, 180.0, w.seq_len, dtype=np.float32)[None, None, :, None]
+    k = k + ramp * u * np.sqrt(128.0) / np.maximum(np.linalg.norm(q, axis=-1).mean(), 1e-6) * 3.0
+    qb, kb = synth.f32_to_bf16_bits(q), synth.f32_to_bf16_bits(k.astype(np.float32))
+    G, I = oracle.score(qb, kb, w.vis_start, w.n_vis, w.txt_start)
+    f = md.Filter(cfg(w))
+    check_variant(f, variant)
+    g, i = f.score(to_dev_bf16(qb), to_dev_bf16(kb))
+    torch.cuda.synchronize()
+    g, i = g.cpu().numpy(), i.cpu().numpy()
+    assert f.device_status() == (0, 0)
+    assert np.isfinite(g).all() and np.isfinite(i).all()
+    big = G > 1e-12
+    assert big.sum() > 10
+    assert_scores_close(g[big], G[big], "G")
+    assert_scores_close(i[big], I[big], "I")
+    assert (g[~big] <= 1e-9).all()
+    f.close()
+
+
 # ---- select ----------------------------------------------------------------------------------
 
 def _random_scores(seed, B, M, N=9):
