@@ -254,9 +254,33 @@ __device__ __forceinline__ void trace_stamp(void* workspace, int n_heads, int h,
       [(static_cast<size_t>(blockIdx.x) * n_heads + h) * 16 + ev] = t;
 }
 #define MD_TRACE(h, ev) trace_stamp(p.workspace, p.H, (h), (ev))
+// SM clock instead of the global timer (finer; only differences within one thread mean anything):
+// thread 0's progress through the exp stage of a head, in the event slots 8.. of heads >= 1
+#define MD_TRACE_CLK(h, ev)                                                                          \
+  do {                                                                                               \
+    if (threadIdx.x == 0 && (h) > 0)                                                                 \
+      reinterpret_cast<long long*>(static_cast<unsigned char*>(p.workspace) + 4096)                  \
+          [(static_cast<size_t>(blockIdx.x) * p.H + (h)) * 16 + (ev)] = clock64();                   \
+  } while (0)
 #else
 #define MD_TRACE(h, ev) ((void)0)
+#define MD_TRACE_CLK(h, ev) ((void)0)
 #endif
+
+// Rare path of the exp warps (kept out of line so that the hot loop stays small): the `count`
+// chunks already stored at first, first + stride, ... are multiplied by this lane's factor.
+// Called by all lanes of a warp together.
+__device__ __noinline__ void rescale_stored(uint32_t first, uint32_t stride, int count, float fac) {
+  tc_wait_st();
+  for (int u = 0; u < count; ++u) {
+    float old[kChunk];
+    tc_ld16(first + stride * u, old);
+    tc_wait_ld();
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) old[j] *= fac;
+    tc_st16(first + stride * u, old);
+  }
+}
 
 struct __align__(8) Barriers {
   uint64_t qfull[kMaxQBufs];     // TMA -> MMA: query tile of a head has landed
@@ -615,64 +639,19 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
       const uint32_t slot_addr = smem_u32(&stats[slot * slot_pairs + pair_idx]);
       const uint32_t bar_addr = smem_u32(&bars.sfull[slot]);
-#ifdef MUSTDROP_EXP_BATCHED
-      // All of this thread's logits of the head are loaded at once; while they are in flight the
-      // previous head is handed to the add warps (its exponentials have been stored by now).
-      float z[ECH][kChunk];
-#pragma unroll
-      for (int t = 0; t < ECH; ++t)
-        if (t < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t), z[t]);
-      if (last_buf >= 0 && !p.tight) {   // the head this warp worked on before
-        tc_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[last_buf]));
-      }
-      tc_wait_ld();
-      if (!all_visible) {
-#pragma unroll
-        for (int t = 0; t < ECH; ++t) {
-          const int nvis = lim - kChunk * chunk_of(t);   // visible columns of this chunk
-          if (nvis < kChunk) {
-#pragma unroll
-            for (int j = 0; j < kChunk; ++j) z[t][j] = (j < nvis) ? z[t][j] : -INFINITY;
-          }
-        }
-      }
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-      for (int t = 0; t < ECH; ++t)
-        if (t < my_chunks) {
-#pragma unroll
-          for (int j = 0; j < kChunk; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], z[t][j]);
-        }
-      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;   // scale > 0 keeps the order
-      if (HALVES == 2) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));            // one stabiliser per row
-      const float sub = (mx == -INFINITY) ? 0.0f : mx;
-      float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-      for (int t = 0; t < ECH; ++t)
-        if (t < my_chunks) {
-#pragma unroll
-          for (int j = 0; j < kChunk; ++j) {
-            const float e = ex2(fmaf(z[t][j], p.scale_log2e, -sub));
-            z[t][j] = e;
-            ls4[j & 3] += e;
-          }
-          tc_st16(tbuf + kChunk * chunk_of(t), z[t]);
-        }
-      float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-      if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
-#else
       // The thread's chunks stream through two register sets: while chunk t is worked on, chunk
       // t + 1 is already on its way from tensor memory, and the exponentials of chunk t - 1 are on
       // their way back.  The stabiliser is the maximum of the thread's FIRST chunk (shared by the two
       // lanes of a row): any value within a few dozen powers of two of the row maximum serves, because
-      // every CTA sends the stabiliser it used along with its sum.  Should a later chunk exceed it
-      // by more than 2^kRescale (extreme logits), the warp rescales what it has already stored.
-      constexpr float kRescale = 32.0f;
-      float z[2][kChunk];
-      tc_ld16(tbuf + kChunk * chunk_of(0), z[0]);
+      // every CTA sends the stabiliser it used along with its sum.  Later chunks compute no maximum:
+      // should their exponentials push the running sum beyond 2^kSumLimit (extreme logits), the warp
+      // takes the rare path - new stabiliser from the chunk at hand, stored chunks rescaled, the
+      // chunk redone (rescale_stored, kept out of line: the loop below is the hot code of the
+      // kernel and is written to stay small - two chunks per trip, not unrolled further).
+      constexpr float kSumLimit = 1.0995116e12f;   // 2^40
+      float z0[kChunk], z1[kChunk];
+      MD_TRACE_CLK(h, 8);
+      tc_ld16(tbuf + kChunk * chunk_of(0), z0);
       if (last_buf >= 0 && !p.tight) {   // the head this warp worked on before: hand it to the add warps
         tc_wait_st();
         tc_fence_before();
@@ -681,60 +660,79 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       }
       float mx = -INFINITY, sub = 0.0f;
       float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      auto mask_chunk = [&](float(&zc)[kChunk], int t) {
+        if (!all_visible) {
+          const int nvis = lim - kChunk * chunk_of(t);   // visible columns of this chunk
+          if (nvis < kChunk) {
 #pragma unroll
-      for (int t = 0; t < ECH; ++t) {
-        if (t < my_chunks) {   // (warp-uniform)
+            for (int j = 0; j < kChunk; ++j) zc[j] = (j < nvis) ? zc[j] : -INFINITY;
+          }
+        }
+      };
+      auto chunk_max = [&](const float(&zc)[kChunk]) {   // in log2 units; scale > 0 keeps the order
+        float c4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int j = 0; j < kChunk; ++j) c4[j & 3] = fmaxf(c4[j & 3], zc[j]);
+        float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3])) * p.scale_log2e;
+        if (HALVES == 2) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 16));   // one stabiliser per row
+        return cm;
+      };
+      // one chunk: mask, (first chunk: stabiliser,) exponentials, running sum, store
+      auto work = [&](float(&zc)[kChunk], int t) {
+        mask_chunk(zc, t);
+        if (t == 0) {
+          mx = chunk_max(zc);
+          sub = (mx == -INFINITY) ? 0.0f : mx;   // (first chunk all masked: so are the later ones)
+        }
+        float part[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int j = 0; j < kChunk; ++j) {
+          const float e = ex2(fmaf(zc[j], p.scale_log2e, -sub));
+          zc[j] = e;
+          part[j & 3] += e;
+        }
+        const float psum = (part[0] + part[1]) + (part[2] + part[3]);
+        if (t > 0 && __any_sync(0xffffffffu, !(psum < kSumLimit))) {
+          // rare: this chunk lies far above the stabiliser.  Take its logits again, move the
+          // stabiliser up (all lanes take part; lanes whose stabiliser stays multiply by 1),
+          // rescale what is stored and redo the chunk.
+          tc_ld16(tbuf + kChunk * chunk_of(t), zc);
           tc_wait_ld();
-          if (t + 1 < ECH && t + 1 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 1), z[(t + 1) & 1]);
-          float(&zc)[kChunk] = z[t & 1];
-          if (!all_visible) {
-            const int nvis = lim - kChunk * chunk_of(t);   // visible columns of this chunk
-            if (nvis < kChunk) {
+          mask_chunk(zc, t);
+          const float up = fmaxf(mx, chunk_max(zc));
+          const float fac = (up == mx) ? 1.0f : ex2(sub - up);
+          rescale_stored(tbuf + kChunk * (kAlt ? 0 : g), kAlt ? kChunk : kChunk * kColGroups, t, fac);
 #pragma unroll
-              for (int j = 0; j < kChunk; ++j) zc[j] = (j < nvis) ? zc[j] : -INFINITY;
-            }
-          }
-          float c4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          for (int x = 0; x < 4; ++x) ls4[x] *= fac;
+          mx = up;
+          sub = up;
 #pragma unroll
-          for (int j = 0; j < kChunk; ++j) c4[j & 3] = fmaxf(c4[j & 3], zc[j]);
-          const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3])) * p.scale_log2e;   // scale > 0 keeps the order
-          if (t == 0) {
-            mx = cm;
-            if (HALVES == 2) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));   // one stabiliser per row
-            sub = (mx == -INFINITY) ? 0.0f : mx;   // (first chunk all masked: so are the later ones)
-          } else if (__any_sync(0xffffffffu, cm - sub > kRescale)) {
-            // rare: move the stabiliser up and rescale the chunks already stored (all lanes take part:
-            // the tensor-memory instructions are warp-wide; lanes whose stabiliser stays multiply by 1)
-            float up = fmaxf(mx, cm);
-            if (HALVES == 2) up = fmaxf(up, __shfl_xor_sync(0xffffffffu, up, 16));
-            const float fac = (up == mx) ? 1.0f : ex2(sub - up);
-            tc_wait_st();
-#pragma unroll
-            for (int u = 0; u < t; ++u) {
-              float old[kChunk];
-              tc_ld16(tbuf + kChunk * chunk_of(u), old);
-              tc_wait_ld();
-#pragma unroll
-              for (int j = 0; j < kChunk; ++j) old[j] *= fac;
-              tc_st16(tbuf + kChunk * chunk_of(u), old);
-            }
-#pragma unroll
-            for (int x = 0; x < 4; ++x) ls4[x] *= fac;
-            mx = up;
-            sub = up;
-          }
+          for (int x = 0; x < 4; ++x) part[x] = 0.0f;
 #pragma unroll
           for (int j = 0; j < kChunk; ++j) {
             const float e = ex2(fmaf(zc[j], p.scale_log2e, -sub));
             zc[j] = e;
-            ls4[j & 3] += e;
+            part[j & 3] += e;
           }
-          tc_st16(tbuf + kChunk * chunk_of(t), zc);
+        }
+#pragma unroll
+        for (int x = 0; x < 4; ++x) ls4[x] += part[x];
+        tc_st16(tbuf + kChunk * chunk_of(t), zc);
+      };
+#pragma unroll 1
+      for (int t = 0; t < my_chunks; t += 2) {   // (my_chunks is warp-uniform)
+        tc_wait_ld();
+        if (t + 1 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 1), z1);
+        work(z0, t);
+        if (t + 1 < my_chunks) {
+          tc_wait_ld();
+          if (t + 2 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 2), z0);
+          work(z1, t + 1);
         }
       }
+      MD_TRACE_CLK(h, 15);
       float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
       if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
-#endif
       if (sender) {
         for (int c = 0; c < p.cluster; ++c)
           st_async_f32x2(map_to_cta(slot_addr, c), mx, lsum, map_to_cta(bar_addr, c));

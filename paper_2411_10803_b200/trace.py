@@ -109,6 +109,12 @@ def main(argv) -> int:
         print("CTA", c)
         for h in sorted({0, 2, 4, w.n_heads // 2 // 2 * 2, (w.n_heads - 1) // 2 * 2}):
             print("  head %02d " % h + " ".join("%s=%.2f" % (n, (t[c, h, e] - t0) / 1e3) for e, n in enumerate(EVENTS)))
+        clk = t[c, 2:, 8:16]
+        clk = clk[clk[:, 0] > 0]
+        if len(clk):
+            d = (clk - clk[:, :1]).mean(axis=0)
+            print("  exp stage of thread 0, SM clocks after its start: first chunk loaded %.0f, stabiliser %.0f, "
+                  "chunks stored %.0f %.0f %.0f %.0f, all done %.0f" % tuple(d[1:]))
         done = t[c, :, 7]
         print("  add_done per head: mean %.2f us" % (np.diff(done)[4:].mean() / 1e3))
         ev = t[c, 4::2]
