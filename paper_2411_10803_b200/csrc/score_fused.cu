@@ -48,7 +48,7 @@ constexpr int kChunk = 16;                  // TMEM columns per tcgen05.ld / st
 constexpr int kMaxCluster = 16;               // beyond 8 the cluster size is non-portable (opt-in per kernel)
 constexpr int kMaxQBufs = 4;                  // shared-memory ring of text-query tiles (one per head)
 constexpr int kMaxKBufs = 8;                  // shared-memory ring of key half-tiles (HALVES per head)
-constexpr int kMinBufs = 3;                 // tensor-memory buffers: MMA, exp and add stages in flight ...
+constexpr int kMinBufs = 3;                 // tensor-memory buffers: MMA, exp and add stages in flight (two for 176-column tiles) ...
 constexpr int kMaxBufs = 8;                 // ... more when the columns per head allow, to hide the per-head latency chain
 constexpr int kMaxSlots = 2 * kMaxBufs;     // statistics slots = 2 x buffers: a peer's exp warps run at most that far ahead of our add warps
 constexpr int kTmemCols = 512;
@@ -658,6 +658,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars.eready[last_buf]));
       }
+      MD_TRACE_CLK(h, 9);
       float mx = -INFINITY, sub = 0.0f;
       float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
       auto mask_chunk = [&](float(&zc)[kChunk], int t) {
@@ -722,12 +723,17 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 #pragma unroll 1
       for (int t = 0; t < my_chunks; t += 2) {   // (my_chunks is warp-uniform)
         tc_wait_ld();
+        if (t == 0) MD_TRACE_CLK(h, 10);
         if (t + 1 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 1), z1);
         work(z0, t);
+        if (t == 0) MD_TRACE_CLK(h, 11);
+        if (t == 2) MD_TRACE_CLK(h, 13);
         if (t + 1 < my_chunks) {
           tc_wait_ld();
           if (t + 2 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 2), z0);
           work(z1, t + 1);
+          if (t == 0) MD_TRACE_CLK(h, 12);
+          if (t == 2) MD_TRACE_CLK(h, 14);
         }
       }
       MD_TRACE_CLK(h, 15);
@@ -1086,8 +1092,9 @@ using FusedKernel = void (*)(const CUtensorMap, const CUtensorMap, const FusedPa
 
 template <bool FILTER, bool PH>
 FusedKernel pick_shape(int halves, int ach) {
-  return halves == 2 ? (ach > 5 ? score_fused_kernel<2, 10, FILTER, PH> : score_fused_kernel<2, 5, FILTER, PH>)
-                     : (ach > 5 ? score_fused_kernel<1, 10, FILTER, PH> : score_fused_kernel<1, 5, FILTER, PH>);
+  if (halves == 2) return ach > 5 ? score_fused_kernel<2, 10, FILTER, PH> : score_fused_kernel<2, 5, FILTER, PH>;
+  if (ach > 10) return score_fused_kernel<1, 11, FILTER, PH>;   // 176 columns per lane (one M=128 tile only)
+  return ach > 5 ? score_fused_kernel<1, 10, FILTER, PH> : score_fused_kernel<1, 5, FILTER, PH>;
 }
 
 FusedKernel pick_kernel(int halves, int ach, bool filter = false, bool per_head = false) {
@@ -1132,7 +1139,10 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
   if (n_rows <= 0) { row0 = 0; n_rows = r.N; }
   const int halves = n_rows <= 64 ? 2 : 1;
   const int nrows = 128 / halves;
-  const int max_cpl = 10 * kChunk;   // 160 columns per TMEM lane (add threads with 10 chunks)
+  // columns per TMEM lane: 160 (add threads with 10 chunks); 176 with one M=128 tile, where an
+  // eleventh chunk per add thread still fits its registers and saves a whole round of clusters
+  // for 128 text rows on 704 keys (4 CTAs per request instead of 5)
+  const int max_cpl = (halves == 1 ? 11 : 10) * kChunk;
   double best = -1.0;
   FusedGeometry g{};
   for (int c = 1; c <= kMaxCluster; ++c) {
@@ -1144,7 +1154,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     if (cpl > max_cpl) continue;
     const int tk = cpl * halves;
     const size_t stage = static_cast<size_t>(nrows + tk) * 256;
-    const int ach = cpl <= 5 * kChunk ? 5 : 10;             // chunks per add thread (kernel variant)
+    const int ach = cpl <= 5 * kChunk ? 5 : (cpl <= 10 * kChunk ? 10 : 11);   // chunks per add thread (kernel variant)
     const int epr = ach <= 5 ? 1 : kColGroups;              // (max, sum) pairs per row and CTA (the kernel's EPR)
     // Shared memory.  Whole stages first (a head's query tile and keys recycled together): as many
     // tensor-memory buffers as the columns allow (3..8), fewer if their statistics slots (2 x
@@ -1160,7 +1170,8 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     auto slots_bytes = [&](int n_slot) { return static_cast<size_t>(n_slot) * c * nrows * epr * 8; };
     int n_buf = kTmemCols / cpl;
     if (n_buf > kMaxBufs) n_buf = kMaxBufs;
-    if (n_buf < kMinBufs) continue;
+    const int min_bufs = cpl > 10 * kChunk ? 2 : kMinBufs;   // 176-column tiles: two buffers is all that fits
+    if (n_buf < min_bufs) continue;
     const int max_buf = n_buf;
     size_t extra = 0;
     int n_q = 0, n_k = 0, n_slot = 0, split = 0;
@@ -1169,7 +1180,7 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
       // then as many buffers as still fit (the MMA -> exp -> exchange -> add chain of ~4.6 us
       // per head is spread over them)
       int best_q = 0, best_buf = 0;
-      for (int nb = max_buf; nb >= kMinBufs; --nb) {
+      for (int nb = max_buf; nb >= min_bufs; --nb) {
         const size_t e = slots_bytes(2 * nb);
         if (e + 2 * stage > avail) continue;
         int q = static_cast<int>((avail - e) / stage);

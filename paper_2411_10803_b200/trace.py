@@ -113,8 +113,8 @@ def main(argv) -> int:
         clk = clk[clk[:, 0] > 0]
         if len(clk):
             d = (clk - clk[:, :1]).mean(axis=0)
-            print("  exp stage of thread 0, SM clocks after its start: first chunk loaded %.0f, stabiliser %.0f, "
-                  "chunks stored %.0f %.0f %.0f %.0f, all done %.0f" % tuple(d[1:]))
+            print("  exp stage of thread 0, SM clocks after its start: previous head handed over %.0f, first chunk "
+                  "loaded %.0f, chunks stored %.0f %.0f %.0f %.0f, all done %.0f" % tuple(d[1:]))
         done = t[c, :, 7]
         print("  add_done per head: mean %.2f us" % (np.diff(done)[4:].mean() / 1e3))
         ev = t[c, 4::2]

@@ -10,6 +10,7 @@ GEOMETRIES = [
     dict(C=2, n_q=2, n_buf=3),                       # the 7B batch-64 plan
     dict(C=4, n_q=4, n_buf=6),
     dict(C=5, n_q=2, n_buf=3),
+    dict(C=4, n_q=2, n_buf=2),                       # 176-column tiles: two buffers only
     dict(C=8, n_q=3, n_buf=8),
     dict(C=10, n_q=2, n_buf=3, n_slot=4, tight=2),   # large clusters: few slots, the exp role held near the add role
     dict(C=12, n_q=2, n_buf=3, n_slot=2, tight=1),
