@@ -131,15 +131,18 @@ typedef enum {
   MUSTDROP_DEBUG_VARIANT_AUTO = 0,
   MUSTDROP_DEBUG_VARIANT_TWO_PASS = 1,   /* the general-shape two-pass kernel */
   MUSTDROP_DEBUG_VARIANT_FUSED = 2,      /* the one-pass tcgen05 kernel, whatever the cost model says */
-  MUSTDROP_DEBUG_VARIANT_ROW_SPLIT = 3   /* the one-pass kernel with the text rows scored by two launches */
+  MUSTDROP_DEBUG_VARIANT_ROW_SPLIT = 3,  /* the one-pass kernel with the text rows scored by two launches */
+  MUSTDROP_DEBUG_VARIANT_GRID = 4        /* the one-pass kernel without clusters: statistics exchanged through global
+                                            memory (debug_cluster then gives the CTAs per request, up to 32) */
 } mustdrop_debug_variant_t;
 
 /*
  * Validate a configuration and build a plan (host only; nothing is launched).
  * config, plan_out and workspace_bytes are (host).  `*workspace_bytes` receives the size of
  * the device workspace the other calls need (>= 256, a multiple of 256).  The workspace must
- * be zeroed once before first use (its first bytes are the device status word); after that
- * the calls keep it consistent.  The plan records the CUDA device current at this call.
+ * be zeroed once before first use (its first bytes are the device status word, and some plans
+ * keep counters in it); after that the calls keep it consistent - except after a device status
+ * of MUSTDROP_ERR_TIMEOUT, when it has to be zeroed again before it is reused.  The plan records the CUDA device current at this call.
  */
 mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t *config, mustdrop_plan_t **plan_out,
                                        size_t *workspace_bytes);

@@ -61,6 +61,7 @@ MUSTDROP_FLAG_INPUTS_READY = 4
 
 MUSTDROP_DEBUG_VARIANT_AUTO, MUSTDROP_DEBUG_VARIANT_TWO_PASS = 0, 1
 MUSTDROP_DEBUG_VARIANT_FUSED, MUSTDROP_DEBUG_VARIANT_ROW_SPLIT = 2, 3
+MUSTDROP_DEBUG_VARIANT_GRID = 4
 
 
 class mustdrop_layer_io_t(ctypes.Structure):

@@ -70,8 +70,8 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
       c->n_vis <= 0 || c->n_txt <= 0 || c->vis_start < 0 || c->txt_start < 0 || c->key_max < 0 ||
       (c->flags & ~(MUSTDROP_FLAG_REBUILD_SEQUENCE | MUSTDROP_FLAG_PER_HEAD_MAX | MUSTDROP_FLAG_INPUTS_READY)) != 0)
     return MUSTDROP_ERR_INVALID_ARG;
-  if (c->debug_score_variant < MUSTDROP_DEBUG_VARIANT_AUTO || c->debug_score_variant > MUSTDROP_DEBUG_VARIANT_ROW_SPLIT ||
-      c->debug_cluster < 0 || c->debug_cluster > 16 || (c->debug_filter_staged & ~1) != 0 || c->debug_wait_cycles < 0)
+  if (c->debug_score_variant < MUSTDROP_DEBUG_VARIANT_AUTO || c->debug_score_variant > MUSTDROP_DEBUG_VARIANT_GRID ||
+      c->debug_cluster < 0 || c->debug_cluster > (c->debug_score_variant == MUSTDROP_DEBUG_VARIANT_GRID ? 32 : 16) || (c->debug_filter_staged & ~1) != 0 || c->debug_wait_cycles < 0)
     return MUSTDROP_ERR_INVALID_ARG;
   // the vision span precedes the text span and both lie inside the sequence
   if (static_cast<int64_t>(c->vis_start) + c->n_vis > c->txt_start ||
@@ -155,11 +155,12 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
     const int forced_cluster = c->debug_cluster;
     const bool allow_fused = c->debug_score_variant != MUSTDROP_DEBUG_VARIANT_TWO_PASS;
     const bool force_split = c->debug_score_variant == MUSTDROP_DEBUG_VARIANT_ROW_SPLIT;
+    const bool force_grid = c->debug_score_variant == MUSTDROP_DEBUG_VARIANT_GRID;
     const double k_mb = 256.0e-6 * r.B * r.H * r.L;
     const double two_pass_us = k_mb * (0.6 + 0.7 * r.N / 128.0);   // the two-pass kernel's measured rate
     double chosen_us = two_pass_us;
     p->row_split = 0;
-    if (allow_fused && !force_split && plan_score_fused(r, p->sm_count, forced_cluster, &p->fused)) {
+    if (allow_fused && !force_split && !force_grid && plan_score_fused(r, p->sm_count, forced_cluster, &p->fused)) {
       p->score_variant = kScoreFusedCluster;
       chosen_us = p->fused.est_us;
       // A fused plan that had to fall back to few statistics slots (sequences needing clusters of
@@ -177,7 +178,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
     // sums to / takes the maximum with the first's.  Taken when estimated faster than the above.
     // (Not with the per-head reading of Eq. 10: its maxima run over ALL text rows of a head before
     // the head mean, which two launches over disjoint rows cannot combine afterwards.)
-    if (allow_fused && r.N > 64 && !r.per_head_max) {
+    if (allow_fused && r.N > 64 && !r.per_head_max && !force_grid) {
       mustdrop::FusedGeometry ga, gb;
       // clusters small enough for both launches to be resident at once, if such a plan exists
       const int fit = p->sm_count / (2 * r.B);
@@ -197,6 +198,19 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
         }
       }
     }
+    // Small batches of long sequences: the same kernel without clusters - every CTA of the batch
+    // resident at once, as many per request as the SMs allow, statistics through global memory.
+    // Taken when estimated faster than what was chosen above.
+    if (allow_fused && !force_split && (force_grid || (!want && forced_cluster == 0))) {
+      mustdrop::FusedGeometry gg;
+      if (plan_score_grid(r, p->sm_count, force_grid ? forced_cluster : 0, &gg) &&
+          (force_grid || gg.est_us < (p->row_split ? 1e30 : chosen_us) * 0.9 ||
+           (p->row_split && gg.est_us < 1.15 * (p->fused.est_us > p->fused_b.est_us ? p->fused.est_us : p->fused_b.est_us)))) {
+        p->score_variant = kScoreFusedCluster;
+        p->row_split = 0;
+        p->fused = gg;
+      }
+    }
     // mustdrop_filter: one launch where the fused kernel covers the shape and a kept row fits its
     // shared-memory ring; debug_filter_staged forces the separate launches.
     p->filter_single = 0;
@@ -207,6 +221,13 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   size_t off = kWsStatusBytes;
   p->ws_rowstats_off = off;
   off += round_up(sizeof(float) * 2 * static_cast<size_t>(r.B) * r.H * r.N, 256);
+  p->ws_gx_cnt_off = p->ws_gx_stats_off = off;
+  if (p->score_variant == kScoreFusedCluster && p->fused.gx) {
+    p->ws_gx_cnt_off = off;
+    off += round_up(sizeof(uint32_t) * (2 * static_cast<size_t>(r.B) * r.H + 2 * static_cast<size_t>(r.B)), 256);
+    p->ws_gx_stats_off = off;
+    off += round_up(grid_plan_stats_bytes(r, p->fused), 256);
+  }
   p->ws_bytes = off;
   p->map_cache = map_cache_create();
   *workspace_bytes = p->ws_bytes;
@@ -404,11 +425,18 @@ int32_t mustdrop_plan_describe(const mustdrop_plan_t* plan, char* buf, size_t n)
   int len;
   if (plan->score_variant == mustdrop::kScoreFusedCluster) {
     const mustdrop::FusedGeometry& g = plan->row_split ? plan->fused_b : plan->fused;
-    len = std::snprintf(text, sizeof(text),
-                        "fused tcgen05 score%s: cluster %d, %d keys per CTA, %s %d/%d, %d tensor-memory buffers, "
-                        "%d statistics slots, %d clusters resident; filter = %d launch(es)",
-                        plan->row_split ? " (text rows in two launches; second launch)" : "", g.cluster, g.tk, g.split ? "query/key-half rings" : "stages", g.n_q, g.split ? g.n_k : 0, g.n_buf, g.n_slot,
-                        g.resident, mustdrop_plan_filter_launches(plan));
+    if (g.gx)
+      len = std::snprintf(text, sizeof(text),
+                          "fused tcgen05 score: grid plan (statistics through global memory), %d CTAs per request, "
+                          "%d keys per CTA, stages %d, %d tensor-memory buffers; filter = %d launch(es)",
+                          g.cluster, g.tk, g.n_q, g.n_buf, mustdrop_plan_filter_launches(plan));
+    else
+      len = std::snprintf(text, sizeof(text),
+                          "fused tcgen05 score%s: cluster %d, %d keys per CTA, %s %d/%d, %d tensor-memory buffers, "
+                          "%d statistics slots, %d clusters resident; filter = %d launch(es)",
+                          plan->row_split ? " (text rows in two launches; second launch)" : "", g.cluster, g.tk,
+                          g.split ? "query/key-half rings" : "stages", g.n_q, g.split ? g.n_k : 0, g.n_buf, g.n_slot,
+                          g.resident, mustdrop_plan_filter_launches(plan));
   } else {
     len = std::snprintf(text, sizeof(text), "two-pass mma.sync score; filter = %d launch(es)",
                         mustdrop_plan_filter_launches(plan));

@@ -34,6 +34,8 @@ struct FusedGeometry {
   int32_t n_slot;     // statistics slots: 2 x n_buf, or 2d (d = 2 or 1) with the exp warps held within d heads of the add warps
   int32_t ach;        // chunks of 16 columns per accumulating thread (kernel variant: 5 or 10)
   int32_t row0, n_rows;   // the text rows this geometry's launch covers
+  int32_t gx;         // 1: grid plan - the request's CTAs are ordinary CTAs of the grid (cluster = their number) and
+                      //    exchange their statistics through global memory
   int32_t resident;   // clusters the device can hold at once (0: not asked)
   float est_us;       // the planner's estimate of the score time
   size_t smem_bytes;  // dynamic shared memory
@@ -87,6 +89,8 @@ struct mustdrop_plan {
   int32_t score_variant;
   size_t ws_bytes;
   size_t ws_rowstats_off;   // float2 [B,H,N]: (row max in log2 units, 1 / row sum)
+  size_t ws_gx_cnt_off;     // grid plans: uint32 counters [2 B H + 2 B], zero between calls
+  size_t ws_gx_stats_off;   // grid plans: float2 [B,H,CTAs per request,rows,pairs]
   mustdrop::FusedGeometry fused;
   int32_t row_split;        // 1: the text rows are scored by two launches (fused: rows 0..63, fused_b: the rest)
   mustdrop::FusedGeometry fused_b;
@@ -105,6 +109,10 @@ cudaError_t launch_score_two_pass(const mustdrop_plan& p, const void* q_text, co
                                   const int32_t* vis_cnt = nullptr);
 bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, FusedGeometry* out, int row0 = 0,
                       int n_rows = 0, int max_cluster = 0);
+// Grid plan of the same kernel (all CTAs of the batch resident at once, statistics through global
+// memory); false when the batch leaves fewer than two CTAs per request or the shape does not fit.
+bool plan_score_grid(const Resolved& r, int sm_count, int forced_ctas, FusedGeometry* out);
+size_t grid_plan_stats_bytes(const Resolved& r, const FusedGeometry& g);
 cudaError_t launch_score_fused(const mustdrop_plan& p, const void* q_text, const void* k, float* g_out,
                                float* i_out, void* workspace, cudaStream_t stream, const int32_t* vis_cnt = nullptr);
 bool plan_filter_single(const Resolved& r, const FusedGeometry& geo, FilterGeometry* out);

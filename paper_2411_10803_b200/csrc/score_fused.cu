@@ -69,6 +69,11 @@ struct FusedParams {
   int32_t split;
   int32_t n_buf, n_slot;              // tensor-memory buffers, statistics slots (2 * n_buf, or 4 when tight)
   int32_t tight;                      // d = 1 or 2: the exp warps start head h only when the add warps are done with head h - d (0: no such rule)
+  // Statistics exchange through global memory instead of distributed shared memory ("grid" plans:
+  // the CTAs of a request are ordinary CTAs of the grid, any number of them, all resident at once).
+  int32_t gx;                         // 1: grid plan (cluster = CTAs per request, launched without a cluster)
+  float2* gx_stats;                   // [B][H][CTAs per request][rows][pairs] (stabiliser, sum)
+  uint32_t* gx_cnt;                   // [B*H] pairs sent, [B*H] readers done, [B] scores stored, [B] barrier passed; zero between calls
   int32_t per_head;                   // 1: i_out = head mean of the per-head maxima over the text rows (PH instantiations)
   int32_t early_inputs;               // 1: q_text / k may be read before the stream's earlier work has completed (caller's promise)
   long long wait_cycles;              // clock cycles after which a wait between the warp roles gives up
@@ -114,6 +119,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "r"(bar), "r"(parity)
       : "memory");
   return ok != 0;
+}
+// Grid plans: release / acquire on a counter in global memory.
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+// Bounded wait until a counter has reached its target (same give-up rules as mbar_wait).
+__device__ __forceinline__ bool count_wait(const uint32_t* p, uint32_t target, volatile int* abort_flag, long long limit) {
+  if (ld_acquire_gpu(p) >= target) return true;
+  const long long t0 = clock64();
+  while (ld_acquire_gpu(p) < target) {
+    if (*abort_flag != 0 || clock64() - t0 > limit) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+  return true;
 }
 // Bounded wait.  Returns false (and raises the CTA's abort flag) when the wait ran out or the
 // CTA has already given up.
@@ -330,7 +353,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   volatile int* abort_flag = &abort_flag_s;
   const long long wait_limit = p.wait_cycles;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_cta_rank();
+  const uint32_t rank = p.gx ? blockIdx.x % static_cast<uint32_t>(p.cluster) : cluster_cta_rank();
   const int b = blockIdx.x / p.cluster;
   MD_PIPE(p.workspace, 0, false, true);
   if (threadIdx.x == 0) MD_TRACE(0, 8);    // (CTA-level stamps use the event slots 8.. of head 0) kernel entry
@@ -404,7 +427,29 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     __syncwarp();   // a warp whose lane 0 had a role of its own is whole again before the aligned instructions below
     tc_fence_before();
     cta_sync();
-    if (threadIdx.x == 0 && *abort_flag != 0) {
+    if (p.gx) {
+      // grid plan: the request's CTAs are no cluster.  In the filter kernel they meet through a
+      // counter in global memory: every CTA's scores are stored before any CTA selects.  (A CTA
+      // that gives up tells nobody: its peers run into their own limits.)
+      if (threadIdx.x == 0) {
+        if (FILTER && *abort_flag == 0) {
+          uint32_t* const stored = p.gx_cnt + 2 * static_cast<size_t>(gridDim.x / p.cluster) * p.H + b;
+          uint32_t* const passed = stored + gridDim.x / p.cluster;
+          __threadfence();
+          atomicAdd(stored, 1u);
+          if (count_wait(stored, static_cast<uint32_t>(p.cluster), abort_flag, wait_limit) &&
+              atomicAdd(passed, 1u) == static_cast<uint32_t>(p.cluster) - 1u) {
+            *stored = 0u;   // the last one through leaves the counters as the next call expects them
+            *passed = 0u;
+          }
+        }
+        if (*abort_flag != 0) {
+          record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
+          cluster_abort_s = 1;
+        }
+      }
+      cta_sync();
+    } else if (threadIdx.x == 0 && *abort_flag != 0) {
       record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
       for (int c = 0; c < p.cluster; ++c) st_remote_u32(map_to_cta(smem_u32(&cluster_abort_s), c), 1u);
     }
@@ -422,7 +467,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   // asynchronous statistics stores may still be on their way into this CTA's shared memory: give
   // them time to land and meet once more, so that no CTA's shared memory goes away under them.
   auto leave_after_give_up = [&](int32_t* kept_cnt) {
-    if (kept_cnt != nullptr && rank == 0 && threadIdx.x == 0) {
+    if (kept_cnt != nullptr && (rank == 0 || p.gx) && threadIdx.x == 0) {
       pdl_wait();
       kept_cnt[b] = -1;   // this request's result is invalid
     }
@@ -615,6 +660,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const uint32_t pair_idx = (rank * NROWS + row) * EPR + (kAlt ? 0 : g);     // this thread's pair in a slot
 
     int last_buf = -1;
+    if (p.gx) pdl_wait();   // the statistics go through global memory: not before the stream's earlier work is done
     for (int h = kAlt ? g : 0; h < p.H; h += kAlt ? kColGroups : 1) {
       const int buf = h % p.n_buf;
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
@@ -631,7 +677,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       }
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag, wait_limit))) break;
       if (threadIdx.x == 0) MD_TRACE(h, 3);
-      if (lane == 0 && q == 0 && (kAlt || g == 0)) {
+      if (!p.gx && lane == 0 && q == 0 && (kAlt || g == 0)) {
         // arm this head's statistics barrier with the bytes all CTAs will send
         mbar_expect_tx(smem_u32(&bars.sfull[slot]), slot_pairs * 8u);
       }
@@ -739,7 +785,16 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       MD_TRACE_CLK(h, 15);
       float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
       if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
-      if (sender) {
+      if (p.gx) {
+        // grid plan: the pair goes to global memory; the warp's pairs are published by one counted release
+        const size_t bh = static_cast<size_t>(b) * p.H + h;
+        if (sender) p.gx_stats[((bh * p.cluster + rank) * NROWS + row) * EPR + (kAlt ? 0 : g)] = make_float2(mx, lsum);
+        __syncwarp();
+        if (lane == 0) {
+          __threadfence();
+          atomicAdd(p.gx_cnt + bh, 1u);
+        }
+      } else if (sender) {
         for (int c = 0; c < p.cluster; ++c)
           st_async_f32x2(map_to_cta(slot_addr, c), mx, lsum, map_to_cta(bar_addr, c));
       }
@@ -805,30 +860,68 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const bool real_row = row < p.N;     // lanes beyond the text rows carry padding
 
     int h = 0;
+    if (p.gx) pdl_wait();   // the counters below belong to the workspace: an earlier call may still be resetting them
     for (; h < p.H; ++h) {
       const int buf = h % p.n_buf;
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
       const int slot = h % p.n_slot;
       const uint32_t sph = static_cast<uint32_t>(h / p.n_slot) & 1u;
-      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag, wait_limit))) break;
-      if (tid_a == 0) MD_TRACE(h, 5);
-      // statistics of this row over the whole key range: every CTA's pairs
-      const float2* srow = stats + slot * slot_pairs + row * EPR;
-      float m = -INFINITY;
-      for (int c = 0; c < p.cluster; ++c)
-#pragma unroll
-        for (int x = 0; x < EPR; ++x) m = fmaxf(m, srow[c * NROWS * EPR + x].x);
-      float l = 0.0f;
-      for (int c = 0; c < p.cluster; ++c)
-#pragma unroll
-        for (int x = 0; x < EPR; ++x) {
-          const float2 v = srow[c * NROWS * EPR + x];
-          l = fmaf(v.y, ex2(v.x - m), l);     // an empty pair is (-inf, 0): contributes 0
-        }
-      const float inv_l = 1.0f / l;
       float f[EPR];                            // factor of each of this CTA's pairs
+      if (p.gx) {
+        // grid plan: wait until every CTA of the request has published its pairs of this head, then
+        // merge this row's pairs straight from global memory (L2), one CTA after the other
+        const size_t bh = static_cast<size_t>(b) * p.H + h;
+        uint32_t* const sent = p.gx_cnt + bh;
+        const uint32_t target = static_cast<uint32_t>(p.cluster) * (kAlt ? kExpWarps / kColGroups : kExpWarps);
+        const bool ok = lane != 0 || count_wait(sent, target, abort_flag, wait_limit);
+        if (!__all_sync(0xffffffffu, ok)) break;
+        (void)ld_acquire_gpu(sent);            // every lane's own acquire orders its loads below
+        if (tid_a == 0) MD_TRACE(h, 5);
+        const float2* const grow = p.gx_stats + (bh * p.cluster * NROWS + row) * EPR;
+        float m = -INFINITY, l = 0.0f, own[EPR];
+#pragma unroll 4
+        for (int c = 0; c < p.cluster; ++c) {
 #pragma unroll
-      for (int x = 0; x < EPR; ++x) f[x] = ex2(srow[rank * NROWS * EPR + x].x - m) * inv_l;
+          for (int x = 0; x < EPR; ++x) {
+            const float2 v = __ldcg(grow + static_cast<size_t>(c) * NROWS * EPR + x);
+            const float m_new = fmaxf(m, v.x);
+            const float ref = (m_new == -INFINITY) ? 0.0f : m_new;
+            l = fmaf(l, ex2(m - ref), v.y * ex2(v.x - ref));   // an empty pair is (-inf, 0): contributes 0
+            m = m_new;
+            if (c == static_cast<int>(rank)) own[x] = v.x;
+          }
+        }
+        const float inv_l = 1.0f / l;
+#pragma unroll
+        for (int x = 0; x < EPR; ++x) f[x] = ex2(own[x] - m) * inv_l;
+        __syncwarp();
+        if (lane == 0) {   // the last reader of the head leaves its counters as the next call expects them
+          uint32_t* const done = sent + static_cast<size_t>(gridDim.x / p.cluster) * p.H;
+          if (atomicAdd(done, 1u) == static_cast<uint32_t>(p.cluster) * kAddWarps - 1u) {
+            *sent = 0u;
+            *done = 0u;
+          }
+        }
+      } else {
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag, wait_limit))) break;
+        if (tid_a == 0) MD_TRACE(h, 5);
+        // statistics of this row over the whole key range: every CTA's pairs
+        const float2* srow = stats + slot * slot_pairs + row * EPR;
+        float m = -INFINITY;
+        for (int c = 0; c < p.cluster; ++c)
+#pragma unroll
+          for (int x = 0; x < EPR; ++x) m = fmaxf(m, srow[c * NROWS * EPR + x].x);
+        float l = 0.0f;
+        for (int c = 0; c < p.cluster; ++c)
+#pragma unroll
+          for (int x = 0; x < EPR; ++x) {
+            const float2 v = srow[c * NROWS * EPR + x];
+            l = fmaf(v.y, ex2(v.x - m), l);     // an empty pair is (-inf, 0): contributes 0
+          }
+        const float inv_l = 1.0f / l;
+#pragma unroll
+        for (int x = 0; x < EPR; ++x) f[x] = ex2(srow[rank * NROWS * EPR + x].x - m) * inv_l;
+      }
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.eready[buf]), bph, abort_flag, wait_limit))) break;
       if (tid_a == 0) MD_TRACE(h, 6);
       tc_fence_after();
@@ -1246,6 +1339,64 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
   return true;
 }
 
+// Grid plan: G CTAs per request with B * G <= SMs, so that every CTA of the batch is resident at
+// once (one CTA per SM: each asks for more than half of the shared memory) and no request waits
+// for a CTA that has not started.  The statistics of a head cross through global memory (L2).
+bool plan_score_grid(const Resolved& r, int sm_count, int forced_ctas, FusedGeometry* out) {
+  const int halves = r.N <= 64 ? 2 : 1;
+  const int nrows = 128 / halves;
+  const int max_g = sm_count / r.B < 32 ? sm_count / r.B : 32;
+  double best = -1.0;
+  FusedGeometry g{};
+  for (int c = 2; c <= max_g; ++c) {
+    if (forced_ctas > 0 && c != forced_ctas) continue;
+    const int per_cta = (r.L + c - 1) / c;
+    int cpl = (per_cta + halves - 1) / halves;
+    cpl = (cpl + kChunk - 1) / kChunk * kChunk;
+    if (cpl > 10 * kChunk) continue;
+    const int tk = cpl * halves;
+    if (static_cast<long>(c - 1) * tk >= r.L) continue;       // a CTA without keys
+    const size_t stage = static_cast<size_t>(nrows + tk) * 256;
+    const int ach = cpl <= 5 * kChunk ? 5 : 10;
+    const size_t ph_bytes = r.per_head_max ? static_cast<size_t>(2 * kAddWarps) * tk * sizeof(float) : 0;
+    const size_t avail = 227 * 1024 - 4096 - 1024 - ph_bytes;
+    int n_buf = kTmemCols / cpl;
+    if (n_buf > kMaxBufs) n_buf = kMaxBufs;
+    if (n_buf < kMinBufs) continue;
+    int n_q = static_cast<int>(avail / stage);
+    if (n_q > 4) n_q = 4;
+    if (n_q < 2) continue;
+    size_t smem_bytes = n_q * stage + 1024 + ph_bytes;
+    if (smem_bytes < 116 * 1024) smem_bytes = 116 * 1024;
+    // Cost per head and CTA (microseconds): streaming the stage at ~45 GB/s per SM; the exp stage
+    // (measured: ~0.011 us per column of a lane, two heads at a time on narrow tiles); the
+    // MMA -> exp -> exchange through L2 -> add chain (~6 us) spread over the buffers.
+    const double t_stream = static_cast<double>(stage) / 45.0e3;
+    const double t_exp = (ach <= 5 ? 0.0075 : 0.011) * cpl + 0.2;
+    const double t_chain = 6.0 / n_buf;
+    double t_head = t_stream > t_exp ? t_stream : t_exp;
+    if (t_chain > t_head) t_head = t_chain;
+    if (t_head < 1.4) t_head = 1.4;
+    const double score = 1.0 / t_head + 1e-4 * c;
+    if (score > best) {
+      best = score;
+      g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_q = n_q; g.n_k = 0; g.split = 0; g.n_buf = n_buf;
+      g.ach = ach; g.n_slot = 2; g.gx = 1; g.resident = sm_count; g.row0 = 0; g.n_rows = r.N;
+      g.est_us = static_cast<float>(r.H * t_head + 12.0);    // (+ filling and draining the longer chain)
+      g.smem_bytes = smem_bytes;
+    }
+  }
+  if (best < 0.0) return false;
+  *out = g;
+  return true;
+}
+
+size_t grid_plan_stats_bytes(const Resolved& r, const FusedGeometry& g) {
+  const int nrows = 128 / g.halves;
+  const int epr = g.ach <= 5 ? 1 : kColGroups;
+  return static_cast<size_t>(r.B) * r.H * g.cluster * nrows * epr * sizeof(float2);
+}
+
 namespace {
 
 // Common launch of the score kernel, with (tail != nullptr) or without the selection / gather tail.
@@ -1290,7 +1441,10 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const FusedGeometry& 
   p.causal = r.causal;
   p.n_txt = r.N; p.row0 = geo.row0; p.combine = combine ? 1 : 0;
   p.cluster = geo.cluster; p.tk = geo.tk; p.cpl = geo.cpl; p.n_q = geo.n_q; p.n_k = geo.n_k; p.split = geo.split;
-  p.n_buf = geo.n_buf; p.n_slot = geo.n_slot; p.tight = geo.n_slot < 2 * geo.n_buf ? geo.n_slot / 2 : 0;
+  p.n_buf = geo.n_buf; p.n_slot = geo.n_slot; p.tight = (!geo.gx && geo.n_slot < 2 * geo.n_buf) ? geo.n_slot / 2 : 0;
+  p.gx = geo.gx;
+  p.gx_cnt = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(workspace) + plan.ws_gx_cnt_off);
+  p.gx_stats = reinterpret_cast<float2*>(static_cast<unsigned char*>(workspace) + plan.ws_gx_stats_off);
   p.per_head = r.per_head_max;
   p.early_inputs = (r.inputs_ready && vis_cnt == nullptr) ? 1 : 0;
   p.wait_cycles = r.wait_cycles > 0 ? r.wait_cycles : kWaitCycles;
@@ -1307,7 +1461,7 @@ cudaError_t launch_fused_common(const mustdrop_plan& plan, const FusedGeometry& 
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = static_cast<unsigned>(geo.cluster);
+  attr[0].val.clusterDim.x = geo.gx ? 1u : static_cast<unsigned>(geo.cluster);   // grid plans: no cluster
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -25,7 +25,7 @@ TIE_RTOL = 1e-3
 DEBUG = {}
 
 VARIANT_CODES = {"two_pass": md.MUSTDROP_DEBUG_VARIANT_TWO_PASS, "fused": md.MUSTDROP_DEBUG_VARIANT_FUSED,
-                 "row_split": md.MUSTDROP_DEBUG_VARIANT_ROW_SPLIT}
+                 "row_split": md.MUSTDROP_DEBUG_VARIANT_ROW_SPLIT, "grid": md.MUSTDROP_DEBUG_VARIANT_GRID}
 
 
 def force(monkeypatch, variant=None, cluster=None, staged=None):

@@ -64,7 +64,8 @@ def test_valid_plan_and_workspace_size():
     (dict(alpha=float("nan")), md.MUSTDROP_ERR_INVALID_ARG),
     (dict(scale=float("inf")), md.MUSTDROP_ERR_INVALID_ARG),
     (dict(flags=8), md.MUSTDROP_ERR_INVALID_ARG),                 # unknown flag bit
-    (dict(debug_score_variant=4), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(debug_score_variant=5), md.MUSTDROP_ERR_INVALID_ARG),
+    (dict(debug_score_variant=4, debug_cluster=33), md.MUSTDROP_ERR_INVALID_ARG),
     (dict(debug_cluster=17), md.MUSTDROP_ERR_INVALID_ARG),
     (dict(debug_filter_staged=2), md.MUSTDROP_ERR_INVALID_ARG),
     (dict(debug_wait_cycles=-1), md.MUSTDROP_ERR_INVALID_ARG),

@@ -58,7 +58,7 @@ def test_full_size_plans_are_single_launches():
     # (every request of these workloads is compared with the oracle, on this path too, by
     # test_full_config_every_request_matches_oracle)
     for name, launches in (("c2_llava7b_b16", 1), ("c2_llava7b_b64", 1), ("c3_next7b", 1), ("c5_13b_b64", 1),
-                           ("c4_video", 2)):
+                           ("c4_video", 1)):
         f = md.Filter(cfg(synth.WORKLOADS[name]))
         assert f.filter_launches == launches, name
         f.close()
@@ -203,6 +203,33 @@ def test_row_split_score_and_filter_match_oracle(n_txt, causal, monkeypatch):
 
 
 # ---- bounded waits: a wait that runs out is reported, not a hang ---------------------------------
+
+@pytest.mark.parametrize("grid_ctas", [2, 5, 9])
+def test_filter_on_a_grid_plan(grid_ctas, monkeypatch):
+    """The request's CTAs as ordinary CTAs of the grid: statistics and the barrier before the
+    selection go through counters in global memory, which every call leaves at zero - so the
+    same plan and workspace are used three times in a row."""
+    force(monkeypatch, variant="grid", cluster=grid_ctas)
+    w = small(batch=5, n_vis=333, n_txt=21, n_heads=3, hidden=384, key_cnt=9, budget=40, vis_start=2)
+    f = md.Filter(cfg(w))
+    assert "grid plan" in f.description and f.filter_launches == 1
+    f.close()
+    run_chain_and_check(w, path="filter", expect_launches=1)
+    run_chain_and_check(w, path="staged")
+    d = synth.make_batch(w)
+    q, k, v, hid = (to_dev_bf16(d[n]) for n in ("q_text", "k", "v", "hidden"))
+    ki, kc = key_args(w, d)
+    f = md.Filter(cfg(w))
+    f.filter(q, k, v, hid, ki, kc)
+    first = (f.g.clone(), f.i.clone(), f.kept_idx.clone(), f.hidden_out.clone(), f.k_out.clone())
+    for _ in range(3):
+        f.filter(q, k, v, hid, ki, kc)
+    torch.cuda.synchronize()
+    assert f.device_status() == (0, 0)
+    for a, b in zip(first, (f.g, f.i, f.kept_idx, f.hidden_out, f.k_out)):
+        assert torch.equal(a, b)
+    f.close()
+
 
 @pytest.mark.parametrize("cluster", [0, 3], indirect=True)
 def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_unaffected(cluster):

@@ -29,7 +29,8 @@ def small(**kw):
     return TINY.with_(**base)
 
 
-VARIANTS = ["auto", "two_pass", "fused:1", "fused:2", "fused:3", "fused:5", "fused:8", "fused:12", "fused:16"]
+VARIANTS = ["auto", "two_pass", "fused:1", "fused:2", "fused:3", "fused:5", "fused:8", "fused:12", "fused:16",
+            "grid:2", "grid:3", "grid:7", "grid:24"]      # grid: CTAs per request of a plan without clusters
 
 
 @pytest.fixture
@@ -40,6 +41,8 @@ def variant(request, monkeypatch):
         force(monkeypatch, variant="two_pass")
     elif v.startswith("fused:"):
         force(monkeypatch, variant="fused", cluster=v.split(":")[1])
+    elif v.startswith("grid:"):
+        force(monkeypatch, variant="grid", cluster=v.split(":")[1])
     return v
 
 
@@ -49,6 +52,9 @@ def check_variant(f, v):
     elif v.startswith("fused:") and f.score_variant != "fused_cluster_tcgen05":
         f.close()
         pytest.skip("this shape does not fit the fused kernel at that cluster size")
+    elif v.startswith("grid:") and "grid plan" not in f.description:
+        f.close()
+        pytest.skip("this shape has no plan with that many CTAs per request")
 
 
 def key_args(w, d):
