@@ -373,7 +373,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   float2* stats = reinterpret_cast<float2*>(stage_ptr + staging);
   const uint32_t slot_pairs = static_cast<uint32_t>(p.cluster) * NROWS * EPR;   // pairs per slot
   // PH only: [2][4 add warps][tk] per-head column maxima of each warp's text rows, double-buffered over heads
-  float* const ph_stage = reinterpret_cast<float*>(stats + static_cast<size_t>(p.n_slot) * slot_pairs);
+  // (grid plans keep no statistics slots in shared memory: the maxima then start where the slots would)
+  float* const ph_stage = reinterpret_cast<float*>(stats + (p.gx ? 0 : static_cast<size_t>(p.n_slot) * slot_pairs));
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
