@@ -373,8 +373,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   float2* stats = reinterpret_cast<float2*>(stage_ptr + staging);
   const uint32_t slot_pairs = static_cast<uint32_t>(p.cluster) * NROWS * EPR;   // pairs per slot
   // PH only: [2][4 add warps][tk] per-head column maxima of each warp's text rows, double-buffered over heads
-  // (grid plans keep no statistics slots in shared memory: the maxima then start where the slots would)
-  float* const ph_stage = reinterpret_cast<float*>(stats + (p.gx ? 0 : static_cast<size_t>(p.n_slot) * slot_pairs));
+  float* const ph_stage = reinterpret_cast<float*>(stats + static_cast<size_t>(p.n_slot) * slot_pairs);
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
@@ -386,7 +385,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       mbar_init(smem_u32(&bars.eready[s]), kAlt ? kExpWarps / kColGroups : kExpWarps);
       mbar_init(smem_u32(&bars.tempty[s]), kAddWarps);
     }
-    for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), 1);
+    // (grid plans: the 32 lanes of the fetch warp each arrive once their copies have landed)
+    for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), p.gx ? 32 : 1);
     mbar_init(smem_u32(&bars.fin), kAddThreads);
     mbar_init(smem_u32(&bars.ph), kAddThreads);
     for (int s = 0; s < kMaxGatherSlots; ++s) mbar_init(smem_u32(&bars.gfull[s]), 1);
@@ -635,6 +635,44 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles) {}
       }
     }
+    if (warp == kMmaWarp + 1 && p.gx) {
+      // ---------------- statistics fetch warp (grid plans) ----------------
+      // Per head: wait until every CTA of the request has published its pairs (a counter in global
+      // memory), then copy the head's block of pairs from global memory (L2) into a statistics slot
+      // with asynchronous copies that arrive on the slot's barrier - the add warps find their
+      // statistics in shared memory exactly as with a cluster, and the round trips to L2 are off
+      // their path.  A slot is reused once the add warps are done with the head that used it.
+      pdl_wait();   // the counters belong to the workspace: an earlier call may still be resetting them
+      const uint32_t target = static_cast<uint32_t>(p.cluster) * (kAlt ? kExpWarps / kColGroups : kExpWarps);
+      const uint32_t slot_bytes_gx = slot_pairs * 8u;
+      for (int h = 0; h < p.H; ++h) {
+        const int slot = h % p.n_slot;
+        if (h >= p.n_slot) {
+          const int u = h - p.n_slot;
+          if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tempty[u % p.n_buf]),
+                                                 static_cast<uint32_t>(u / p.n_buf) & 1u, abort_flag, wait_limit)))
+            break;
+        }
+        const size_t bh = static_cast<size_t>(b) * p.H + h;
+        uint32_t* const sent = p.gx_cnt + bh;
+        const bool ok = lane != 0 || count_wait(sent, target, abort_flag, wait_limit);
+        if (!__all_sync(0xffffffffu, ok)) break;
+        (void)ld_acquire_gpu(sent);            // every lane's own acquire orders its copies below
+        const unsigned char* const src = reinterpret_cast<const unsigned char*>(p.gx_stats + bh * slot_pairs);
+        const uint32_t dst = smem_u32(stats + static_cast<size_t>(slot) * slot_pairs);
+        for (uint32_t off = lane * 16u; off < slot_bytes_gx; off += 32u * 16u)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + off), "l"(src + off) : "memory");
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&bars.sfull[slot])) : "memory");
+        if (lane == 0) {   // the last CTA to have seen the head complete leaves its counters as the next call expects them
+          uint32_t* const done = sent + static_cast<size_t>(gridDim.x / p.cluster) * p.H;
+          if (atomicAdd(done, 1u) == static_cast<uint32_t>(p.cluster) - 1u) {
+            *sent = 0u;
+            *done = 0u;
+          }
+        }
+      }
+      asm volatile("cp.async.wait_all;" ::: "memory");   // no copy of this warp is in flight when the CTA leaves
+    }
     if constexpr (FILTER) {
       // filter tail, TMA / MMA warps: nothing to do but to meet the others
       common_exit();
@@ -861,49 +899,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const bool real_row = row < p.N;     // lanes beyond the text rows carry padding
 
     int h = 0;
-    if (p.gx) pdl_wait();   // the counters below belong to the workspace: an earlier call may still be resetting them
     for (; h < p.H; ++h) {
       const int buf = h % p.n_buf;
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
       const int slot = h % p.n_slot;
       const uint32_t sph = static_cast<uint32_t>(h / p.n_slot) & 1u;
       float f[EPR];                            // factor of each of this CTA's pairs
-      if (p.gx) {
-        // grid plan: wait until every CTA of the request has published its pairs of this head, then
-        // merge this row's pairs straight from global memory (L2), one CTA after the other
-        const size_t bh = static_cast<size_t>(b) * p.H + h;
-        uint32_t* const sent = p.gx_cnt + bh;
-        const uint32_t target = static_cast<uint32_t>(p.cluster) * (kAlt ? kExpWarps / kColGroups : kExpWarps);
-        const bool ok = lane != 0 || count_wait(sent, target, abort_flag, wait_limit);
-        if (!__all_sync(0xffffffffu, ok)) break;
-        (void)ld_acquire_gpu(sent);            // every lane's own acquire orders its loads below
-        if (tid_a == 0) MD_TRACE(h, 5);
-        const float2* const grow = p.gx_stats + (bh * p.cluster * NROWS + row) * EPR;
-        float m = -INFINITY, l = 0.0f, own[EPR];
-#pragma unroll 4
-        for (int c = 0; c < p.cluster; ++c) {
-#pragma unroll
-          for (int x = 0; x < EPR; ++x) {
-            const float2 v = __ldcg(grow + static_cast<size_t>(c) * NROWS * EPR + x);
-            const float m_new = fmaxf(m, v.x);
-            const float ref = (m_new == -INFINITY) ? 0.0f : m_new;
-            l = fmaf(l, ex2(m - ref), v.y * ex2(v.x - ref));   // an empty pair is (-inf, 0): contributes 0
-            m = m_new;
-            if (c == static_cast<int>(rank)) own[x] = v.x;
-          }
-        }
-        const float inv_l = 1.0f / l;
-#pragma unroll
-        for (int x = 0; x < EPR; ++x) f[x] = ex2(own[x] - m) * inv_l;
-        __syncwarp();
-        if (lane == 0) {   // the last reader of the head leaves its counters as the next call expects them
-          uint32_t* const done = sent + static_cast<size_t>(gridDim.x / p.cluster) * p.H;
-          if (atomicAdd(done, 1u) == static_cast<uint32_t>(p.cluster) * kAddWarps - 1u) {
-            *sent = 0u;
-            *done = 0u;
-          }
-        }
-      } else {
+      {
         if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag, wait_limit))) break;
         if (tid_a == 0) MD_TRACE(h, 5);
         // statistics of this row over the whole key range: every CTA's pairs
@@ -1364,10 +1366,16 @@ bool plan_score_grid(const Resolved& r, int sm_count, int forced_ctas, FusedGeom
     int n_buf = kTmemCols / cpl;
     if (n_buf > kMaxBufs) n_buf = kMaxBufs;
     if (n_buf < kMinBufs) continue;
-    int n_q = static_cast<int>(avail / stage);
-    if (n_q > 4) n_q = 4;
-    if (n_q < 2) continue;
-    size_t smem_bytes = n_q * stage + 1024 + ph_bytes;
+    // shared memory: statistics slots the fetch warp fills (a head's pairs of all the request's
+    // CTAs; at least two, so that the next head's are fetched while this one is added) and stages
+    const int epr = ach <= 5 ? 1 : kColGroups;
+    const size_t slot = static_cast<size_t>(c) * nrows * epr * 8;
+    if (2 * slot + 2 * stage > avail) continue;
+    int n_q = static_cast<int>((avail - 2 * slot) / stage);
+    if (n_q > 3) n_q = 3;
+    int n_slot = static_cast<int>((avail - n_q * stage) / slot);
+    if (n_slot > 4) n_slot = 4;
+    size_t smem_bytes = n_q * stage + n_slot * slot + 1024 + ph_bytes;
     if (smem_bytes < 116 * 1024) smem_bytes = 116 * 1024;
     // Cost per head and CTA (microseconds): streaming the stage at ~45 GB/s per SM; the exp stage
     // (measured: ~0.011 us per column of a lane, two heads at a time on narrow tiles); the
@@ -1382,7 +1390,7 @@ bool plan_score_grid(const Resolved& r, int sm_count, int forced_ctas, FusedGeom
     if (score > best) {
       best = score;
       g.halves = halves; g.cluster = c; g.tk = tk; g.cpl = cpl; g.n_q = n_q; g.n_k = 0; g.split = 0; g.n_buf = n_buf;
-      g.ach = ach; g.n_slot = 2; g.gx = 1; g.resident = sm_count; g.row0 = 0; g.n_rows = r.N;
+      g.ach = ach; g.n_slot = n_slot; g.gx = 1; g.resident = sm_count; g.row0 = 0; g.n_rows = r.N;
       g.est_us = static_cast<float>(r.H * t_head + 12.0);    // (+ filling and draining the longer chain)
       g.smem_bytes = smem_bytes;
     }
