@@ -316,6 +316,7 @@ struct __align__(8) Barriers {
   uint64_t sfull[kMaxSlots];    // all CTAs' (max, sum) pairs of a head have arrived
   uint64_t fin;                  // add warps meet before / after staging the head sums
   uint64_t ph;                   // add warps meet once per head (per-head maxima of Eq. 10)
+  uint64_t gsent[kMaxBufs];      // grid plans: exp warps -> publishing thread: this CTA's pairs of a head are in global memory
   uint64_t gfull[kMaxGatherSlots];   // filter tail: a gathered row has landed in its slot
 };
 
@@ -389,6 +390,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), p.gx ? 32 : 1);
     mbar_init(smem_u32(&bars.fin), kAddThreads);
     mbar_init(smem_u32(&bars.ph), kAddThreads);
+    for (int s = 0; s < kMaxBufs; ++s) mbar_init(smem_u32(&bars.gsent[s]), kAlt ? kExpWarps / kColGroups : kExpWarps);
     for (int s = 0; s < kMaxGatherSlots; ++s) mbar_init(smem_u32(&bars.gfull[s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -657,7 +659,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         uint32_t* const sent = p.gx_cnt + bh;
         const bool ok = lane != 0 || count_wait(sent, target, abort_flag, wait_limit);
         if (!__all_sync(0xffffffffu, ok)) break;
-        (void)ld_acquire_gpu(sent);            // every lane's own acquire orders its copies below
+        __syncwarp();                          // lane 0's acquire, then the warp's copies
         const unsigned char* const src = reinterpret_cast<const unsigned char*>(p.gx_stats + bh * slot_pairs);
         const uint32_t dst = smem_u32(stats + static_cast<size_t>(slot) * slot_pairs);
         for (uint32_t off = lane * 16u; off < slot_bytes_gx; off += 32u * 16u)
@@ -672,6 +674,17 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         }
       }
       asm volatile("cp.async.wait_all;" ::: "memory");   // no copy of this warp is in flight when the CTA leaves
+    } else if (warp == kMmaWarp + 2 && lane == 0 && p.gx) {
+      // ---------------- publishing thread (grid plans) ----------------
+      // Once all exp warps of this CTA have stored their pairs of a head: one fence, one counted
+      // release - the round trip of the fence is off the exp warps' path.
+      pdl_wait();
+      const uint32_t senders = kAlt ? kExpWarps / kColGroups : kExpWarps;
+      for (int h = 0; h < p.H; ++h) {
+        if (!mbar_wait(smem_u32(&bars.gsent[h % p.n_buf]), static_cast<uint32_t>(h / p.n_buf) & 1u, abort_flag, wait_limit)) break;
+        __threadfence();
+        atomicAdd(p.gx_cnt + static_cast<size_t>(b) * p.H + h, senders);
+      }
     }
     if constexpr (FILTER) {
       // filter tail, TMA / MMA warps: nothing to do but to meet the others
@@ -825,14 +838,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
       if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
       if (p.gx) {
-        // grid plan: the pair goes to global memory; the warp's pairs are published by one counted release
+        // grid plan: the pair goes to global memory; the CTA's pairs of the head are published together
         const size_t bh = static_cast<size_t>(b) * p.H + h;
         if (sender) p.gx_stats[((bh * p.cluster + rank) * NROWS + row) * EPR + (kAlt ? 0 : g)] = make_float2(mx, lsum);
         __syncwarp();
-        if (lane == 0) {
-          __threadfence();
-          atomicAdd(p.gx_cnt + bh, 1u);
-        }
+        if (lane == 0) mbar_arrive(smem_u32(&bars.gsent[buf]));   // (the publishing thread takes the fence off this warp's path)
       } else if (sender) {
         for (int c = 0; c < p.cluster; ++c)
           st_async_f32x2(map_to_cta(slot_addr, c), mx, lsum, map_to_cta(bar_addr, c));
