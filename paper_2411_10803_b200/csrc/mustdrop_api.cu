@@ -221,6 +221,11 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   size_t off = kWsStatusBytes;
   p->ws_rowstats_off = off;
   off += round_up(sizeof(float) * 2 * static_cast<size_t>(r.B) * r.H * r.N, 256);
+#ifdef MUSTDROP_TRACE
+  // trace builds stamp into the workspace from byte 4096 on (up to 32 CTAs per request): keep the
+  // regions the kernels really use clear of that
+  if (off < 4096 + static_cast<size_t>(r.B) * 32 * r.H * 16 * 8) off = round_up(4096 + static_cast<size_t>(r.B) * 32 * r.H * 16 * 8, 256);
+#endif
   p->ws_gx_cnt_off = p->ws_gx_stats_off = off;
   if (p->score_variant == kScoreFusedCluster && p->fused.gx) {
     p->ws_gx_cnt_off = off;

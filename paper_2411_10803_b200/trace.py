@@ -63,8 +63,8 @@ def main(argv) -> int:
         text = ctypes.create_string_buffer(256)
         L.mustdrop_plan_describe(plan, text, 256)
         print(text.value.decode())
-        n_cta = w.batch * 16
-        ws = torch.zeros(4096 + n_cta * w.n_heads * 16 * 8, dtype=torch.uint8, device="cuda")
+        n_cta = w.batch * 32
+        ws = torch.zeros(max(int(ws_bytes.value), 4096 + n_cta * w.n_heads * 16 * 8), dtype=torch.uint8, device="cuda")
         stream = torch.cuda.current_stream().cuda_stream
         if whole:
             v = torch.from_numpy(host["v"].view(np.int16)).cuda()
@@ -86,7 +86,7 @@ def main(argv) -> int:
             if st != 0:
                 raise RuntimeError("call refused: %d" % st)
             torch.cuda.synchronize()
-        t = ws[4096:].cpu().numpy().view(np.uint64).reshape(n_cta, w.n_heads, 16).astype(np.float64)
+        t = ws[4096:4096 + n_cta * w.n_heads * 16 * 8].cpu().numpy().view(np.uint64).reshape(n_cta, w.n_heads, 16).astype(np.float64)
     used = [c for c in range(n_cta) if t[c, 0, 0] > 0]
     if not used:
         print("no stamps: the plan does not use the fused kernel")
