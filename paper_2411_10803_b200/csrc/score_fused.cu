@@ -1383,8 +1383,12 @@ bool plan_score_grid(const Resolved& r, int sm_count, int forced_ctas, FusedGeom
     if (2 * slot + 2 * stage > avail) continue;
     int n_q = static_cast<int>((avail - 2 * slot) / stage);
     if (n_q > 3) n_q = 3;
+    // (No more slots than buffers: the fetch warp learns that a slot is free from the buffer barrier
+    // of the head that used it, by parity; were it n_buf heads behind the add warps, that barrier
+    // could complete a second phase unseen.)
     int n_slot = static_cast<int>((avail - n_q * stage) / slot);
     if (n_slot > 4) n_slot = 4;
+    if (n_slot > n_buf) n_slot = n_buf;
     size_t smem_bytes = n_q * stage + n_slot * slot + 1024 + ph_bytes;
     if (smem_bytes < 116 * 1024) smem_bytes = 116 * 1024;
     // Cost per head and CTA (microseconds): streaming the stage at ~45 GB/s per SM; the exp stage
