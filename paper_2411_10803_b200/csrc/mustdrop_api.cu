@@ -433,8 +433,8 @@ int32_t mustdrop_plan_describe(const mustdrop_plan_t* plan, char* buf, size_t n)
     if (g.gx)
       len = std::snprintf(text, sizeof(text),
                           "fused tcgen05 score: grid plan (statistics through global memory), %d CTAs per request, "
-                          "%d keys per CTA, stages %d, %d tensor-memory buffers; filter = %d launch(es)",
-                          g.cluster, g.tk, g.n_q, g.n_buf, mustdrop_plan_filter_launches(plan));
+                          "%d keys per CTA, stages %d, %d tensor-memory buffers, %d statistics slots; filter = %d launch(es)",
+                          g.cluster, g.tk, g.n_q, g.n_buf, g.n_slot, mustdrop_plan_filter_launches(plan));
     else
       len = std::snprintf(text, sizeof(text),
                           "fused tcgen05 score%s: cluster %d, %d keys per CTA, %s %d/%d, %d tensor-memory buffers, "

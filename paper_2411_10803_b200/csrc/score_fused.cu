@@ -372,9 +372,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const size_t staging = p.split ? static_cast<size_t>(p.n_q) * q_bytes + static_cast<size_t>(p.n_k) * kh_bytes
                                  : static_cast<size_t>(p.n_q) * stage_bytes;
   float2* stats = reinterpret_cast<float2*>(stage_ptr + staging);
-  const uint32_t slot_pairs = static_cast<uint32_t>(p.cluster) * NROWS * EPR;   // pairs per slot
+  // pairs per slot: EPR per text row and CTA; grid plans merge a CTA's pairs of a row before they
+  // leave the CTA (one pair per row and CTA crosses global memory and fills the slots)
+  const uint32_t slot_pairs = static_cast<uint32_t>(p.cluster) * NROWS * (p.gx ? 1 : EPR);
   // PH only: [2][4 add warps][tk] per-head column maxima of each warp's text rows, double-buffered over heads
   float* const ph_stage = reinterpret_cast<float*>(stats + static_cast<size_t>(p.n_slot) * slot_pairs);
+  // grid plans only: [n_buf][rows][EPR] the pairs of this CTA's own exp warps, per tensor-memory buffer
+  float2* const own_pairs = reinterpret_cast<float2*>(ph_stage + (PH ? 2 * kAddWarps * p.tk : 0));
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
@@ -645,7 +649,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       // statistics in shared memory exactly as with a cluster, and the round trips to L2 are off
       // their path.  A slot is reused once the add warps are done with the head that used it.
       pdl_wait();   // the counters belong to the workspace: an earlier call may still be resetting them
-      const uint32_t target = static_cast<uint32_t>(p.cluster) * (kAlt ? kExpWarps / kColGroups : kExpWarps);
+      const uint32_t target = static_cast<uint32_t>(p.cluster);   // one counted release per CTA and head
       const uint32_t slot_bytes_gx = slot_pairs * 8u;
       for (int h = 0; h < p.H; ++h) {
         const int slot = h % p.n_slot;
@@ -674,16 +678,35 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         }
       }
       asm volatile("cp.async.wait_all;" ::: "memory");   // no copy of this warp is in flight when the CTA leaves
-    } else if (warp == kMmaWarp + 2 && lane == 0 && p.gx) {
-      // ---------------- publishing thread (grid plans) ----------------
-      // Once all exp warps of this CTA have stored their pairs of a head: one fence, one counted
-      // release - the round trip of the fence is off the exp warps' path.
-      pdl_wait();
-      const uint32_t senders = kAlt ? kExpWarps / kColGroups : kExpWarps;
+    } else if (warp == kMmaWarp + 2 && p.gx) {
+      // ---------------- publishing warp (grid plans) ----------------
+      // Once all exp warps of this CTA have left their pairs of a head in shared memory: merge the
+      // pairs of each row into one, store it to global memory, then one fence and one counted
+      // release for the CTA - the round trip of the fence is off the exp warps' path.
+      pdl_wait();   // global memory of the workspace: not before the stream's earlier work is done
       for (int h = 0; h < p.H; ++h) {
-        if (!mbar_wait(smem_u32(&bars.gsent[h % p.n_buf]), static_cast<uint32_t>(h / p.n_buf) & 1u, abort_flag, wait_limit)) break;
-        __threadfence();
-        atomicAdd(p.gx_cnt + static_cast<size_t>(b) * p.H + h, senders);
+        const int buf = h % p.n_buf;
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.gsent[buf]), static_cast<uint32_t>(h / p.n_buf) & 1u,
+                                               abort_flag, wait_limit)))
+          break;
+        const size_t bh = static_cast<size_t>(b) * p.H + h;
+        float2* const dst = p.gx_stats + (bh * p.cluster + rank) * NROWS;
+        for (int r = lane; r < NROWS; r += 32) {
+          const float2* const pr = own_pairs + (buf * NROWS + r) * EPR;
+          float2 v = pr[0];
+          if (EPR == 2) {
+            const float2 w2 = pr[EPR - 1];
+            const float m2 = fmaxf(v.x, w2.x);
+            const float ref = (m2 == -INFINITY) ? 0.0f : m2;
+            v = make_float2(m2, v.y * ex2(v.x - ref) + w2.y * ex2(w2.x - ref));   // an empty pair is (-inf, 0)
+          }
+          dst[r] = v;
+        }
+        __syncwarp();
+        if (lane == 0) {
+          __threadfence();
+          atomicAdd(p.gx_cnt + bh, 1u);
+        }
       }
     }
     if constexpr (FILTER) {
@@ -712,7 +735,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const uint32_t pair_idx = (rank * NROWS + row) * EPR + (kAlt ? 0 : g);     // this thread's pair in a slot
 
     int last_buf = -1;
-    if (p.gx) pdl_wait();   // the statistics go through global memory: not before the stream's earlier work is done
     for (int h = kAlt ? g : 0; h < p.H; h += kAlt ? kColGroups : 1) {
       const int buf = h % p.n_buf;
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
@@ -838,11 +860,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
       if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
       if (p.gx) {
-        // grid plan: the pair goes to global memory; the CTA's pairs of the head are published together
-        const size_t bh = static_cast<size_t>(b) * p.H + h;
-        if (sender) p.gx_stats[((bh * p.cluster + rank) * NROWS + row) * EPR + (kAlt ? 0 : g)] = make_float2(mx, lsum);
+        // grid plan: the pair stays in this CTA's shared memory; the publishing warp merges the CTA's
+        // pairs of a row and sends one pair per row on its way through global memory
+        if (sender) own_pairs[(buf * NROWS + row) * EPR + (kAlt ? 0 : g)] = make_float2(mx, lsum);
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars.gsent[buf]));   // (the publishing thread takes the fence off this warp's path)
+        if (lane == 0) mbar_arrive(smem_u32(&bars.gsent[buf]));
       } else if (sender) {
         for (int c = 0; c < p.cluster; ++c)
           st_async_f32x2(map_to_cta(slot_addr, c), mx, lsum, map_to_cta(bar_addr, c));
@@ -915,9 +937,23 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const int slot = h % p.n_slot;
       const uint32_t sph = static_cast<uint32_t>(h / p.n_slot) & 1u;
       float f[EPR];                            // factor of each of this CTA's pairs
-      {
-        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag, wait_limit))) break;
-        if (tid_a == 0) MD_TRACE(h, 5);
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag, wait_limit))) break;
+      if (tid_a == 0) MD_TRACE(h, 5);
+      if (p.gx) {
+        // grid plan: one merged pair per CTA in the slot; this CTA's own stabilisers are still in
+        // its shared memory (until the buffer is released below)
+        const float2* srow = stats + slot * slot_pairs + row;
+        float m = -INFINITY;
+        for (int c = 0; c < p.cluster; ++c) m = fmaxf(m, srow[c * NROWS].x);
+        float l = 0.0f;
+        for (int c = 0; c < p.cluster; ++c) {
+          const float2 v = srow[c * NROWS];
+          l = fmaf(v.y, ex2(v.x - m), l);
+        }
+        const float inv_l = 1.0f / l;
+#pragma unroll
+        for (int x = 0; x < EPR; ++x) f[x] = ex2(own_pairs[(buf * NROWS + row) * EPR + x].x - m) * inv_l;
+      } else {
         // statistics of this row over the whole key range: every CTA's pairs
         const float2* srow = stats + slot * slot_pairs + row * EPR;
         float m = -INFINITY;
@@ -1379,17 +1415,18 @@ bool plan_score_grid(const Resolved& r, int sm_count, int forced_ctas, FusedGeom
     // shared memory: statistics slots the fetch warp fills (a head's pairs of all the request's
     // CTAs; at least two, so that the next head's are fetched while this one is added) and stages
     const int epr = ach <= 5 ? 1 : kColGroups;
-    const size_t slot = static_cast<size_t>(c) * nrows * epr * 8;
-    if (2 * slot + 2 * stage > avail) continue;
-    int n_q = static_cast<int>((avail - 2 * slot) / stage);
+    const size_t slot = static_cast<size_t>(c) * nrows * 8;                 // one merged pair per row and CTA
+    const size_t own = static_cast<size_t>(n_buf) * nrows * epr * 8;        // the CTA's own pairs, per buffer
+    if (avail < own + 2 * slot + 2 * stage) continue;
+    int n_q = static_cast<int>((avail - own - 2 * slot) / stage);
     if (n_q > 3) n_q = 3;
     // (No more slots than buffers: the fetch warp learns that a slot is free from the buffer barrier
     // of the head that used it, by parity; were it n_buf heads behind the add warps, that barrier
     // could complete a second phase unseen.)
-    int n_slot = static_cast<int>((avail - n_q * stage) / slot);
-    if (n_slot > 4) n_slot = 4;
+    int n_slot = static_cast<int>((avail - own - n_q * stage) / slot);
+    if (n_slot > 6) n_slot = 6;
     if (n_slot > n_buf) n_slot = n_buf;
-    size_t smem_bytes = n_q * stage + n_slot * slot + 1024 + ph_bytes;
+    size_t smem_bytes = n_q * stage + n_slot * slot + own + 1024 + ph_bytes;
     if (smem_bytes < 116 * 1024) smem_bytes = 116 * 1024;
     // Cost per head and CTA (microseconds): streaming the stage at ~45 GB/s per SM; the exp stage
     // (measured: ~0.011 us per column of a lane, two heads at a time on narrow tiles); the
@@ -1416,8 +1453,7 @@ bool plan_score_grid(const Resolved& r, int sm_count, int forced_ctas, FusedGeom
 
 size_t grid_plan_stats_bytes(const Resolved& r, const FusedGeometry& g) {
   const int nrows = 128 / g.halves;
-  const int epr = g.ach <= 5 ? 1 : kColGroups;
-  return static_cast<size_t>(r.B) * r.H * g.cluster * nrows * epr * sizeof(float2);
+  return static_cast<size_t>(r.B) * r.H * g.cluster * nrows * sizeof(float2);   // one merged pair per row, CTA and head
 }
 
 namespace {
