@@ -117,6 +117,7 @@ __global__ void __launch_bounds__(kThreads) spatial_merge_kernel(MergeParams p) 
     const uint4* r2 = r0 + static_cast<size_t>(g) * p.vecs; // (y+1, x)
     const uint4* r3 = r2 + p.vecs;
     float n0 = 0, n1 = 0, n2 = 0, n3 = 0, d01 = 0, d02 = 0, d03 = 0, d12 = 0, d13 = 0, d23 = 0;
+#pragma unroll 2
     for (int x = lane; x < p.vecs; x += 32) {
       const uint4 a = r0[x], c = r1[x], e = r2[x], f = r3[x];
       const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
@@ -199,7 +200,16 @@ __global__ void __launch_bounds__(kThreads) spatial_merge_kernel(MergeParams p) 
     const uint4* r0 = in + static_cast<size_t>(s) * p.vecs;
     uint4* dst = out + static_cast<size_t>(o) * p.vecs;
     if (!m) {
-      for (int v = lane; v < p.vecs; v += 32) dst[v] = r0[v];
+      // a copy: four independent 16-byte loads in flight per lane, then the stores
+      for (int v0 = lane; v0 < p.vecs; v0 += 4 * 32) {
+        uint4 t[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (v0 + 32 * u < p.vecs) t[u] = r0[v0 + 32 * u];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (v0 + 32 * u < p.vecs) dst[v0 + 32 * u] = t[u];
+      }
     } else {
       const uint4* r1 = r0 + p.vecs;
       const uint4* r2 = r0 + static_cast<size_t>(g) * p.vecs;
