@@ -927,7 +927,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     float ph_acc[PHK];
 #pragma unroll
     for (int x = 0; x < PHK; ++x) ph_acc[x] = 0.0f;
-    const unsigned grp_mask = (HALVES == 2) ? (half ? 0xffff0000u : 0x0000ffffu) : 0xffffffffu;   // lanes sharing a key range
     const bool real_row = row < p.N;     // lanes beyond the text rows carry padding
 
     int h = 0;
@@ -991,21 +990,34 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             for (int j = 0; j < kChunk; ++j) acc[c0 + 1][j] = fmaf(e[1][j], f1, acc[c0 + 1][j]);
           }
           if constexpr (PH) {
-            // column maxima over this warp's text rows: probabilities are >= 0, so their bit
-            // patterns order like unsigned integers and one warp reduction per column does it;
-            // lane j of the group keeps column j's result and stores it for the other warps
+            // Column maxima over this warp's text rows (the lanes): recursive halving - in each of
+            // four steps a lane keeps half of its columns and takes its partner's maxima for them,
+            // so that after 8 + 4 + 2 + 1 shuffles lane j of a 16-lane group holds column j's maximum
+            // over the group (about one shuffle per column).  With 128 text rows the two 16-lane
+            // groups of a warp hold the same columns and are folded first.
             float* const dst = ph_stage + ((h & 1) * kAddWarps + q) * p.tk + half * p.cpl + (lane & 15);
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
               if (c0 + x < ACH && c0 + x < total_chunks) {
                 const float fx = real_row ? (x ? f1 : f0) : 0.0f;
-                unsigned mine = 0u;
+                float v[kChunk];
 #pragma unroll
-                for (int j = 0; j < kChunk; ++j) {
-                  const unsigned m = __reduce_max_sync(grp_mask, __float_as_uint(e[x][j] * fx));
-                  mine = ((lane & 15) == j) ? m : mine;
+                for (int j = 0; j < kChunk; ++j) v[j] = e[x][j] * fx;
+                if (HALVES == 1) {
+#pragma unroll
+                  for (int j = 0; j < kChunk; ++j) v[j] = fmaxf(v[j], __shfl_xor_sync(0xffffffffu, v[j], 16));
                 }
-                if (HALVES == 2 || lane < 16) dst[kChunk * (c0 + x)] = __uint_as_float(mine);
+#pragma unroll
+                for (int step = kChunk / 2; step >= 1; step >>= 1) {
+                  const bool upper = (lane & step) != 0;
+#pragma unroll
+                  for (int i = 0; i < step; ++i) {
+                    const float give = upper ? v[i] : v[i + step];
+                    const float keep = upper ? v[i + step] : v[i];
+                    v[i] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, step));
+                  }
+                }
+                if (HALVES == 2 || lane < 16) dst[kChunk * (c0 + x)] = v[0];
               }
             }
           }
