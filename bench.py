@@ -222,7 +222,10 @@ class BufferSets:
     rotated by r places (distinct addresses and a distinct request order: what matters to the caches
     is the address, and every set is a valid instance of the workload)."""
 
-    def __init__(self, torch, md, w, host, dev, l2_bytes, flags=0, max_sets=96):
+    MAX_SETS = 96      # (--max-sets: a profiler capture wants little memory on the device)
+
+    def __init__(self, torch, md, w, host, dev, l2_bytes, flags=0, max_sets=None):
+        max_sets = BufferSets.MAX_SETS if max_sets is None else max_sets
         bm = bytes_model(w)
         streams = [bm["score"], bm["headline"] - (bm["score"] - 2 * w.batch * w.n_vis * 4)]   # K + Q read; rows written
         need = max(4.0 * l2_bytes / max(b, 1) for b in streams)
@@ -799,6 +802,8 @@ def main():
                     help="filter: the one-call entry point; staged: score, select and compact as three calls")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="the K timed steps are repeated in rounds until the timed span exceeds this")
+    ap.add_argument("--max-sets", type=int, default=96,
+                    help="upper limit on the rotating buffer sets (for profiler captures, which want a small footprint)")
     ap.add_argument("--kernel-hash", action="store_true", help="print the fingerprint of the kernel sources and exit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the short runs of the other listed configurations")
@@ -810,6 +815,7 @@ def main():
     if args.kernel_hash:
         print(kernel_source_hash())
         return
+    BufferSets.MAX_SETS = max(2, args.max_sets)
     w = synth.WORKLOADS[args.workload]
     if args.budget:
         w = w.with_(budget=args.budget)
