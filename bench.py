@@ -391,6 +391,7 @@ def run_ours(args, w):
     # every rank filters its own batch of w.batch requests (distinct request numbers per rank)
     reqs = range(rank * w.batch, (rank + 1) * w.batch)
     host = synth.make_batch(w, requests=reqs)
+    input_sha256 = {n: synth.sha256_of(host[n])[:16] for n in ("q_text", "k", "v", "hidden", "key_idx")} if rank == 0 else None
     sets = BufferSets(torch, md, w, host, dev, l2_bytes)
     f = sets.filters[0]
     stream = torch.cuda.current_stream()
@@ -547,6 +548,7 @@ def run_ours(args, w):
                              "address repeats, %.0f MB of keys + queries are read and %.0f MB of rows written "
                              "(L2: %.0f MB)" % (sets.n, sets.footprints_mb[0], sets.footprints_mb[1], l2_bytes / 1e6),
                        "buffer_sets": sets.n,
+                       "input_sha256": input_sha256,      # first 16 hex digits, rank 0's batch (seeded: the same on every run)
                        "timing": "median of %d rounds of %d steps (%.2f s timed), each round between two events" % (
                            len(rounds), K, sum(rounds) * K / 1e3),
                        "score_variant": f.score_variant, "plan": f.description,

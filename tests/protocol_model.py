@@ -14,6 +14,12 @@ slots) and the bounded waits: a wait that runs out raises the CTA's abort flag, 
 of that CTA then returns at once, the CTA records a time-out, tells its peers before the exit
 barrier of the cluster, and the request is marked invalid (kept_cnt = -1).
 
+Grid plans (``grid=True``): the CTAs of the request are no cluster; the exp role leaves its pair in
+the CTA's own memory and arrives on ``gsent``; a publishing role stores the pair to (modelled)
+global memory and adds one to the head's counter; a fetch role waits until the counter shows every
+CTA, copies the head's pairs into a statistics slot and completes the slot's barrier - it learns
+that a slot is free from the buffer barrier (``tempty``) of the head that used it, by parity.
+
 The model checks what the kernel relies on: no statistics slot is written before its previous
 content has been read, no buffer is refilled before it was released, every head is processed
 exactly once per CTA, and a missing arrive ends in a clean time-out everywhere instead of a hang.
@@ -73,6 +79,8 @@ class Cta:
         self.eready = [Mbarrier(1) for _ in range(geo["n_buf"])]
         self.tempty = [Mbarrier(1) for _ in range(geo["n_buf"])]
         self.sfull = [Mbarrier(1) for _ in range(geo["n_slot"])]
+        self.gsent = [Mbarrier(1) for _ in range(geo["n_buf"])]     # grid plans: exp role -> publishing role
+        self.own_pair = [None] * geo["n_buf"]
         self.stats = [[None] * geo["C"] for _ in range(geo["n_slot"])]   # head whose pair sits there
         self.stage_head = [None] * geo["n_q"]
         self.buf_state = [("free", None)] * geo["n_buf"]
@@ -94,8 +102,13 @@ class Cluster:
     """One request: C CTAs x 4 roles.  fault = (rank, role, head, what) makes that role skip one
     arrive ("full", "tfull", "eready", "tempty", "empty") or one statistics store ("stats")."""
 
-    def __init__(self, C=2, H=12, n_q=2, n_buf=3, n_slot=None, tight=0, limit=0.25, fault=None, jitter=None):
-        n_slot = 2 * n_buf if n_slot is None else n_slot
+    def __init__(self, C=2, H=12, n_q=2, n_buf=3, n_slot=None, tight=0, limit=0.25, fault=None, jitter=None,
+                 grid=False):
+        n_slot = (min(n_buf, 4) if grid else 2 * n_buf) if n_slot is None else n_slot
+        self.grid = grid
+        self.g_lock = threading.Lock()
+        self.g_cnt = [0] * H                       # global memory: pairs published per head
+        self.g_pairs = [[None] * C for _ in range(H)]
         self.geo = dict(C=C, H=H, n_q=n_q, n_buf=n_buf, n_slot=n_slot, tight=tight)
         self.limit, self.fault, self.jitter = limit, fault, jitter or {}
         self.ctas = [Cta(self, r, self.geo) for r in range(C)]
@@ -155,12 +168,19 @@ class Cluster:
                     return
             if not c.wait(c.tfull[buf], (h // g["n_buf"]) & 1, self.limit):
                 return
-            c.sfull[slot].arrive(expect_tx=g["C"])        # arm: every CTA will send one pair
+            if not self.grid:
+                c.sfull[slot].arrive(expect_tx=g["C"])    # arm: every CTA will send one pair
             self._pause(c.rank, "exp")
             if c.buf_state[buf] != ("logits", h):
                 raise ProtocolError("exp role of head %d found %s" % (h, c.buf_state[buf],))
             c.buf_state[buf] = ("exps", h)
-            if not self._skips(c.rank, "exp", h, "stats"):
+            if self.grid:
+                if c.own_pair[buf] is not None:
+                    raise ProtocolError("own pair of buffer %d overwritten before head %s was added" % (buf, c.own_pair[buf]))
+                c.own_pair[buf] = h
+                if not self._skips(c.rank, "exp", h, "stats"):
+                    c.gsent[buf].arrive()
+            elif not self._skips(c.rank, "exp", h, "stats"):
                 for peer in self.ctas:                    # st.async into every CTA, counted on ITS barrier
                     with peer.guard:
                         if peer.stats[slot][c.rank] is not None:
@@ -181,6 +201,10 @@ class Cluster:
                 if c.stats[slot] != [h] * g["C"]:
                     raise ProtocolError("add role of head %d read pairs of heads %s" % (h, c.stats[slot]))
                 c.stats[slot] = [None] * g["C"]
+                if self.grid:
+                    if c.own_pair[buf] != h:
+                        raise ProtocolError("add role of head %d found own pair of head %s" % (h, c.own_pair[buf]))
+                    c.own_pair[buf] = None
             if not c.wait(c.eready[buf], (h // g["n_buf"]) & 1, self.limit):
                 return
             self._pause(c.rank, "add")
@@ -190,6 +214,44 @@ class Cluster:
             c.added.append(h)
             if not self._skips(c.rank, "add", h, "tempty"):
                 c.tempty[buf].arrive()
+
+    def publish(self, c):
+        g = self.geo
+        for h in range(g["H"]):
+            buf = h % g["n_buf"]
+            if not c.wait(c.gsent[buf], (h // g["n_buf"]) & 1, self.limit):
+                return
+            self._pause(c.rank, "publish")
+            with self.g_lock:
+                self.g_pairs[h][c.rank] = h
+                if not self._skips(c.rank, "publish", h, "count"):
+                    self.g_cnt[h] += 1
+
+    def fetch(self, c):
+        g = self.geo
+        for h in range(g["H"]):
+            slot = h % g["n_slot"]
+            self._pause(c.rank, "fetch_late")       # (a fetch role that gets to its next head late)
+            if h >= g["n_slot"]:
+                u = h - g["n_slot"]
+                if not c.wait(c.tempty[u % g["n_buf"]], (u // g["n_buf"]) & 1, self.limit):
+                    return
+            t0 = time.monotonic()
+            while True:
+                with self.g_lock:
+                    if self.g_cnt[h] >= g["C"]:
+                        break
+                if c.abort or time.monotonic() - t0 > self.limit:
+                    c.abort = True
+                    return
+                time.sleep(0.0002)
+            self._pause(c.rank, "fetch")
+            with c.guard:
+                if c.stats[slot] != [None] * g["C"]:
+                    raise ProtocolError("slot %d of CTA %d refilled for head %d before heads %s were read"
+                                        % (slot, c.rank, h, c.stats[slot]))
+                c.stats[slot] = list(self.g_pairs[h])
+            c.sfull[slot].arrive()
 
     # ---- a run ---------------------------------------------------------------------------------------
     def run(self, join_limit=20.0):
@@ -201,8 +263,9 @@ class Cluster:
                 self.errors.append(str(e))
                 c.abort = True
 
+        roles = (self.tma, self.mma, self.exp, self.add) + ((self.publish, self.fetch) if self.grid else ())
         threads = [threading.Thread(target=guarded, args=(fn, c), daemon=True)
-                   for c in self.ctas for fn in (self.tma, self.mma, self.exp, self.add)]
+                   for c in self.ctas for fn in roles]
         for t in threads:
             t.start()
         t_end = time.monotonic() + join_limit

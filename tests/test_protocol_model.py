@@ -62,3 +62,49 @@ def test_a_skipped_arrive_times_out_everywhere(fault, tight):
     assert all(c.status == TIMEOUT for c in cl.ctas)         # every CTA of the cluster reports the time-out
     assert cl.cluster_abort and cl.kept_cnt == -1            # and the request is marked invalid
     assert all(len(c.added) < 12 for c in cl.ctas)
+
+
+# ---- grid plans: statistics through (modelled) global memory, publishing and fetch roles -----------
+
+GRID_GEOMETRIES = [
+    dict(C=2, n_q=2, n_buf=3),                # slots default to min(buffers, 4)
+    dict(C=6, n_q=3, n_buf=5, n_slot=3),
+    dict(C=17, n_q=2, n_buf=4, n_slot=4),     # the video workload's plan
+    dict(C=5, n_q=4, n_buf=8, n_slot=6),
+]
+
+
+@pytest.mark.parametrize("geo", GRID_GEOMETRIES, ids=lambda g: "C%d_b%d_s%s" % (g["C"], g["n_buf"], g.get("n_slot", "d")))
+def test_grid_protocol_completes_and_keeps_its_invariants(geo):
+    cl = Cluster(H=13, limit=5.0, grid=True, **geo)
+    assert cl.run(), "a role never came back"
+    assert cl.errors == []
+    for c in cl.ctas:
+        assert c.status == OK and c.added == list(range(13))
+
+
+@pytest.mark.parametrize("slow", [(0, "fetch"), (0, "fetch_late"), (1, "publish"), (0, "add"), (1, "exp")])
+def test_grid_protocol_tolerates_a_slow_role(slow):
+    cl = Cluster(C=3, H=10, n_q=2, n_buf=3, limit=5.0, grid=True, jitter={slow: 0.01})
+    assert cl.run() and cl.errors == []
+    assert all(c.added == list(range(10)) for c in cl.ctas)
+
+
+def test_more_slots_than_buffers_stalls_the_fetch_role():
+    # the fetch role reads "slot free" off the parity of a buffer barrier: with four slots on three
+    # buffers the add role can finish a second head on that buffer before a slow fetch role looks,
+    # the parity is back where it was, and the wait runs out (seen once on the GPU: 0.1 s per call).
+    # With no more slots than buffers the same slow role is harmless (test above).
+    cl = Cluster(C=2, H=16, n_q=2, n_buf=3, n_slot=4, limit=0.3, grid=True, jitter={(0, "fetch_late"): 0.02})
+    assert cl.run(join_limit=15.0), "a role hung instead of giving up"
+    assert cl.cluster_abort and cl.kept_cnt == -1
+
+
+@pytest.mark.parametrize("fault", [(1, "publish", 3, "count"), (0, "exp", 2, "stats"), (1, "add", 4, "tempty")],
+                         ids=lambda f: "cta%d_%s_h%d_%s" % f)
+def test_grid_protocol_times_out_everywhere_after_a_skipped_signal(fault):
+    cl = Cluster(C=3, H=12, n_q=2, n_buf=3, limit=0.2, fault=fault, grid=True)
+    assert cl.run(join_limit=10.0), "a role hung instead of giving up"
+    assert cl.errors == []
+    assert all(c.status == TIMEOUT for c in cl.ctas)
+    assert cl.kept_cnt == -1
