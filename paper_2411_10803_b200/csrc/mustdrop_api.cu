@@ -229,7 +229,7 @@ mustdrop_status_t mustdrop_filter_plan(const mustdrop_config_t* c, mustdrop_plan
   p->ws_gx_cnt_off = p->ws_gx_stats_off = off;
   if (p->score_variant == kScoreFusedCluster && p->fused.gx) {
     p->ws_gx_cnt_off = off;
-    off += round_up(sizeof(uint32_t) * (2 * static_cast<size_t>(r.B) * r.H + 2 * static_cast<size_t>(r.B)), 256);
+    off += round_up(sizeof(uint32_t) * (static_cast<size_t>(r.B) * r.H + 3 * static_cast<size_t>(r.B)), 256);
     p->ws_gx_stats_off = off;
     off += round_up(grid_plan_stats_bytes(r, p->fused), 256);
   }

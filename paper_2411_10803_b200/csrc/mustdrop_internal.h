@@ -89,7 +89,7 @@ struct mustdrop_plan {
   int32_t score_variant;
   size_t ws_bytes;
   size_t ws_rowstats_off;   // float2 [B,H,N]: (row max in log2 units, 1 / row sum)
-  size_t ws_gx_cnt_off;     // grid plans: uint32 counters [2 B H + 2 B], zero between calls
+  size_t ws_gx_cnt_off;     // grid plans: uint32 counters [B H + 3 B], zero between calls
   size_t ws_gx_stats_off;   // grid plans: float2 [B,H,CTAs per request,rows,pairs]
   mustdrop::FusedGeometry fused;
   int32_t row_split;        // 1: the text rows are scored by two launches (fused: rows 0..63, fused_b: the rest)

@@ -73,7 +73,7 @@ struct FusedParams {
   // the CTAs of a request are ordinary CTAs of the grid, any number of them, all resident at once).
   int32_t gx;                         // 1: grid plan (cluster = CTAs per request, launched without a cluster)
   float2* gx_stats;                   // [B][H][CTAs per request][rows][pairs] (stabiliser, sum)
-  uint32_t* gx_cnt;                   // [B*H] pairs sent, [B*H] readers done, [B] scores stored, [B] barrier passed; zero between calls
+  uint32_t* gx_cnt;                   // [B*H] CTAs that published a head, [B] scores stored, [B] barrier passed, [B] CTAs that left; zero between calls
   int32_t per_head;                   // 1: i_out = head mean of the per-head maxima over the text rows (PH instantiations)
   int32_t early_inputs;               // 1: q_text / k may be read before the stream's earlier work has completed (caller's promise)
   long long wait_cycles;              // clock cycles after which a wait between the warp roles gives up
@@ -439,9 +439,20 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       // counter in global memory: every CTA's scores are stored before any CTA selects.  (A CTA
       // that gives up tells nobody: its peers run into their own limits.)
       if (threadIdx.x == 0) {
+        const size_t n_req = gridDim.x / p.cluster;
+        if (*abort_flag == 0) {
+          // every CTA has seen all of its heads complete when it gets here: the last one of the
+          // request to do so clears the heads' counters for the next call (one counted visit per
+          // CTA instead of one per head, whose returned value the fetch warp would have to wait for)
+          uint32_t* const left = p.gx_cnt + n_req * p.H + 2 * n_req + b;
+          if (atomicAdd(left, 1u) == static_cast<uint32_t>(p.cluster) - 1u) {
+            for (int hh = 0; hh < p.H; ++hh) p.gx_cnt[static_cast<size_t>(b) * p.H + hh] = 0u;
+            *left = 0u;
+          }
+        }
         if (FILTER && *abort_flag == 0) {
-          uint32_t* const stored = p.gx_cnt + 2 * static_cast<size_t>(gridDim.x / p.cluster) * p.H + b;
-          uint32_t* const passed = stored + gridDim.x / p.cluster;
+          uint32_t* const stored = p.gx_cnt + n_req * p.H + b;
+          uint32_t* const passed = stored + n_req;
           __threadfence();
           atomicAdd(stored, 1u);
           if (count_wait(stored, static_cast<uint32_t>(p.cluster), abort_flag, wait_limit) &&
@@ -651,6 +662,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       pdl_wait();   // the counters belong to the workspace: an earlier call may still be resetting them
       const uint32_t target = static_cast<uint32_t>(p.cluster);   // one counted release per CTA and head
       const uint32_t slot_bytes_gx = slot_pairs * 8u;
+      int ready = 0;   // heads below this one are known to be published by every CTA of the request
       for (int h = 0; h < p.H; ++h) {
         const int slot = h % p.n_slot;
         if (h >= p.n_slot) {
@@ -660,22 +672,27 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             break;
         }
         const size_t bh = static_cast<size_t>(b) * p.H + h;
-        uint32_t* const sent = p.gx_cnt + bh;
-        const bool ok = lane != 0 || count_wait(sent, target, abort_flag, wait_limit);
-        if (!__all_sync(0xffffffffu, ok)) break;
-        __syncwarp();                          // lane 0's acquire, then the warp's copies
+        if (h >= ready) {
+          // one round trip tells about 32 heads: lane i looks at the counter of head h + i, and
+          // the run of complete heads from h on is taken in one go
+          const uint32_t* const mine = p.gx_cnt + static_cast<size_t>(b) * p.H + (h + lane < p.H ? h + lane : p.H - 1);
+          const long long t0 = clock64();
+          bool ok = true;
+          for (;;) {
+            const bool full = ld_acquire_gpu(mine) >= target;
+            const unsigned not_full = __ballot_sync(0xffffffffu, !(full && h + lane < p.H));
+            const int run = not_full == 0u ? 32 : __ffs(not_full) - 1;
+            if (run > 0) { ready = h + run; break; }
+            if (*abort_flag != 0 || clock64() - t0 > wait_limit) { *abort_flag = 1; ok = false; }
+            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+          }
+          if (!ok) break;
+        }
         const unsigned char* const src = reinterpret_cast<const unsigned char*>(p.gx_stats + bh * slot_pairs);
         const uint32_t dst = smem_u32(stats + static_cast<size_t>(slot) * slot_pairs);
         for (uint32_t off = lane * 16u; off < slot_bytes_gx; off += 32u * 16u)
           asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + off), "l"(src + off) : "memory");
         asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&bars.sfull[slot])) : "memory");
-        if (lane == 0) {   // the last CTA to have seen the head complete leaves its counters as the next call expects them
-          uint32_t* const done = sent + static_cast<size_t>(gridDim.x / p.cluster) * p.H;
-          if (atomicAdd(done, 1u) == static_cast<uint32_t>(p.cluster) - 1u) {
-            *sent = 0u;
-            *done = 0u;
-          }
-        }
       }
       asm volatile("cp.async.wait_all;" ::: "memory");   // no copy of this warp is in flight when the CTA leaves
     } else if (warp == kMmaWarp + 2 && p.gx) {
