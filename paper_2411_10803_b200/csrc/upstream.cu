@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
     __syncthreads();
     const uint4* kh = p.k + (static_cast<size_t>(b) * p.H + h) * M * dv;
     // Coalesced rows: a group of `grp` lanes (the power of two >= D/8) reads one token's row as
-    // 16-byte vectors; a warp takes 32/grp consecutive tokens per step, two steps in flight.  Each
+    // 16-byte vectors; a warp takes 32/grp consecutive tokens per step, four steps in flight.  Each
     // lane keeps its eight query values in registers for the whole head.
     int grp = 1;
     while (grp < dv) grp <<= 1;
@@ -278,26 +278,32 @@ __global__ void __launch_bounds__(kThreads) key_set_kernel(KeySetParams p) {
     for (int e = 0; e < 8; ++e) qv[e] = sub < dv ? q_s[sub * 8 + e] : 0.0f;
     float mx = -INFINITY;
     const int step = kWarps * per_warp;
-    for (int base = warp * per_warp; base < M; base += 2 * step) {   // warp-uniform trip count
-      const int ja = base + tok_in_warp, jb = ja + step;
-      uint4 ka = make_uint4(0, 0, 0, 0), kb = make_uint4(0, 0, 0, 0);
-      if (ja < M && sub < dv) ka = kh[static_cast<size_t>(ja) * dv + sub];
-      if (jb < M && sub < dv) kb = kh[static_cast<size_t>(jb) * dv + sub];
-      float da = bf16_lo(ka.x) * qv[0], db = bf16_lo(kb.x) * qv[0];
-      da = fmaf(bf16_hi(ka.x), qv[1], da); db = fmaf(bf16_hi(kb.x), qv[1], db);
-      da = fmaf(bf16_lo(ka.y), qv[2], da); db = fmaf(bf16_lo(kb.y), qv[2], db);
-      da = fmaf(bf16_hi(ka.y), qv[3], da); db = fmaf(bf16_hi(kb.y), qv[3], db);
-      da = fmaf(bf16_lo(ka.z), qv[4], da); db = fmaf(bf16_lo(kb.z), qv[4], db);
-      da = fmaf(bf16_hi(ka.z), qv[5], da); db = fmaf(bf16_hi(kb.z), qv[5], db);
-      da = fmaf(bf16_lo(ka.w), qv[6], da); db = fmaf(bf16_lo(kb.w), qv[6], db);
-      da = fmaf(bf16_hi(ka.w), qv[7], da); db = fmaf(bf16_hi(kb.w), qv[7], db);
-      for (int d = grp >> 1; d >= 1; d >>= 1) {       // sum over the group's lanes (fixed tree)
-        da += __shfl_xor_sync(0xffffffffu, da, d);
-        db += __shfl_xor_sync(0xffffffffu, db, d);
+    constexpr int kFly = 4;   // key rows in flight per lane
+    for (int base = warp * per_warp; base < M; base += kFly * step) {   // warp-uniform trip count
+      int jt[kFly];
+      uint4 kv[kFly];
+#pragma unroll
+      for (int u = 0; u < kFly; ++u) {
+        jt[u] = base + u * step + tok_in_warp;
+        kv[u] = make_uint4(0, 0, 0, 0);
+        if (jt[u] < M && sub < dv) kv[u] = kh[static_cast<size_t>(jt[u]) * dv + sub];
       }
-      if (sub == 0) {
-        if (ja < M) { const float zz = da * p.scale_log2e; z[ja] = zz; mx = fmaxf(mx, zz); }
-        if (jb < M) { const float zz = db * p.scale_log2e; z[jb] = zz; mx = fmaxf(mx, zz); }
+#pragma unroll
+      for (int u = 0; u < kFly; ++u) {
+        float da = bf16_lo(kv[u].x) * qv[0];
+        da = fmaf(bf16_hi(kv[u].x), qv[1], da);
+        da = fmaf(bf16_lo(kv[u].y), qv[2], da);
+        da = fmaf(bf16_hi(kv[u].y), qv[3], da);
+        da = fmaf(bf16_lo(kv[u].z), qv[4], da);
+        da = fmaf(bf16_hi(kv[u].z), qv[5], da);
+        da = fmaf(bf16_lo(kv[u].w), qv[6], da);
+        da = fmaf(bf16_hi(kv[u].w), qv[7], da);
+        for (int d = grp >> 1; d >= 1; d >>= 1) da += __shfl_xor_sync(0xffffffffu, da, d);   // sum over the group's lanes (fixed tree)
+        if (sub == 0 && jt[u] < M) {
+          const float zz = da * p.scale_log2e;
+          z[jt[u]] = zz;
+          mx = fmaxf(mx, zz);
+        }
       }
     }
 #pragma unroll
