@@ -29,6 +29,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <type_traits>
 
 #include "mustdrop_internal.h"
 #include "select_body.cuh"
@@ -245,6 +246,19 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
   for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
 }
+// The same store under a predicate that must be uniform over the warp (no branch around it).
+__device__ __forceinline__ void tc_st16_if(bool go, uint32_t taddr, const float (&v)[16]) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %17, 0;\n\t"
+      "@p tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};\n\t}"
+      ::"r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])),
+        "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])),
+        "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15])), "r"(taddr), "r"(static_cast<uint32_t>(go))
+      : "memory");
+}
 __device__ __forceinline__ void tc_st16(uint32_t taddr, const float (&v)[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
@@ -277,23 +291,14 @@ __device__ __forceinline__ void trace_stamp(void* workspace, int n_heads, int h,
       [(static_cast<size_t>(blockIdx.x) * n_heads + h) * 16 + ev] = t;
 }
 #define MD_TRACE(h, ev) trace_stamp(p.workspace, p.H, (h), (ev))
-// SM clock instead of the global timer (finer; only differences within one thread mean anything):
-// thread 0's progress through the exp stage of a head, in the event slots 8.. of heads >= 1
-#define MD_TRACE_CLK(h, ev)                                                                          \
-  do {                                                                                               \
-    if (threadIdx.x == 0 && (h) > 0)                                                                 \
-      reinterpret_cast<long long*>(static_cast<unsigned char*>(p.workspace) + 4096)                  \
-          [(static_cast<size_t>(blockIdx.x) * p.H + (h)) * 16 + (ev)] = clock64();                   \
-  } while (0)
 #else
 #define MD_TRACE(h, ev) ((void)0)
-#define MD_TRACE_CLK(h, ev) ((void)0)
 #endif
 
 // Rare path of the exp warps (kept out of line so that the hot loop stays small): the `count`
 // chunks already stored at first, first + stride, ... are multiplied by this lane's factor.
 // Called by all lanes of a warp together.
-__device__ __noinline__ void rescale_stored(uint32_t first, uint32_t stride, int count, float fac) {
+__device__ __forceinline__ void rescale_stored(uint32_t first, uint32_t stride, int count, float fac) {
   tc_wait_st();
   for (int u = 0; u < count; ++u) {
     float old[kChunk];
@@ -303,6 +308,49 @@ __device__ __noinline__ void rescale_stored(uint32_t first, uint32_t stride, int
     for (int j = 0; j < kChunk; ++j) old[j] *= fac;
     tc_st16(first + stride * u, old);
   }
+}
+
+// The careful way through the chunks t_begin .. t_end - 1 of a thread (first + stride * t in
+// tensor memory), out of line as well: a chunk lay so far above the row's stabiliser that the sum
+// left its range, so from that chunk on nothing was stored.  Per chunk: its logits are taken
+// again, the stabiliser moves up to their maximum if that is larger, the chunks stored before it
+// are rescaled, the chunk's exponentials are computed and stored.  nvis0 - nvis_step * t columns of
+// chunk t are visible to this lane.  Returns the final stabiliser and the row's running sum.
+struct RedoResult {
+  float mx, l;
+};
+__device__ __forceinline__ RedoResult redo_rest(uint32_t first, uint32_t stride, int t_begin, int t_end, int nvis0, int nvis_step,
+                                             float scale_log2e, bool two_halves, float mx, float l) {
+  for (int t = t_begin; t < t_end; ++t) {
+    const int nvis = nvis0 - nvis_step * t;
+    float zc[kChunk];
+    tc_ld16(first + stride * t, zc);
+    tc_wait_ld();
+    float cm = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) {
+      zc[j] = (j < nvis) ? zc[j] : -INFINITY;
+      cm = fmaxf(cm, zc[j]);
+    }
+    cm *= scale_log2e;
+    if (two_halves) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 16));   // one stabiliser per row
+    const float up = fmaxf(mx, cm);
+    const float sub = (up == -INFINITY) ? 0.0f : up;     // a lane with nothing visible so far keeps 0
+    // (a lane whose stabiliser stays, or that has stored nothing but zeros so far, multiplies by 1)
+    const float fac = (up == mx || mx == -INFINITY) ? 1.0f : ex2(mx - up);
+    if (__any_sync(0xffffffffu, fac != 1.0f)) rescale_stored(first, stride, t, fac);   // (all lanes take part)
+    float part[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) {
+      const float e = ex2(fmaf(zc[j], scale_log2e, -sub));
+      zc[j] = e;
+      part[j & 3] += e;
+    }
+    tc_st16(first + stride * t, zc);
+    l = l * fac + ((part[0] + part[1]) + (part[2] + part[3]));
+    mx = up;
+  }
+  return RedoResult{mx, l};
 }
 
 struct __align__(8) Barriers {
@@ -325,6 +373,106 @@ struct GatherMaps {
   CUtensorMap k_src, v_src, k_dst, v_dst;
 };
 
+// ---- the filter tail, out of line ----------------------------------------------------------------
+// Both parts run once per CTA after the score part.  They are kept out of the kernel's body on
+// purpose: inlined, their code and registers changed how the score part's loops were compiled and
+// laid out, and the one-launch filter lost what the score-only kernel had gained.
+
+// Selection of request b by the 256 threads of the exp warps (tid = 0..255); rank 0 of the
+// request's CTAs stores the list, every CTA keeps it in its shared memory.
+__device__ __forceinline__ void filter_select(const SelectParams& sel, SelectShared& sel_sh, int b, int tid, bool writer,
+                                           int32_t* kept_list, int32_t* kept_total) {
+  select_clear(sel_sh, tid);
+  const int own = (sel.M + kSelThreads - 1) / kSelThreads;
+  if (own <= 1) select_request<1, SelectSyncGroup>(sel, sel_sh, b, tid, writer, kept_list, kept_total);
+  else if (own <= 2) select_request<2, SelectSyncGroup>(sel, sel_sh, b, tid, writer, kept_list, kept_total);
+  else if (own <= 4) select_request<4, SelectSyncGroup>(sel, sel_sh, b, tid, writer, kept_list, kept_total);
+  else if (own <= 8) select_request<8, SelectSyncGroup>(sel, sel_sh, b, tid, writer, kept_list, kept_total);
+  else select_request<16, SelectSyncGroup>(sel, sel_sh, b, tid, writer, kept_list, kept_total);
+}
+
+// Gather of the request's kept rows, driven by ONE thread of the CTA: row r of the compacted
+// outputs is copied by CTA r mod cluster.
+__device__ __forceinline__ void filter_gather(const FilterTail& ft, const GatherMaps& gm, uint64_t* gfull, volatile int* abort_flag,
+                                           const int32_t* kept_list, int kept_total_s, uint32_t stage_base, int rank, int b,
+                                           int Mb, int cluster, void* workspace) {
+  // One thread drives the copies: rows are loaded into a ring of shared-memory slots by bulk
+  // copies that count on the slot's mbarrier, and stored from there by bulk copies tracked in
+  // bulk groups.  Loads run n_slot - 2 rows ahead of the stores.
+  fence_proxy_async();   // earlier generic-proxy accesses to the slots precede the async-proxy writes
+  const int total = kept_total_s < ft.sel.cap ? kept_total_s : ft.sel.cap;
+  const int C = cluster;
+  // items: the kept vision rows, then (rebuild) the prefix rows and the request's text rows
+  const int n_items = total + (ft.rebuild ? ft.vis_start + ft.N : 0);
+  const int n_mine = n_items > rank ? (n_items - rank + C - 1) / C : 0;
+  const int S = ft.n_slot, ahead = S - 2;
+  const uint32_t ring = stage_base + kKeptListBytes;
+  const uint32_t payload = static_cast<uint32_t>(ft.hidden_bytes) + static_cast<uint32_t>(ft.has_k + ft.has_v) * ft.kv_bytes;
+  const uint64_t once = l2_evict_first_policy();
+  // item -> (source row, destination row)
+  auto src_row = [&](int it) {
+    if (it < total) return ft.vis_start + kept_list[it];
+    const int x = it - total;
+    return x < ft.vis_start ? x : ft.vis_start + Mb + (x - ft.vis_start);
+  };
+  auto dst_row = [&](int it) {
+    if (!ft.rebuild) return it;
+    if (it < total) return ft.vis_start + it;
+    const int x = it - total;
+    return x < ft.vis_start ? x : ft.vis_start + total + (x - ft.vis_start);
+  };
+  bool ok = true;
+  int loaded = 0;
+  for (int i = 0; i < n_mine + ahead && ok; ++i) {
+    if (i < n_mine) {
+      const int slot = i % S;
+      if (i >= S) bulk_wait_read_1();   // the stores of item i - S have finished reading the slot
+      const int row = src_row(rank + i * C);
+      const uint32_t bar = smem_u32(&gfull[slot]);
+      uint32_t dst = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
+      mbar_expect_tx(bar, payload);
+      if (ft.hidden_bytes > 0) {
+        bulk_load_1d(dst, ft.hidden + b * ft.hid_sb + row * ft.hid_sl, ft.hidden_bytes, bar, once);
+        dst += ft.hidden_pad;
+      }
+      if (ft.has_k) {
+        tma_load_4d_hint(dst, &gm.k_src, 0, row, 0, b, bar, once);
+        dst += ft.kv_bytes;
+      }
+      if (ft.has_v) tma_load_4d_hint(dst, &gm.v_src, 0, row, 0, b, bar, once);
+      loaded = i + 1;
+    }
+    const int c = i - ahead;
+    if (c >= 0) {
+      const int slot = c % S;
+      if (!mbar_wait(smem_u32(&gfull[slot]), static_cast<uint32_t>(c / S) & 1u, abort_flag, kWaitCycles)) { ok = false; break; }
+      const int r = dst_row(rank + c * C);
+      uint32_t src = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
+      if (ft.hidden_bytes > 0) {
+        bulk_store_1d(ft.hidden_out + (static_cast<int64_t>(b) * ft.out_rows + r) * ft.hidden_bytes, src, ft.hidden_bytes);
+        src += ft.hidden_pad;
+      }
+      if (ft.has_k) {
+        tma_store_4d(&gm.k_dst, 0, r, 0, b, src);
+        src += ft.kv_bytes;
+      }
+      if (ft.has_v) tma_store_4d(&gm.v_dst, 0, r, 0, b, src);
+      bulk_commit();
+    }
+  }
+  if (!ok) {
+    // gave up: still leave only when every load this thread started has landed (bounded)
+    record_status(workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
+    ft.sel.kept_cnt[b] = -1;   // some of this request's rows were not copied
+    for (int i = (loaded > S ? loaded - S : 0); i < loaded; ++i) {
+      const uint32_t bar = smem_u32(&gfull[i % S]);
+      const long long t0 = clock64();
+      while (!mbar_try_wait(bar, static_cast<uint32_t>(i / S) & 1u) && clock64() - t0 < kWaitCycles) {}
+    }
+  }
+  bulk_wait_all();   // the stores have been written before the CTA (and its shared memory) goes away
+}
+
 // HALVES: 2 = two M=64 tiles per head (N <= 64), 1 = one M=128 tile.
 // ACH: chunks (of 16 columns) an add thread may own; an exp thread owns up to (ACH+1)/2.
 // FILTER: after the scores, the cluster also selects the request's tokens and gathers them.
@@ -333,7 +481,7 @@ struct GatherMaps {
 template <int HALVES, int ACH, bool FILTER, bool PH>
 __global__ void __launch_bounds__(kThreads, 1)
 score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
-                   const FusedParams p, const __grid_constant__ GatherMaps gm, const FilterTail ft) {
+                   const FusedParams p, const __grid_constant__ GatherMaps gm, const __grid_constant__ FilterTail ft) {
   constexpr int NROWS = 128 / HALVES;            // text rows carried by the TMEM lanes
   // How the two exp warps of a lane quadrant share the work.  Wide tiles (ACH > 5): each takes
   // every second chunk of columns of every head (one (max, sum) pair per warp).  Narrow tiles: the
@@ -573,6 +721,18 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles) {}
         }
       }
+#ifdef MUSTDROP_TRACE
+    } else if (warp == kTmaWarp && lane == 1 && !p.split) {
+      // trace build only: an onlooker that stamps the moment a stage's copies have landed (it tests
+      // the barrier's phase and changes nothing; the MMA thread's own stamp comes when its turn does)
+      for (int h = 0; h < p.H; ++h) {
+        const uint32_t bar = smem_u32(&bars.full[h % p.n_q]);
+        const uint32_t ph = static_cast<uint32_t>(h / p.n_q) & 1u;
+        const long long t0 = clock64();
+        while (!mbar_try_wait(bar, ph) && clock64() - t0 < kWaitCycles && *abort_flag == 0) {}
+        MD_TRACE(h, 14);
+      }
+#endif
     } else if (warp == kMmaWarp && lane == 0) {
       // ---------------- MMA issuer ----------------
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(p.cpl >> 3) << 17) |
@@ -747,7 +907,24 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const int key_lane0 = static_cast<int>(rank) * p.tk + half * p.cpl;        // key of this lane's column 0
     int lim = p.causal ? (txt_start + p.row0 + row + 1) : Lb;                  // keys below lim are visible
     lim = (lim < Lb ? lim : Lb) - key_lane0;                                   // ... as a column count of this lane
-    const bool all_visible = lim >= p.cpl;
+    // Masking.  A lane sees the first `lim` of its columns (causal rows, end of the sequence); the
+    // hidden ones are text keys or lie beyond the sequence, i.e. never columns of the output, so all
+    // that matters about them is that they stay out of the row's sum.  A chunk is visible to a lane
+    // in full (nothing to do), not at all (its exponents are formed with scale 0 and addend -inf,
+    // and the lane's sum of that chunk is dropped), or in part: the chunks partly visible to some
+    // lane of the warp - [mix_lo, mix_hi), one or two per head and only in the CTA that holds the
+    // causal triangle or the end of the sequence - get their hidden logits overwritten before the loop.
+    const bool partial = lim > 0 && lim < p.cpl;
+    int lim_lo = partial ? lim : (1 << 30), lim_hi = partial ? lim : 0;
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+      const int a = __shfl_xor_sync(0xffffffffu, lim_lo, d), c = __shfl_xor_sync(0xffffffffu, lim_hi, d);
+      lim_lo = a < lim_lo ? a : lim_lo;
+      lim_hi = c > lim_hi ? c : lim_hi;
+    }
+    // chunk c (columns 16c .. 16c + 15) is partly visible to a lane only if 16c < lim < 16c + 16
+    const int mix_lo = lim_lo / kChunk;
+    const int mix_hi = (lim_hi + kChunk - 1) / kChunk;
     const bool sender = (half == 0);           // with two halves, lanes s and s+16 share a row: the lower one sends
     const uint32_t pair_idx = (rank * NROWS + row) * EPR + (kAlt ? 0 : g);     // this thread's pair in a slot
 
@@ -776,105 +953,100 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const uint32_t tbuf = tmem_base + static_cast<uint32_t>(buf * p.cpl) + lane_addr;
       const uint32_t slot_addr = smem_u32(&stats[slot * slot_pairs + pair_idx]);
       const uint32_t bar_addr = smem_u32(&bars.sfull[slot]);
-      // The thread's chunks stream through two register sets: while chunk t is worked on, chunk
-      // t + 1 is already on its way from tensor memory, and the exponentials of chunk t - 1 are on
-      // their way back.  The stabiliser is the maximum of the thread's FIRST chunk (shared by the two
-      // lanes of a row): any value within a few dozen powers of two of the row maximum serves, because
-      // every CTA sends the stabiliser it used along with its sum.  Later chunks compute no maximum:
-      // should their exponentials push the running sum beyond 2^kSumLimit (extreme logits), the warp
-      // takes the rare path - new stabiliser from the chunk at hand, stored chunks rescaled, the
-      // chunk redone (rescale_stored, kept out of line: the loop below is the hot code of the
-      // kernel and is written to stay small - two chunks per trip, not unrolled further).
+      // The thread's chunks go through a loop of one chunk per trip whose only taken branch is the
+      // loop edge, and whose body is small: with two exp warps per scheduler nobody fills the
+      // fetch bubble behind a taken branch (a loop of two chunks per trip with five or six of them
+      // per trip - loop edge, jumps around the mask, the first-chunk and the rare-path code - took
+      // twice the special-function unit's time), and straight-line code for all chunks of a head
+      // misses the instruction cache on every head.  z takes a chunk's logits from tensor memory;
+      // once they are turned into exponents in e, the next chunk's load goes out into z and runs
+      // under the exponentials, the sum, the check and the store of this one.
+      // The stabiliser is the maximum of the thread's FIRST chunk (shared by the two lanes of a
+      // row): any value within a few dozen powers of two of the row maximum serves, because every
+      // CTA sends the stabiliser it used along with its sum.  Later chunks compute no maximum:
+      // should their exponentials push a chunk's sum beyond kSumLimit (extreme logits), that chunk
+      // and the ones after it are not stored and not summed (predicates, no branch); after the
+      // last chunk one test sends the warp through the careful path for the rest (redo_rest, out
+      // of line: a maximum per chunk, stored chunks rescaled whenever the stabiliser moves).
       constexpr float kSumLimit = 1.0995116e12f;   // 2^40
-      float z0[kChunk], z1[kChunk];
-      MD_TRACE_CLK(h, 8);
-      tc_ld16(tbuf + kChunk * chunk_of(0), z0);
+      constexpr float kHidden = -3.0e38f;           // logit of a column the lane must not see (finite: 0 * kHidden = 0)
+      float z[kChunk], e[kChunk];
+      tc_ld16(tbuf + kChunk * chunk_of(0), z);
       if (last_buf >= 0 && !p.tight) {   // the head this warp worked on before: hand it to the add warps
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars.eready[last_buf]));
       }
-      MD_TRACE_CLK(h, 9);
       float mx = -INFINITY, sub = 0.0f;
-      float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      auto mask_chunk = [&](float(&zc)[kChunk], int t) {
-        if (!all_visible) {
-          const int nvis = lim - kChunk * chunk_of(t);   // visible columns of this chunk
-          if (nvis < kChunk) {
+      tc_wait_ld();
+      if (mix_lo < mix_hi) {
+        // Chunks partly visible to some lane of this warp (the causal triangle, the end of the
+        // sequence: one or two per head, and only in the CTA that holds them): the logits of the
+        // hidden columns are overwritten in tensor memory with a huge negative number before the
+        // loop, so that the loop itself carries no per-column mask.
+#pragma unroll 1
+        for (int t = 0; t < my_chunks; ++t) {
+          const int c = chunk_of(t);
+          if (c < mix_lo || c >= mix_hi) continue;
+          const int nvis = lim - kChunk * c;
+          if (t > 0) {
+            tc_ld16(tbuf + kChunk * c, e);
+            tc_wait_ld();
+          }
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) zc[j] = (j < nvis) ? zc[j] : -INFINITY;
+          for (int j = 0; j < kChunk; ++j) e[j] = (j < nvis) ? (t > 0 ? e[j] : z[j]) : kHidden;
+          tc_st16(tbuf + kChunk * c, e);
+          if (t == 0) {
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) z[j] = e[j];
           }
         }
-      };
-      auto chunk_max = [&](const float(&zc)[kChunk]) {   // in log2 units; scale > 0 keeps the order
+        tc_wait_st();
+      }
+      if (my_chunks > 0) {   // stabiliser from the first chunk
         float c4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        const int nvis = lim - kChunk * chunk_of(0);
 #pragma unroll
-        for (int j = 0; j < kChunk; ++j) c4[j & 3] = fmaxf(c4[j & 3], zc[j]);
-        float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3])) * p.scale_log2e;
-        if (HALVES == 2) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 16));   // one stabiliser per row
-        return cm;
-      };
-      // one chunk: mask, (first chunk: stabiliser,) exponentials, running sum, store
-      auto work = [&](float(&zc)[kChunk], int t) {
-        mask_chunk(zc, t);
-        if (t == 0) {
-          mx = chunk_max(zc);
-          sub = (mx == -INFINITY) ? 0.0f : mx;   // (first chunk all masked: so are the later ones)
-        }
+        for (int j = 0; j < kChunk; ++j) c4[j & 3] = fmaxf(c4[j & 3], (j < nvis) ? z[j] : -INFINITY);
+        mx = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3])) * p.scale_log2e;   // log2 units; scale > 0 keeps the order
+        if (HALVES == 2) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));  // one stabiliser per row
+        sub = (mx == -INFINITY) ? 0.0f : mx;   // (first chunk all masked: so are the later ones)
+      }
+      bool ok = true;   // warp-uniform: no chunk so far left the range
+      int stored = 0;   // chunks stored (my_chunks at the end unless a sum left its range)
+      float lsum = 0.0f;
+#pragma unroll 1
+      for (int t = 0; t < my_chunks; ++t) {
+        const int c = chunk_of(t);
+        const int nvis = lim - kChunk * c;                   // visible columns of this lane in this chunk
+        const float sc = nvis > 0 ? p.scale_log2e : 0.0f;    // nothing visible: exponent 0 * z - inf
+        const float ns = nvis > 0 ? -sub : -INFINITY;
+        tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < kChunk; ++j) e[j] = fmaf(z[j], sc, ns);
+        if (t + 1 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 1), z);
         float part[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
         for (int j = 0; j < kChunk; ++j) {
-          const float e = ex2(fmaf(zc[j], p.scale_log2e, -sub));
-          zc[j] = e;
-          part[j & 3] += e;
+          e[j] = ex2(e[j]);
+          part[j & 3] += e[j];
         }
-        const float psum = (part[0] + part[1]) + (part[2] + part[3]);
-        if (t > 0 && __any_sync(0xffffffffu, !(psum < kSumLimit))) {
-          // rare: this chunk lies far above the stabiliser.  Take its logits again, move the
-          // stabiliser up (all lanes take part; lanes whose stabiliser stays multiply by 1),
-          // rescale what is stored and redo the chunk.
-          tc_ld16(tbuf + kChunk * chunk_of(t), zc);
-          tc_wait_ld();
-          mask_chunk(zc, t);
-          const float up = fmaxf(mx, chunk_max(zc));
-          const float fac = (up == mx) ? 1.0f : ex2(sub - up);
-          rescale_stored(tbuf + kChunk * (kAlt ? 0 : g), kAlt ? kChunk : kChunk * kColGroups, t, fac);
-#pragma unroll
-          for (int x = 0; x < 4; ++x) ls4[x] *= fac;
-          mx = up;
-          sub = up;
-#pragma unroll
-          for (int x = 0; x < 4; ++x) part[x] = 0.0f;
-#pragma unroll
-          for (int j = 0; j < kChunk; ++j) {
-            const float e = ex2(fmaf(zc[j], p.scale_log2e, -sub));
-            zc[j] = e;
-            part[j & 3] += e;
-          }
-        }
-#pragma unroll
-        for (int x = 0; x < 4; ++x) ls4[x] += part[x];
-        tc_st16(tbuf + kChunk * chunk_of(t), zc);
-      };
-#pragma unroll 1
-      for (int t = 0; t < my_chunks; t += 2) {   // (my_chunks is warp-uniform)
-        tc_wait_ld();
-        if (t == 0) MD_TRACE_CLK(h, 10);
-        if (t + 1 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 1), z1);
-        work(z0, t);
-        if (t == 0) MD_TRACE_CLK(h, 11);
-        if (t == 2) MD_TRACE_CLK(h, 13);
-        if (t + 1 < my_chunks) {
-          tc_wait_ld();
-          if (t + 2 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 2), z0);
-          work(z1, t + 1);
-          if (t == 0) MD_TRACE_CLK(h, 12);
-          if (t == 2) MD_TRACE_CLK(h, 14);
-        }
+        // (a lane that sees nothing of this chunk: exponent -inf unless the hidden keys hold NaN or
+        // inf bits - its sum does not count either way, and what it stores lands in columns nobody reads)
+        const float psum = nvis > 0 ? (part[0] + part[1]) + (part[2] + part[3]) : 0.0f;
+        ok = ok && !__any_sync(0xffffffffu, !(psum < kSumLimit));   // (the first chunk's sum is at most 16)
+        lsum += ok ? psum : 0.0f;
+        tc_st16_if(ok, tbuf + kChunk * c, e);
+        stored += ok ? 1 : 0;
       }
-      MD_TRACE_CLK(h, 15);
-      float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+      if (stored < my_chunks) {   // rare
+        const RedoResult r = redo_rest(tbuf + kChunk * chunk_of(0), kAlt ? kChunk : kChunk * kColGroups, stored, my_chunks,
+                                       lim - kChunk * chunk_of(0),
+                                       kAlt ? kChunk : kChunk * kColGroups, p.scale_log2e, HALVES == 2, mx, lsum);
+        mx = r.mx;
+        lsum = r.l;
+      }
       if (HALVES == 2) lsum += __shfl_xor_sync(0xffffffffu, lsum, 16);
       if (p.gx) {
         // grid plan: the pair stays in this CTA's shared memory; the publishing warp merges the CTA's
@@ -911,15 +1083,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       common_exit();
       if (cluster_gave_up()) { leave_after_give_up(ft.sel.kept_cnt); return; }
       pdl_wait();   // the outputs written below may still be read by an earlier kernel in the stream
-      const int tid = threadIdx.x;
-      select_clear(sel_sh, tid);
-      const bool writer = rank == 0;
-      const int own = (ft.sel.M + kSelThreads - 1) / kSelThreads;
-      if (own <= 1) select_request<1, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-      else if (own <= 2) select_request<2, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-      else if (own <= 4) select_request<4, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-      else if (own <= 8) select_request<8, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
-      else select_request<16, SelectSyncGroup>(ft.sel, sel_sh, b, tid, writer, kept_list, &kept_total_s);
+      filter_select(ft.sel, sel_sh, b, threadIdx.x, rank == 0, kept_list, &kept_total_s);
       if (threadIdx.x == 0) MD_TRACE(0, 12);   // selection done
       cta_sync();   // the list is complete: the copy thread may start
       return;
@@ -1109,81 +1273,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       pdl_wait();
       cta_sync();   // the exp warps have finished the selection
       if (warp == kExpWarps && lane == 0) {
-        // One thread drives the copies: rows are loaded into a ring of shared-memory slots by bulk
-        // copies that count on the slot's mbarrier, and stored from there by bulk copies tracked in
-        // bulk groups.  Loads run n_slot - 2 rows ahead of the stores.
-        fence_proxy_async();   // earlier generic-proxy accesses to the slots precede the async-proxy writes
-        const int total = kept_total_s < ft.sel.cap ? kept_total_s : ft.sel.cap;
-        const int C = p.cluster;
-        // items: the kept vision rows, then (rebuild) the prefix rows and the request's text rows
-        const int n_items = total + (ft.rebuild ? ft.vis_start + ft.N : 0);
-        const int n_mine = n_items > static_cast<int>(rank) ? (n_items - static_cast<int>(rank) + C - 1) / C : 0;
-        const int S = ft.n_slot, ahead = S - 2;
-        const uint32_t ring = stage_base + kKeptListBytes;
-        const uint32_t payload = static_cast<uint32_t>(ft.hidden_bytes) + static_cast<uint32_t>(ft.has_k + ft.has_v) * ft.kv_bytes;
-        const uint64_t once = l2_evict_first_policy();
-        // item -> (source row, destination row)
-        auto src_row = [&](int it) {
-          if (it < total) return ft.vis_start + kept_list[it];
-          const int x = it - total;
-          return x < ft.vis_start ? x : ft.vis_start + Mb + (x - ft.vis_start);
-        };
-        auto dst_row = [&](int it) {
-          if (!ft.rebuild) return it;
-          if (it < total) return ft.vis_start + it;
-          const int x = it - total;
-          return x < ft.vis_start ? x : ft.vis_start + total + (x - ft.vis_start);
-        };
-        bool ok = true;
-        int loaded = 0;
-        for (int i = 0; i < n_mine + ahead && ok; ++i) {
-          if (i < n_mine) {
-            const int slot = i % S;
-            if (i >= S) bulk_wait_read_1();   // the stores of item i - S have finished reading the slot
-            const int row = src_row(static_cast<int>(rank) + i * C);
-            const uint32_t bar = smem_u32(&bars.gfull[slot]);
-            uint32_t dst = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
-            mbar_expect_tx(bar, payload);
-            if (ft.hidden_bytes > 0) {
-              bulk_load_1d(dst, ft.hidden + b * ft.hid_sb + row * ft.hid_sl, ft.hidden_bytes, bar, once);
-              dst += ft.hidden_pad;
-            }
-            if (ft.has_k) {
-              tma_load_4d_hint(dst, &gm.k_src, 0, row, 0, b, bar, once);
-              dst += ft.kv_bytes;
-            }
-            if (ft.has_v) tma_load_4d_hint(dst, &gm.v_src, 0, row, 0, b, bar, once);
-            loaded = i + 1;
-          }
-          const int c = i - ahead;
-          if (c >= 0) {
-            const int slot = c % S;
-            if (!mbar_wait(smem_u32(&bars.gfull[slot]), static_cast<uint32_t>(c / S) & 1u, abort_flag, kWaitCycles)) { ok = false; break; }
-            const int r = dst_row(static_cast<int>(rank) + c * C);
-            uint32_t src = ring + static_cast<uint32_t>(slot) * ft.slot_bytes;
-            if (ft.hidden_bytes > 0) {
-              bulk_store_1d(ft.hidden_out + (static_cast<int64_t>(b) * ft.out_rows + r) * ft.hidden_bytes, src, ft.hidden_bytes);
-              src += ft.hidden_pad;
-            }
-            if (ft.has_k) {
-              tma_store_4d(&gm.k_dst, 0, r, 0, b, src);
-              src += ft.kv_bytes;
-            }
-            if (ft.has_v) tma_store_4d(&gm.v_dst, 0, r, 0, b, src);
-            bulk_commit();
-          }
-        }
-        if (!ok) {
-          // gave up: still leave only when every load this thread started has landed (bounded)
-          record_status(p.workspace, MUSTDROP_ERR_TIMEOUT, blockIdx.x);
-          ft.sel.kept_cnt[b] = -1;   // some of this request's rows were not copied
-          for (int i = (loaded > S ? loaded - S : 0); i < loaded; ++i) {
-            const uint32_t bar = smem_u32(&bars.gfull[i % S]);
-            const long long t0 = clock64();
-            while (!mbar_try_wait(bar, static_cast<uint32_t>(i / S) & 1u) && clock64() - t0 < kWaitCycles) {}
-          }
-        }
-        bulk_wait_all();   // the stores have been written before the CTA (and its shared memory) goes away
+        filter_gather(ft, gm, bars.gfull, abort_flag, kept_list, kept_total_s, stage_base, static_cast<int>(rank), b, Mb,
+                      p.cluster, p.workspace);
         MD_TRACE(0, 13);   // gather done
       }
       return;

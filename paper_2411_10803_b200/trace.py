@@ -6,6 +6,7 @@ first 4096 bytes.  Runs the score call on a synthetic workload and prints, for a
 each stage of each head happened and the mean duration of the stages.
 
     python -m paper_2411_10803_b200.trace [workload]        # default c2_llava7b_b16
+    python -m paper_2411_10803_b200.trace [workload] score|filter [stamps.npy]
     python -m paper_2411_10803_b200.trace [workload] filter # the one-launch filter call: also the
                                                             # CTA-level stamps (entry, prologue,
                                                             # scores stored, selection, gather)
@@ -87,6 +88,8 @@ def main(argv) -> int:
                 raise RuntimeError("call refused: %d" % st)
             torch.cuda.synchronize()
         t = ws[4096:4096 + n_cta * w.n_heads * 16 * 8].cpu().numpy().view(np.uint64).reshape(n_cta, w.n_heads, 16).astype(np.float64)
+    if len(argv) > 3:   # third argument: keep the raw stamps (ns; [CTA][head][event]) for a closer look
+        np.save(argv[3], t)
     used = [c for c in range(n_cta) if t[c, 0, 0] > 0]
     if not used:
         print("no stamps: the plan does not use the fused kernel")
@@ -108,15 +111,15 @@ def main(argv) -> int:
         t0 = t[c, 0, 0]
         print("CTA", c)
         for h in sorted({0, 2, 4, w.n_heads // 2 // 2 * 2, (w.n_heads - 1) // 2 * 2}):
-            print("  head %02d " % h + " ".join("%s=%.2f" % (n, (t[c, h, e] - t0) / 1e3) for e, n in enumerate(EVENTS)))
-        clk = t[c, 2:, 8:16]
-        clk = clk[clk[:, 0] > 0]
-        if len(clk):
-            d = (clk - clk[:, :1]).mean(axis=0)
-            print("  exp stage of thread 0, SM clocks after its start: previous head handed over %.0f, first chunk "
-                  "loaded %.0f, chunks stored %.0f %.0f %.0f %.0f, all done %.0f" % tuple(d[1:]))
+            print("  head %02d " % h + " ".join("%s=%.2f" % (n, (t[c, h, e] - t0) / 1e3) for e, n in enumerate(EVENTS))
+                  + (" landed=%.2f" % ((t[c, h, 14] - t0) / 1e3) if t[c, h, 14] > 0 else ""))
         done = t[c, :, 7]
         print("  add_done per head: mean %.2f us" % (np.diff(done)[4:].mean() / 1e3))
+        if t[c, 4, 14] > 0:   # whole-stage plans: an onlooker stamps the landing of every stage
+            hs = t[c, 4:]
+            print("  stage: copies issued -> landed %.2f us, landed -> MMA thread takes it %.2f us, issue -> next issue "
+                  "into the same stage %.2f us" % ((hs[:, 14] - hs[:, 0]).mean() / 1e3, (hs[:, 2] - hs[:, 14]).mean() / 1e3,
+                                                  np.diff(t[c, 4:, 0]).mean() / 1e3))
         ev = t[c, 4::2]
         print("  exp stage %.2f us, exp_done -> statistics complete %.2f us, add stage %.2f us" % (
             (ev[:, 4] - ev[:, 3]).mean() / 1e3, (ev[:, 5] - ev[:, 4]).mean() / 1e3, (ev[:, 7] - ev[:, 6]).mean() / 1e3))
