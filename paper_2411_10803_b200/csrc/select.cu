@@ -18,15 +18,12 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
   const int tid = threadIdx.x;
   // Work that touches no global data, then let the next kernel start its prologue and wait for
   // the kernel that produced g / i.
-  SEL_STAMP(0);
   MD_PIPE(p.workspace, 1, false, false);
   select_clear(s, tid);
   pdl_launch_dependents();
   pdl_wait();
-  SEL_STAMP(1);
   select_request<OWN, SelectSyncCta>(p, s, blockIdx.x, tid, true, nullptr, nullptr);
   MD_PIPE(p.workspace, 1, true, false);
-  SEL_STAMP(12);
 }
 
 }  // namespace

@@ -49,6 +49,7 @@ struct SelectShared {
   double dsum[kSelWarps];
   int warp[kSelWarps];
   int wsuf[kSelWarps];
+  uint32_t band[kSelWarps], bor[kSelWarps];   // per warp: AND / OR of the tokens' ordered score bits
   int pick[3];
   int nkey;
 };
@@ -93,12 +94,6 @@ __device__ __noinline__ int group_exclusive_scan(int v, int tid, int* warp_sums 
   return base + inc - v;
 }
 
-#ifdef MUSTDROP_TRACE
-#define SEL_STAMP(ev) do { if (tid == 0 && blockIdx.x == 0 && p.workspace) { \
-  reinterpret_cast<long long*>(static_cast<unsigned char*>(p.workspace) + 2048)[ev] = clock64(); } } while (0)
-#else
-#define SEL_STAMP(ev) ((void)0)
-#endif
 
 // Clears the group's shared state; touches no global data.  select_request's first group barrier
 // orders the clear before every use, so no barrier is needed in between.
@@ -150,9 +145,7 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
 #pragma unroll
   for (int d = 16; d >= 1; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
   if (lane == 0) s.dsum[warp] = part;
-  SEL_STAMP(2);
   Sync::sync();   // also orders the bitmap clear before the key marks below
-  SEL_STAMP(3);
   // key set: mark distinct in-range indices
   if (p.key_max > 0) {
     const int c = key_c < p.key_max ? key_c : p.key_max;
@@ -189,9 +182,25 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
       if (write_out && p.s_out != nullptr) p.s_out[static_cast<size_t>(b) * ld + j] = sc;
     }
   }
-  SEL_STAMP(4);
+  // Bits that all of the request's scores share need no radix pass (scores of one request lie
+  // within a few powers of two: their top byte is the same for all, and a pass over it would be
+  // every thread's atomics on one or two counters): AND and OR over the tokens, per warp here,
+  // over the group behind the barrier below.
+  uint32_t all_and = 0xffffffffu, all_or = 0u;
+#pragma unroll
+  for (int e = 0; e < kOwn; ++e) {
+    if (e < own && j0 + e < M) {
+      all_and &= u[e];
+      all_or |= u[e];
+    }
+  }
+  all_and = __reduce_and_sync(0xffffffffu, all_and);
+  all_or = __reduce_or_sync(0xffffffffu, all_or);
+  if (lane == 0) {
+    s.band[warp] = all_and;
+    s.bor[warp] = all_or;
+  }
   Sync::sync();   // key marks complete
-  SEL_STAMP(5);
 
   // per-token bits: bit e of `valid` = token exists, of `key` = in the key set, of `keep` = retained
   uint32_t valid = 0u, key = 0u, keep = 0u;
@@ -221,27 +230,34 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
     keep |= key;
   } else {
     const int n_key = s.nkey;
-    SEL_STAMP(6);
     int want = p.budget - n_key;
     const int n_cand = M - n_key;
     want = want < n_cand ? want : n_cand;
     keep = key;
     if (want > 0) {
-      // radix select of the want-th largest candidate: four 8-bit digits from the top
-      uint32_t prefix = 0, mask = 0;
+      // radix select of the want-th largest candidate: 8-bit digits from the highest bit in
+      // which two tokens differ downwards (the bits above it are the same in every candidate)
+      uint32_t g_and = 0xffffffffu, g_or = 0u;
+#pragma unroll
+      for (int w = 0; w < kSelWarps; ++w) {
+        g_and &= s.band[w];
+        g_or |= s.bor[w];
+      }
+      const uint32_t differ = g_and ^ g_or;
+      const int hb = differ ? 31 - __clz(differ) : 7;                  // (all equal: one pass over the low byte)
+      uint32_t mask = hb >= 31 ? 0u : ~((2u << hb) - 1u);               // the shared bits
+      uint32_t prefix = g_and & mask;
       int remaining = want;
       // (kept as a real loop: the kernel runs once per launch from a cold instruction cache, so
       // code size, not instruction count, sets its latency)
 #pragma unroll 1
-      for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int shift = hb >= 7 ? hb - 7 : 0;; shift = shift > 8 ? shift - 8 : 0) {
 #pragma unroll
         for (int e = 0; e < kOwn; ++e) {
           const bool act = ((cand >> e) & 1u) && (u[e] & mask) == prefix;
           if (act) atomicAdd(&s.hist[(u[e] >> shift) & 255u], 1);
         }
-        if (shift == 16) SEL_STAMP(13);
         Sync::sync();
-        if (shift == 16) SEL_STAMP(14);
         // digit d is the cut iff (#candidates with a larger digit) < remaining <= that + hist[d];
         // thread d owns bin d: suffix sums by warp shuffles, then across the eight warps
         const int here = s.hist[tid];
@@ -253,9 +269,7 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
           if (lane + d < 32) suf += t;
         }
         if (lane == 0) s.wsuf[warp] = suf;
-        if (shift == 16) SEL_STAMP(15);
         Sync::sync();
-        if (shift == 16) SEL_STAMP(16);
         int above = suf - here;
 #pragma unroll
         for (int w = 0; w < kSelWarps; ++w)
@@ -266,11 +280,13 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
           s.pick[2] = here;
         }
         Sync::sync();
-        SEL_STAMP(7 + (24 - shift) / 8);
-        prefix |= static_cast<uint32_t>(s.pick[0]) << shift;
+        // (the lowest digit may reach over bits that are resolved already: they are the same in
+        // every token still in the running, so the bins keep their order)
+        prefix = (prefix & ~(255u << shift)) | (static_cast<uint32_t>(s.pick[0]) << shift);
         mask |= 255u << shift;
         remaining = s.pick[1];
         if (remaining == s.pick[2]) break;   // the whole bin is taken: lower digits cannot matter
+        if (shift == 0) break;
       }
       // Over the resolved digits, prefix is the cut: larger tokens are kept, and `remaining` of
       // the tokens equal to it, lowest index first (all of them after an early exit).
@@ -298,7 +314,6 @@ __device__ __forceinline__ void select_request(const SelectParams& p, SelectShar
     }
   }
 
-  SEL_STAMP(11);
   // index-ordered emit
   int total;
   int pos = group_exclusive_scan<Sync>(__popc(keep), tid, s.warp, &total);
