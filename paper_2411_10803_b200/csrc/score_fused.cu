@@ -270,6 +270,26 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const float (&v)[16]) {
         "r"(__float_as_uint(v[15])), "r"(taddr)
       : "memory");
 }
+// Two fp32 operations per instruction (packed in a 64-bit register pair): the exp and add warps'
+// loops are as much bound by the number of instructions they issue as by any unit.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -1023,15 +1043,20 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const float sc = nvis > 0 ? p.scale_log2e : 0.0f;    // nothing visible: exponent 0 * z - inf
         const float ns = nvis > 0 ? -sub : -INFINITY;
         tc_wait_ld();
+        const uint64_t sc2 = pack2(sc, sc), ns2 = pack2(ns, ns);
 #pragma unroll
-        for (int j = 0; j < kChunk; ++j) e[j] = fmaf(z[j], sc, ns);
+        for (int j = 0; j < kChunk; j += 2) unpack2(fma2(pack2(z[j], z[j + 1]), sc2, ns2), e[j], e[j + 1]);
         if (t + 1 < my_chunks) tc_ld16(tbuf + kChunk * chunk_of(t + 1), z);
-        float part[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        uint64_t part2[2] = {0ull, 0ull};   // (two packed zeros)
 #pragma unroll
-        for (int j = 0; j < kChunk; ++j) {
+        for (int j = 0; j < kChunk; j += 2) {
           e[j] = ex2(e[j]);
-          part[j & 3] += e[j];
+          e[j + 1] = ex2(e[j + 1]);
+          part2[(j >> 1) & 1] = add2(part2[(j >> 1) & 1], pack2(e[j], e[j + 1]));
         }
+        float part[4];
+        unpack2(part2[0], part[0], part[1]);
+        unpack2(part2[1], part[2], part[3]);
         // (a lane that sees nothing of this chunk: exponent -inf unless the hidden keys hold NaN or
         // inf bits - its sum does not count either way, and what it stores lands in columns nobody reads)
         const float psum = nvis > 0 ? (part[0] + part[1]) + (part[2] + part[3]) : 0.0f;
@@ -1098,11 +1123,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const int total_chunks = p.cpl / kChunk;
     const int tid_a = threadIdx.x - kExpThreads;
 
-    float acc[ACH][kChunk];
+    uint64_t acc[ACH][kChunk / 2];   // head sums, two columns per register pair
 #pragma unroll
     for (int c = 0; c < ACH; ++c)
 #pragma unroll
-      for (int j = 0; j < kChunk; ++j) acc[c][j] = 0.0f;
+      for (int j = 0; j < kChunk / 2; ++j) acc[c][j] = 0ull;
     // PH: this thread's keys tid_a, tid_a + 128, ... of the CTA: running sum over heads of the per-head maxima
     constexpr int PHK = (ACH * kChunk * HALVES + kAddThreads - 1) / kAddThreads;
     float ph_acc[PHK];
@@ -1164,11 +1189,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           tc_wait_ld();
           // chunk c was exponentiated by column group c & 1 (c0 is even)
           const float f0 = f[0], f1 = f[EPR - 1];
+          const uint64_t f0_2 = pack2(f0, f0), f1_2 = pack2(f1, f1);
 #pragma unroll
-          for (int j = 0; j < kChunk; ++j) acc[c0][j] = fmaf(e[0][j], f0, acc[c0][j]);
+          for (int j = 0; j < kChunk; j += 2) acc[c0][j >> 1] = fma2(pack2(e[0][j], e[0][j + 1]), f0_2, acc[c0][j >> 1]);
           if (c0 + 1 < ACH && c0 + 1 < total_chunks) {
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) acc[c0 + 1][j] = fmaf(e[1][j], f1, acc[c0 + 1][j]);
+            for (int j = 0; j < kChunk; j += 2)
+              acc[c0 + 1][j >> 1] = fma2(pack2(e[1][j], e[1][j + 1]), f1_2, acc[c0 + 1][j >> 1]);
           }
           if constexpr (PH) {
             // Column maxima over this warp's text rows (the lanes): recursive halving - in each of
@@ -1234,7 +1261,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           if (c < total_chunks) {
             const int key_local = half * p.cpl + kChunk * c;
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) mat[row * ld + key_local + j] = acc[c][j];
+            for (int j = 0; j < kChunk; j += 2) unpack2(acc[c][j >> 1], mat[row * ld + key_local + j], mat[row * ld + key_local + j + 1]);
           }
         }
       }
