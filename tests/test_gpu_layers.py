@@ -115,6 +115,43 @@ def test_ragged_layer_without_key_set_many_text_rows(path):
     run_ragged_layer(w, np.array([200, 30, 97], np.int32), True)
 
 
+@pytest.mark.parametrize("cluster", [2, 3, 5])
+def test_ragged_layer_with_logits_that_grow_along_the_keys(monkeypatch, cluster):
+    """The careful path of the exp warps (a chunk's sum leaves its range: new stabiliser, stored
+    chunks rescaled) in a ragged batch: lanes of the same warp see nothing at all of their half of
+    the CTA's keys (short requests), and the rows behind a request's sequence hold NaN bits."""
+    force(monkeypatch, variant="fused", cluster=cluster)
+    w = small(batch=4, n_vis=600, n_txt=40, n_heads=2, hidden=256, n_salient=0, key_cnt=0, budget=64, vis_start=0)
+    d = synth.make_batch(w)
+    q = synth.bf16_bits_to_f32(d["q_text"])
+    k = synth.bf16_bits_to_f32(d["k"])
+    u = q.mean(axis=2, keepdims=True)
+    u /= np.linalg.norm(u, axis=-1, keepdims=True)
+    ramp = np.linspace(0.0, 160.0, w.n_vis, dtype=np.float32)[None, None, :, None]     # over the vision keys only
+    k[:, :, :w.n_vis] += ramp * u * np.sqrt(128.0) / np.maximum(np.linalg.norm(q, axis=-1).mean(), 1e-6) * 3.0
+    d["k"] = synth.f32_to_bf16_bits(k.astype(np.float32))
+    vis_cnt = np.array([600, 150, 290, 40], np.int32)
+    p = synth.pack_ragged(d, w, vis_cnt)
+    f = md.Filter(cfg(w, flags=md.MUSTDROP_FLAG_REBUILD_SEQUENCE))
+    qd, kd, vd, hd = (to_dev_bf16(p[n]) for n in ("q_text", "k", "v", "hidden"))
+    f.filter_layer(qd, kd, vd, hd, None, None, vis_cnt=to_dev(p["vis_cnt"]), want_s=True)
+    torch.cuda.synchronize()
+    assert f.device_status() == (0, 0)
+    assert f.score_variant == "fused_cluster_tcgen05"
+    ref = layers.filter_layer_ragged(p["q_text"], p["k"], p["v"], p["hidden"], w.vis_start, p["vis_cnt"], w.budget,
+                                     None, None, rebuild=True)
+    g, i = f.g.cpu().numpy(), f.i.cpu().numpy()
+    assert np.isfinite(g).all() and np.isfinite(i).all()
+    big = ref["G"] > 1e-9                                   # compare where the mass is; the rest underflows alike
+    assert big.sum() > 20
+    assert_scores_close(g[big], ref["G"][big], "G")
+    assert_scores_close(i[big], ref["I"][big], "I")
+    assert (g[~big] <= 1e-7).all()
+    for b in range(w.batch):
+        assert not g[b, vis_cnt[b]:].any() and not i[b, vis_cnt[b]:].any()
+    f.close()
+
+
 def test_ragged_layer_llava7b_batch16():
     w = synth.WORKLOADS["c2_llava7b_b16"]
     assert run_ragged_layer(w, synth.draw_vis_cnt(w), True) == 1
