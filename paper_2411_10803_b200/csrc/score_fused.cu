@@ -393,10 +393,9 @@ struct GatherMaps {
   CUtensorMap k_src, v_src, k_dst, v_dst;
 };
 
-// ---- the filter tail, out of line ----------------------------------------------------------------
-// Both parts run once per CTA after the score part.  They are kept out of the kernel's body on
-// purpose: inlined, their code and registers changed how the score part's loops were compiled and
-// laid out, and the one-launch filter lost what the score-only kernel had gained.
+// ---- the filter tail ------------------------------------------------------------------------------
+// Both parts run once per CTA after the score part.  Functions of their own for reading only: they
+// are inlined (as real calls - like any call in this kernel - they slowed the gather by a third).
 
 // Selection of request b by the 256 threads of the exp warps (tid = 0..255); rank 0 of the
 // request's CTAs stores the list, every CTA keeps it in its shared memory.
