@@ -502,14 +502,11 @@ __global__ void __launch_bounds__(kThreads, 1)
 score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                    const FusedParams p, const __grid_constant__ GatherMaps gm, const __grid_constant__ FilterTail ft) {
   constexpr int NROWS = 128 / HALVES;            // text rows carried by the TMEM lanes
-  // How the two exp warps of a lane quadrant share the work.  Wide tiles (ACH > 5): each takes
-  // every second chunk of columns of every head (one (max, sum) pair per warp).  Narrow tiles: the
-  // whole row of a head fits one thread's registers, so the two warps ALTERNATE heads - two heads
-  // are in the exp stage at a time, which hides the tensor-memory load / store latencies that
-  // bound that stage when a head is only a few chunks wide.
-  constexpr bool kAlt = ACH <= 5;
-  constexpr int ECH = kAlt ? ACH : (ACH + 1) / 2;   // chunks per exp thread
-  constexpr int EPR = kAlt ? 1 : kColGroups;        // (max, sum) pairs per text row and CTA
+  // The two exp warps of a lane quadrant ALTERNATE heads (group g = 0, 1 takes the heads g,
+  // g + 2, ...): two heads are in the exp stage at a time, so what a head costs besides its chunk
+  // loop - waiting for its MMAs, the first chunk's load and maximum, the hand-over, the statistics
+  // stores - runs under the other group's loop.  (Splitting every head's chunks over the two warps
+  // instead left those 0.7 us per head on the path of every head: 7 % of a step at the target point.)
   constexpr bool kRealloc = ACH > 5;             // move registers from the other warpgroups to the add warps
 
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
@@ -525,7 +522,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const int b = blockIdx.x / p.cluster;
   MD_PIPE(p.workspace, 0, false, true);
   if (threadIdx.x == 0) MD_TRACE(0, 8);    // (CTA-level stamps use the event slots 8.. of head 0) kernel entry
-  // dynamic shared memory: [n_q query tiles][n_k key half-tiles][stats: n_slot x cluster x NROWS x EPR float2]
+  // dynamic shared memory: [n_q query tiles][n_k key half-tiles][stats: n_slot x cluster x NROWS float2]
   // A tile is two slabs of 64 elements (128 bytes per row, 128-byte swizzle), rows contiguous per slab.
   // Two layouts of the staging area: whole stages (a head's query tile and all its keys, n_q of
   // them, recycled together), or - where shared memory is short - a ring of n_q query tiles and a
@@ -539,12 +536,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
   const size_t staging = p.split ? static_cast<size_t>(p.n_q) * q_bytes + static_cast<size_t>(p.n_k) * kh_bytes
                                  : static_cast<size_t>(p.n_q) * stage_bytes;
   float2* stats = reinterpret_cast<float2*>(stage_ptr + staging);
-  // pairs per slot: EPR per text row and CTA; grid plans merge a CTA's pairs of a row before they
-  // leave the CTA (one pair per row and CTA crosses global memory and fills the slots)
-  const uint32_t slot_pairs = static_cast<uint32_t>(p.cluster) * NROWS * (p.gx ? 1 : EPR);
+  // pairs per slot: one (max, sum) pair per text row and CTA
+  const uint32_t slot_pairs = static_cast<uint32_t>(p.cluster) * NROWS;
   // PH only: [2][4 add warps][tk] per-head column maxima of each warp's text rows, double-buffered over heads
   float* const ph_stage = reinterpret_cast<float*>(stats + static_cast<size_t>(p.n_slot) * slot_pairs);
-  // grid plans only: [n_buf][rows][EPR] the pairs of this CTA's own exp warps, per tensor-memory buffer
+  // grid plans only: [n_buf][rows] the pairs of this CTA's own exp warps, per tensor-memory buffer
   float2* const own_pairs = reinterpret_cast<float2*>(ph_stage + (PH ? 2 * kAddWarps * p.tk : 0));
 
   if (threadIdx.x == 0) {
@@ -554,14 +550,14 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     for (int s = 0; s < kMaxKBufs; ++s) { mbar_init(smem_u32(&bars.full[s]), 1); mbar_init(smem_u32(&bars.empty[s]), 1); }
     for (int s = 0; s < kMaxBufs; ++s) {
       mbar_init(smem_u32(&bars.tfull[s]), 1);
-      mbar_init(smem_u32(&bars.eready[s]), kAlt ? kExpWarps / kColGroups : kExpWarps);
+      mbar_init(smem_u32(&bars.eready[s]), kExpWarps / kColGroups);   // (the four warps of the head's group)
       mbar_init(smem_u32(&bars.tempty[s]), kAddWarps);
     }
     // (grid plans: the 32 lanes of the fetch warp each arrive once their copies have landed)
     for (int s = 0; s < kMaxSlots; ++s) mbar_init(smem_u32(&bars.sfull[s]), p.gx ? 32 : 1);
     mbar_init(smem_u32(&bars.fin), kAddThreads);
     mbar_init(smem_u32(&bars.ph), kAddThreads);
-    for (int s = 0; s < kMaxBufs; ++s) mbar_init(smem_u32(&bars.gsent[s]), kAlt ? kExpWarps / kColGroups : kExpWarps);
+    for (int s = 0; s < kMaxBufs; ++s) mbar_init(smem_u32(&bars.gsent[s]), kExpWarps / kColGroups);
     for (int s = 0; s < kMaxGatherSlots; ++s) mbar_init(smem_u32(&bars.gfull[s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -888,15 +884,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const size_t bh = static_cast<size_t>(b) * p.H + h;
         float2* const dst = p.gx_stats + (bh * p.cluster + rank) * NROWS;
         for (int r = lane; r < NROWS; r += 32) {
-          const float2* const pr = own_pairs + (buf * NROWS + r) * EPR;
-          float2 v = pr[0];
-          if (EPR == 2) {
-            const float2 w2 = pr[EPR - 1];
-            const float m2 = fmaxf(v.x, w2.x);
-            const float ref = (m2 == -INFINITY) ? 0.0f : m2;
-            v = make_float2(m2, v.y * ex2(v.x - ref) + w2.y * ex2(w2.x - ref));   // an empty pair is (-inf, 0)
-          }
-          dst[r] = v;
+          dst[r] = own_pairs[buf * NROWS + r];
         }
         __syncwarp();
         if (lane == 0) {
@@ -921,8 +909,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const uint32_t lane_addr = static_cast<uint32_t>(32 * q) << 16;
     const int total_chunks = p.cpl / kChunk;
     // chunks g, g+2, ... of every head, or all chunks of every second head (uniform per warp)
-    const int my_chunks = kAlt ? total_chunks : (total_chunks - g + kColGroups - 1) / kColGroups;
-    auto chunk_of = [&](int t) { return kAlt ? t : g + t * kColGroups; };
+    const int my_chunks = total_chunks;
+    auto chunk_of = [&](int t) { return t; };
     const int key_lane0 = static_cast<int>(rank) * p.tk + half * p.cpl;        // key of this lane's column 0
     int lim = p.causal ? (txt_start + p.row0 + row + 1) : Lb;                  // keys below lim are visible
     lim = (lim < Lb ? lim : Lb) - key_lane0;                                   // ... as a column count of this lane
@@ -945,10 +933,14 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const int mix_lo = lim_lo / kChunk;
     const int mix_hi = (lim_hi + kChunk - 1) / kChunk;
     const bool sender = (half == 0);           // with two halves, lanes s and s+16 share a row: the lower one sends
-    const uint32_t pair_idx = (rank * NROWS + row) * EPR + (kAlt ? 0 : g);     // this thread's pair in a slot
+    const uint32_t pair_idx = rank * NROWS + row;                              // this thread's pair in a slot
 
     int last_buf = -1;
-    for (int h = kAlt ? g : 0; h < p.H; h += kAlt ? kColGroups : 1) {
+    // Hand-over of a head's exponentials to the add warps: one head of this group later (the wait
+    // for the stores then costs nothing) - unless that next head needs the very buffer (two
+    // buffers: its MMAs wait for the add warps, who wait for this hand-over), or the window is tight.
+    const bool eager = p.tight != 0 || p.n_buf <= kColGroups;
+    for (int h = g; h < p.H; h += kColGroups) {
       const int buf = h % p.n_buf;
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
       const int slot = h % p.n_slot;
@@ -964,7 +956,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       }
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.tfull[buf]), bph, abort_flag, wait_limit))) break;
       if (threadIdx.x == 0) MD_TRACE(h, 3);
-      if (!p.gx && lane == 0 && q == 0 && (kAlt || g == 0)) {
+      if (!p.gx && lane == 0 && q == 0) {
         // arm this head's statistics barrier with the bytes all CTAs will send
         mbar_expect_tx(smem_u32(&bars.sfull[slot]), slot_pairs * 8u);
       }
@@ -991,7 +983,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       constexpr float kHidden = -3.0e38f;           // logit of a column the lane must not see (finite: 0 * kHidden = 0)
       float z[kChunk], e[kChunk];
       tc_ld16(tbuf + kChunk * chunk_of(0), z);
-      if (last_buf >= 0 && !p.tight) {   // the head this warp worked on before: hand it to the add warps
+      if (last_buf >= 0 && !eager) {   // the head this warp worked on before: hand it to the add warps
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -1065,9 +1057,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         stored += ok ? 1 : 0;
       }
       if (stored < my_chunks) {   // rare
-        const RedoResult r = redo_rest(tbuf + kChunk * chunk_of(0), kAlt ? kChunk : kChunk * kColGroups, stored, my_chunks,
-                                       lim - kChunk * chunk_of(0),
-                                       kAlt ? kChunk : kChunk * kColGroups, p.scale_log2e, HALVES == 2, mx, lsum);
+        const RedoResult r = redo_rest(tbuf, kChunk, stored, my_chunks, lim, kChunk, p.scale_log2e, HALVES == 2, mx, lsum);
         mx = r.mx;
         lsum = r.l;
       }
@@ -1075,7 +1065,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       if (p.gx) {
         // grid plan: the pair stays in this CTA's shared memory; the publishing warp merges the CTA's
         // pairs of a row and sends one pair per row on its way through global memory
-        if (sender) own_pairs[(buf * NROWS + row) * EPR + (kAlt ? 0 : g)] = make_float2(mx, lsum);
+        if (sender) own_pairs[buf * NROWS + row] = make_float2(mx, lsum);
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars.gsent[buf]));
       } else if (sender) {
@@ -1083,7 +1073,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           st_async_f32x2(map_to_cta(slot_addr, c), mx, lsum, map_to_cta(bar_addr, c));
       }
       last_buf = buf;
-      if (p.tight) {   // hand over at once: the add warps of this head gate our next heads
+      if (eager) {   // hand over at once: the add warps of this head gate our next heads
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -1140,7 +1130,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
       const int slot = h % p.n_slot;
       const uint32_t sph = static_cast<uint32_t>(h / p.n_slot) & 1u;
-      float f[EPR];                            // factor of each of this CTA's pairs
+      float f;                                 // factor of this CTA's exponentials of the row
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.sfull[slot]), sph, abort_flag, wait_limit))) break;
       if (tid_a == 0) MD_TRACE(h, 5);
       if (p.gx) {
@@ -1155,25 +1145,19 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           l = fmaf(v.y, ex2(v.x - m), l);
         }
         const float inv_l = 1.0f / l;
-#pragma unroll
-        for (int x = 0; x < EPR; ++x) f[x] = ex2(own_pairs[(buf * NROWS + row) * EPR + x].x - m) * inv_l;
+        f = ex2(own_pairs[buf * NROWS + row].x - m) * inv_l;
       } else {
         // statistics of this row over the whole key range: every CTA's pairs
-        const float2* srow = stats + slot * slot_pairs + row * EPR;
+        const float2* srow = stats + slot * slot_pairs + row;
         float m = -INFINITY;
-        for (int c = 0; c < p.cluster; ++c)
-#pragma unroll
-          for (int x = 0; x < EPR; ++x) m = fmaxf(m, srow[c * NROWS * EPR + x].x);
+        for (int c = 0; c < p.cluster; ++c) m = fmaxf(m, srow[c * NROWS].x);
         float l = 0.0f;
-        for (int c = 0; c < p.cluster; ++c)
-#pragma unroll
-          for (int x = 0; x < EPR; ++x) {
-            const float2 v = srow[c * NROWS * EPR + x];
-            l = fmaf(v.y, ex2(v.x - m), l);     // an empty pair is (-inf, 0): contributes 0
-          }
+        for (int c = 0; c < p.cluster; ++c) {
+          const float2 v = srow[c * NROWS];
+          l = fmaf(v.y, ex2(v.x - m), l);     // an empty pair is (-inf, 0): contributes 0
+        }
         const float inv_l = 1.0f / l;
-#pragma unroll
-        for (int x = 0; x < EPR; ++x) f[x] = ex2(srow[rank * NROWS * EPR + x].x - m) * inv_l;
+        f = ex2(srow[rank * NROWS].x - m) * inv_l;
       }
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.eready[buf]), bph, abort_flag, wait_limit))) break;
       if (tid_a == 0) MD_TRACE(h, 6);
@@ -1186,9 +1170,8 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           tc_ld16(tbuf + kChunk * c0, e[0]);
           if (c0 + 1 < ACH && c0 + 1 < total_chunks) tc_ld16(tbuf + kChunk * (c0 + 1), e[1]);
           tc_wait_ld();
-          // chunk c was exponentiated by column group c & 1 (c0 is even)
-          const float f0 = f[0], f1 = f[EPR - 1];
-          const uint64_t f0_2 = pack2(f0, f0), f1_2 = pack2(f1, f1);
+          const float f0 = f, f1 = f;
+          const uint64_t f0_2 = pack2(f, f), f1_2 = f0_2;
 #pragma unroll
           for (int j = 0; j < kChunk; j += 2) acc[c0][j >> 1] = fma2(pack2(e[0][j], e[0][j + 1]), f0_2, acc[c0][j >> 1]);
           if (c0 + 1 < ACH && c0 + 1 < total_chunks) {
@@ -1443,7 +1426,10 @@ bool plan_score_fused(const Resolved& r, int sm_count, int forced_cluster, Fused
     const int tk = cpl * halves;
     const size_t stage = static_cast<size_t>(nrows + tk) * 256;
     const int ach = cpl <= 5 * kChunk ? 5 : (cpl <= 10 * kChunk ? 10 : 11);   // chunks per add thread (kernel variant)
-    const int epr = ach <= 5 ? 1 : kColGroups;              // (max, sum) pairs per row and CTA (the kernel's EPR)
+    // slot size in pairs per row and CTA.  The kernel sends ONE pair per row; wide tiles keep the room for
+    // two that they had when the two exp warps of a quadrant shared a head: the cost model's constants and
+    // every measured plan choice rest on the stage / buffer / slot counts that this sizing gives.
+    const int epr = ach <= 5 ? 1 : kColGroups;
     // Shared memory.  Whole stages first (a head's query tile and keys recycled together): as many
     // tensor-memory buffers as the columns allow (3..8), fewer if their statistics slots (2 x
     // buffers x cluster x rows x pairs x 8 bytes) would leave no room for 2 stages; four stages
@@ -1560,7 +1546,7 @@ bool plan_score_grid(const Resolved& r, int sm_count, int forced_ctas, FusedGeom
     if (n_buf < kMinBufs) continue;
     // shared memory: statistics slots the fetch warp fills (a head's pairs of all the request's
     // CTAs; at least two, so that the next head's are fetched while this one is added) and stages
-    const int epr = ach <= 5 ? 1 : kColGroups;
+    const int epr = ach <= 5 ? 1 : kColGroups;   // (room for two pairs per row on wide tiles: see plan_score_fused)
     const size_t slot = static_cast<size_t>(c) * nrows * 8;                 // one merged pair per row and CTA
     const size_t own = static_cast<size_t>(n_buf) * nrows * epr * 8;        // the CTA's own pairs, per buffer
     if (avail < own + 2 * slot + 2 * stage) continue;

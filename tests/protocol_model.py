@@ -1,14 +1,18 @@
 """Host model of the barrier protocol of the fused score kernel: threads stand for the warp roles
 of every CTA of one cluster, Python objects for the mbarriers.
 
-What is modelled (names as in the kernel): per CTA a copy role (TMA), an MMA role, an exp role and
-an add role, joined by the barriers
+What is modelled (names as in the kernel): per CTA a copy role (TMA), an MMA role, TWO exp roles
+(the two groups of exp warps alternate heads: group g takes the heads g, g + 2, ...) and an add
+role, joined by the barriers
     full / empty      staged keys of a head have landed / have been consumed        (n_q stages)
     tfull             logits of a head are in a tensor-memory buffer                 (n_buf buffers)
     eready            the exponentials of a head are in the buffer
     tempty            the buffer is free again
     sfull             every CTA's (max, sum) pair of a head has arrived in a slot    (n_slot slots)
 with the phase-parity waits, the transaction counts of the asynchronous statistics stores, the
+hand-over rule (an exp group hands a head's exponentials to the add role only when it has got to
+its NEXT head - the wait for its stores then costs nothing - except where that next head needs
+the very same buffer, i.e. with two buffers, or under the tight rule: then at once), the
 "tight" rule (the exp role stays within d heads of the local add role when there are only 2 d
 slots) and the bounded waits: a wait that runs out raises the CTA's abort flag, every other wait
 of that CTA then returns at once, the CTA records a time-out, tells its peers before the exit
@@ -28,6 +32,7 @@ import threading
 import time
 
 OK, TIMEOUT = 0, 6          # MUSTDROP_OK, MUSTDROP_ERR_TIMEOUT
+N_GROUPS = 2                # groups of exp warps per CTA; they alternate heads
 
 
 class ProtocolError(AssertionError):
@@ -103,13 +108,15 @@ class Cluster:
     arrive ("full", "tfull", "eready", "tempty", "empty") or one statistics store ("stats")."""
 
     def __init__(self, C=2, H=12, n_q=2, n_buf=3, n_slot=None, tight=0, limit=0.25, fault=None, jitter=None,
-                 grid=False):
+                 grid=False, handover="auto"):
         n_slot = (min(n_buf, 4) if grid else 2 * n_buf) if n_slot is None else n_slot
         self.grid = grid
         self.g_lock = threading.Lock()
         self.g_cnt = [0] * H                       # global memory: pairs published per head
         self.g_pairs = [[None] * C for _ in range(H)]
         self.geo = dict(C=C, H=H, n_q=n_q, n_buf=n_buf, n_slot=n_slot, tight=tight)
+        # "auto": the kernel's rule; "late": always one head of the group later (what the rule prevents)
+        self.eager = (tight != 0 or n_buf <= N_GROUPS) if handover == "auto" else False
         self.limit, self.fault, self.jitter = limit, fault, jitter or {}
         self.ctas = [Cta(self, r, self.geo) for r in range(C)]
         self.errors = []
@@ -149,18 +156,20 @@ class Cluster:
             self._pause(c.rank, "mma")
             if c.stage_head[s] != h:
                 raise ProtocolError("MMA of head %d found head %s staged" % (h, c.stage_head[s]))
-            if c.buf_state[buf][0] != "free":
-                raise ProtocolError("buffer %d overwritten while %s" % (buf, c.buf_state[buf],))
-            c.buf_state[buf] = ("logits", h)
+            with c.guard:
+                if c.buf_state[buf][0] != "free":
+                    raise ProtocolError("buffer %d overwritten while %s" % (buf, c.buf_state[buf],))
+                c.buf_state[buf] = ("logits", h)
             c.stage_head[s] = None
             if not self._skips(c.rank, "mma", h, "empty"):
                 c.empty[s].arrive()
             if not self._skips(c.rank, "mma", h, "tfull"):
                 c.tfull[buf].arrive()
 
-    def exp(self, c):
+    def exp(self, c, grp=0):
         g = self.geo
-        for h in range(g["H"]):
+        last = None                                   # head this group worked on before, not yet handed over
+        for h in range(grp, g["H"], N_GROUPS):
             buf, slot = h % g["n_buf"], h % g["n_slot"]
             if g["tight"] and h >= g["tight"]:
                 u = h - g["tight"]
@@ -170,10 +179,15 @@ class Cluster:
                 return
             if not self.grid:
                 c.sfull[slot].arrive(expect_tx=g["C"])    # arm: every CTA will send one pair
+            if last is not None:                          # late hand-over of the group's previous head
+                if not self._skips(c.rank, "exp", last, "eready"):
+                    c.eready[last % g["n_buf"]].arrive()
+                last = None
             self._pause(c.rank, "exp")
-            if c.buf_state[buf] != ("logits", h):
-                raise ProtocolError("exp role of head %d found %s" % (h, c.buf_state[buf],))
-            c.buf_state[buf] = ("exps", h)
+            with c.guard:
+                if c.buf_state[buf] != ("logits", h):
+                    raise ProtocolError("exp role of head %d found %s" % (h, c.buf_state[buf],))
+                c.buf_state[buf] = ("exps", h)
             if self.grid:
                 if c.own_pair[buf] is not None:
                     raise ProtocolError("own pair of buffer %d overwritten before head %s was added" % (buf, c.own_pair[buf]))
@@ -188,8 +202,16 @@ class Cluster:
                                                 % (slot, peer.rank, peer.stats[slot][c.rank], h))
                         peer.stats[slot][c.rank] = h
                     peer.sfull[slot].complete_tx(1)
-            if not self._skips(c.rank, "exp", h, "eready"):
-                c.eready[buf].arrive()
+            if self.eager:
+                if not self._skips(c.rank, "exp", h, "eready"):
+                    c.eready[buf].arrive()
+            else:
+                last = h
+        if last is not None and not self._skips(c.rank, "exp", last, "eready"):
+            c.eready[last % g["n_buf"]].arrive()          # the last head the group worked on
+
+    def exp1(self, c):
+        self.exp(c, 1)
 
     def add(self, c):
         g = self.geo
@@ -208,9 +230,10 @@ class Cluster:
             if not c.wait(c.eready[buf], (h // g["n_buf"]) & 1, self.limit):
                 return
             self._pause(c.rank, "add")
-            if c.buf_state[buf] != ("exps", h):
-                raise ProtocolError("add role of head %d found %s" % (h, c.buf_state[buf],))
-            c.buf_state[buf] = ("free", None)
+            with c.guard:
+                if c.buf_state[buf] != ("exps", h):
+                    raise ProtocolError("add role of head %d found %s" % (h, c.buf_state[buf],))
+                c.buf_state[buf] = ("free", None)
             c.added.append(h)
             if not self._skips(c.rank, "add", h, "tempty"):
                 c.tempty[buf].arrive()
@@ -263,7 +286,7 @@ class Cluster:
                 self.errors.append(str(e))
                 c.abort = True
 
-        roles = (self.tma, self.mma, self.exp, self.add) + ((self.publish, self.fetch) if self.grid else ())
+        roles = (self.tma, self.mma, self.exp, self.exp1, self.add) + ((self.publish, self.fetch) if self.grid else ())
         threads = [threading.Thread(target=guarded, args=(fn, c), daemon=True)
                    for c in self.ctas for fn in roles]
         for t in threads:

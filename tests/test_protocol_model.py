@@ -35,6 +35,19 @@ def test_protocol_tolerates_a_slow_role(slow):
     assert all(c.added == list(range(10)) for c in cl.ctas) and cl.kept_cnt == 10
 
 
+@pytest.mark.parametrize("n_buf,ends", [(2, False), (3, True), (4, True)])
+def test_a_late_hand_over_needs_a_third_buffer(n_buf, ends):
+    # An exp group hands a head over when it has got to its next head, two heads on.  With two
+    # buffers that next head needs the same buffer: its MMAs wait for the add role, which waits
+    # for the hand-over - every wait runs out (the kernel hands over at once in that case).
+    cl = Cluster(C=2, H=9, n_q=2, n_buf=n_buf, limit=0.3, handover="late")
+    assert cl.run(join_limit=10.0), "a role hung instead of giving up"
+    assert cl.errors == []
+    assert (cl.kept_cnt == 9) == ends
+    if not ends:
+        assert all(c.status == TIMEOUT for c in cl.ctas)
+
+
 def test_fewer_slots_than_the_protocol_needs_is_caught_by_the_model():
     # 2 x buffers slots are needed without the tight rule: with fewer, a fast peer overwrites an unread pair
     cl = Cluster(C=2, H=16, n_q=4, n_buf=4, n_slot=4, tight=0, limit=0.3, jitter={(0, "add"): 0.01})
