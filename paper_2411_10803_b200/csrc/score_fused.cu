@@ -25,6 +25,7 @@
 // (which still frees tensor memory and joins the cluster barrier).
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <cstring>
 #include <mutex>
@@ -39,6 +40,7 @@ namespace {
 
 constexpr int kExpWarps = 8;                // warps 0-7: 4 TMEM lane quadrants x 2 column groups
 constexpr int kColGroups = 2;
+constexpr float kPhScale = 16384.0f;        // per-head maxima travel as fp16 times 2^14
 constexpr int kAddWarps = 4;                // warps 8-11: one per lane quadrant, all columns
 constexpr int kExpThreads = kExpWarps * 32;
 constexpr int kAddThreads = kAddWarps * 32;
@@ -283,6 +285,11 @@ __device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
 __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
   uint64_t d;
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
 __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
@@ -1182,32 +1189,48 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           if constexpr (PH) {
             // Column maxima over this warp's text rows (the lanes): recursive halving - in each of
             // four steps a lane keeps half of its columns and takes its partner's maxima for them,
-            // so that after 8 + 4 + 2 + 1 shuffles lane j of a 16-lane group holds column j's maximum
-            // over the group (about one shuffle per column).  With 128 text rows the two 16-lane
-            // groups of a warp hold the same columns and are folded first.
+            // so that lane j of a 16-lane group ends up with column j's maximum over the group.  The
+            // probabilities travel as fp16 pairs (two columns per register: half the shuffles,
+            // selects and maxima), scaled by 2^14 so that nothing above 4e-9 is subnormal; rounding
+            // them costs 2^-11 relative, a quarter of the score tolerance.  With 128 text rows the
+            // two 16-lane groups of a warp hold the same columns and are folded first.
             float* const dst = ph_stage + ((h & 1) * kAddWarps + q) * p.tk + half * p.cpl + (lane & 15);
+            auto hmax2 = [](uint32_t a, uint32_t b2) {
+              uint32_t r;
+              asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b2));
+              return r;
+            };
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
               if (c0 + x < ACH && c0 + x < total_chunks) {
-                const float fx = real_row ? (x ? f1 : f0) : 0.0f;
-                float v[kChunk];
+                const float fx = real_row ? f * kPhScale : 0.0f;
+                const uint64_t fx2 = pack2(fx, fx);
+                uint32_t hv[kChunk / 2];
 #pragma unroll
-                for (int j = 0; j < kChunk; ++j) v[j] = e[x][j] * fx;
+                for (int k = 0; k < kChunk / 2; ++k) {
+                  float lo, hi;
+                  unpack2(mul2(pack2(e[x][2 * k], e[x][2 * k + 1]), fx2), lo, hi);
+                  const __half2 t = __floats2half2_rn(lo, hi);   // (lo, hi) = columns 2k, 2k + 1
+                  hv[k] = *reinterpret_cast<const uint32_t*>(&t);
+                }
                 if (HALVES == 1) {
 #pragma unroll
-                  for (int j = 0; j < kChunk; ++j) v[j] = fmaxf(v[j], __shfl_xor_sync(0xffffffffu, v[j], 16));
+                  for (int k = 0; k < kChunk / 2; ++k) hv[k] = hmax2(hv[k], __shfl_xor_sync(0xffffffffu, hv[k], 16));
                 }
 #pragma unroll
-                for (int step = kChunk / 2; step >= 1; step >>= 1) {
-                  const bool upper = (lane & step) != 0;
+                for (int step = kChunk / 4; step >= 1; step >>= 1) {   // registers apart: 8, 4, 2 columns
+                  const bool upper = (lane & (2 * step)) != 0;
 #pragma unroll
                   for (int i = 0; i < step; ++i) {
-                    const float give = upper ? v[i] : v[i + step];
-                    const float keep = upper ? v[i + step] : v[i];
-                    v[i] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, step));
+                    const uint32_t give = upper ? hv[i] : hv[i + step];
+                    const uint32_t keep = upper ? hv[i + step] : hv[i];
+                    hv[i] = hmax2(keep, __shfl_xor_sync(0xffffffffu, give, 2 * step));
                   }
                 }
-                if (HALVES == 2 || lane < 16) dst[kChunk * (c0 + x)] = v[0];
+                // the last step is inside the register: even lanes end with its low half, odd ones with its high half
+                const uint32_t r2 = hmax2(hv[0], __shfl_xor_sync(0xffffffffu, hv[0], 1));
+                const unsigned short bits = static_cast<unsigned short>((lane & 1) ? (r2 >> 16) : (r2 & 0xffffu));
+                if (HALVES == 2 || lane < 16) dst[kChunk * (c0 + x)] = __half2float(__ushort_as_half(bits));
               }
             }
           }
@@ -1263,6 +1286,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           mx = 0.0f;   // (x < PHK always; a compile-time unrolled pick keeps ph_acc in registers)
 #pragma unroll
           for (int y = 0; y < PHK; ++y) mx = (y == x) ? ph_acc[y] : mx;
+          mx *= 1.0f / kPhScale;
         }
         const bool present = j < Mb;    // beyond the request's own tokens: zeros
         float gv = present ? s * p.inv_heads : 0.0f, iv = present ? mx * p.inv_heads : 0.0f;
