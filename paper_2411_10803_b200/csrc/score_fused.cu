@@ -942,11 +942,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const bool sender = (half == 0);           // with two halves, lanes s and s+16 share a row: the lower one sends
     const uint32_t pair_idx = rank * NROWS + row;                              // this thread's pair in a slot
 
-    int last_buf = -1;
-    // Hand-over of a head's exponentials to the add warps: one head of this group later (the wait
-    // for the stores then costs nothing) - unless that next head needs the very buffer (two
-    // buffers: its MMAs wait for the add warps, who wait for this hand-over), or the window is tight.
-    const bool eager = p.tight != 0 || p.n_buf <= kColGroups;
     for (int h = g; h < p.H; h += kColGroups) {
       const int buf = h % p.n_buf;
       const uint32_t bph = static_cast<uint32_t>(h / p.n_buf) & 1u;
@@ -990,12 +985,6 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
       constexpr float kHidden = -3.0e38f;           // logit of a column the lane must not see (finite: 0 * kHidden = 0)
       float z[kChunk], e[kChunk];
       tc_ld16(tbuf + kChunk * chunk_of(0), z);
-      if (last_buf >= 0 && !eager) {   // the head this warp worked on before: hand it to the add warps
-        tc_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[last_buf]));
-      }
       float mx = -INFINITY, sub = 0.0f;
       tc_wait_ld();
       if (mix_lo < mix_hi) {
@@ -1079,21 +1068,15 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         for (int c = 0; c < p.cluster; ++c)
           st_async_f32x2(map_to_cta(slot_addr, c), mx, lsum, map_to_cta(bar_addr, c));
       }
-      last_buf = buf;
-      if (eager) {   // hand over at once: the add warps of this head gate our next heads
-        tc_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars.eready[buf]));
-        last_buf = -1;
-      }
-      if (threadIdx.x == 0) MD_TRACE(h, 4);
-    }
-    if (last_buf >= 0) {   // hand over the last head that was worked on
+      // Hand the head's exponentials to the add warps at once.  (The wait for the stores runs under
+      // the other group's loop.  Handing over only when the group gets to its next head - two heads
+      // on - saves that wait but measured the same, and with two buffers that next head needs the
+      // very buffer: its MMAs wait for the add warps, who wait for the hand-over.)
       tc_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars.eready[last_buf]));
+      if (lane == 0) mbar_arrive(smem_u32(&bars.eready[buf]));
+      if (threadIdx.x == 0) MD_TRACE(h, 4);
     }
     if constexpr (FILTER) {
       // filter tail, exp warps: selection of this request.  Dynamic shared memory is free by now:
@@ -1177,14 +1160,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
           tc_ld16(tbuf + kChunk * c0, e[0]);
           if (c0 + 1 < ACH && c0 + 1 < total_chunks) tc_ld16(tbuf + kChunk * (c0 + 1), e[1]);
           tc_wait_ld();
-          const float f0 = f, f1 = f;
-          const uint64_t f0_2 = pack2(f, f), f1_2 = f0_2;
+          const uint64_t f_2 = pack2(f, f);
 #pragma unroll
-          for (int j = 0; j < kChunk; j += 2) acc[c0][j >> 1] = fma2(pack2(e[0][j], e[0][j + 1]), f0_2, acc[c0][j >> 1]);
+          for (int j = 0; j < kChunk; j += 2) acc[c0][j >> 1] = fma2(pack2(e[0][j], e[0][j + 1]), f_2, acc[c0][j >> 1]);
           if (c0 + 1 < ACH && c0 + 1 < total_chunks) {
 #pragma unroll
             for (int j = 0; j < kChunk; j += 2)
-              acc[c0 + 1][j >> 1] = fma2(pack2(e[1][j], e[1][j + 1]), f1_2, acc[c0 + 1][j >> 1]);
+              acc[c0 + 1][j >> 1] = fma2(pack2(e[1][j], e[1][j + 1]), f_2, acc[c0 + 1][j >> 1]);
           }
           if constexpr (PH) {
             // Column maxima over this warp's text rows (the lanes): recursive halving - in each of

@@ -10,9 +10,9 @@ role, joined by the barriers
     tempty            the buffer is free again
     sfull             every CTA's (max, sum) pair of a head has arrived in a slot    (n_slot slots)
 with the phase-parity waits, the transaction counts of the asynchronous statistics stores, the
-hand-over rule (an exp group hands a head's exponentials to the add role only when it has got to
-its NEXT head - the wait for its stores then costs nothing - except where that next head needs
-the very same buffer, i.e. with two buffers, or under the tight rule: then at once), the
+hand-over (an exp group hands a head's exponentials to the add role at once; ``handover="late"``
+models the alternative - only when the group has got to its NEXT head, two heads on - which ends
+in time-outs with two buffers: that next head needs the very same buffer), the
 "tight" rule (the exp role stays within d heads of the local add role when there are only 2 d
 slots) and the bounded waits: a wait that runs out raises the CTA's abort flag, every other wait
 of that CTA then returns at once, the CTA records a time-out, tells its peers before the exit
@@ -115,8 +115,8 @@ class Cluster:
         self.g_cnt = [0] * H                       # global memory: pairs published per head
         self.g_pairs = [[None] * C for _ in range(H)]
         self.geo = dict(C=C, H=H, n_q=n_q, n_buf=n_buf, n_slot=n_slot, tight=tight)
-        # "auto": the kernel's rule; "late": always one head of the group later (what the rule prevents)
-        self.eager = (tight != 0 or n_buf <= N_GROUPS) if handover == "auto" else False
+        # "auto": what the kernel does (at once); "late": one head of the group later
+        self.eager = handover == "auto"
         self.limit, self.fault, self.jitter = limit, fault, jitter or {}
         self.ctas = [Cta(self, r, self.geo) for r in range(C)]
         self.errors = []
@@ -163,8 +163,9 @@ class Cluster:
             c.stage_head[s] = None
             if not self._skips(c.rank, "mma", h, "empty"):
                 c.empty[s].arrive()
-            if not self._skips(c.rank, "mma", h, "tfull"):
-                c.tfull[buf].arrive()
+            if self._skips(c.rank, "mma", h, "tfull"):
+                return      # MMAs complete in order: if this head's never do, no later commit arrives either
+            c.tfull[buf].arrive()
 
     def exp(self, c, grp=0):
         g = self.geo

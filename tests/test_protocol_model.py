@@ -37,9 +37,9 @@ def test_protocol_tolerates_a_slow_role(slow):
 
 @pytest.mark.parametrize("n_buf,ends", [(2, False), (3, True), (4, True)])
 def test_a_late_hand_over_needs_a_third_buffer(n_buf, ends):
-    # An exp group hands a head over when it has got to its next head, two heads on.  With two
-    # buffers that next head needs the same buffer: its MMAs wait for the add role, which waits
-    # for the hand-over - every wait runs out (the kernel hands over at once in that case).
+    # Had an exp group handed a head over only when it has got to its next head, two heads on:
+    # with two buffers that next head needs the same buffer - its MMAs wait for the add role, which
+    # waits for the hand-over - and every wait runs out.  (The kernel hands over at once.)
     cl = Cluster(C=2, H=9, n_q=2, n_buf=n_buf, limit=0.3, handover="late")
     assert cl.run(join_limit=10.0), "a role hung instead of giving up"
     assert cl.errors == []
