@@ -423,6 +423,30 @@ def run_ours(args, w):
         host_burst.append(1e3 * (time.perf_counter() - t0) / 8)
     torch.cuda.synchronize()
     host_call_ms = min(host_burst)
+    # ... and of the C-ABI call by itself: the same calls with their 17 arguments marshalled once
+    # (the Python binding fetches ten data pointers and converts every argument on every call)
+    host_c_ms = None
+    if single_call:
+        import ctypes
+        L = md.lib()
+        calls = []
+        for r in range(sets.n):
+            q, k, v, hid, ki, kc = sets.inputs[r]
+            f = sets.filters[r]
+            ptrs = [q, k, v, hid, ki, kc, f.g, f.i, None, f.kept_idx, f.kept_cnt, f.hidden_out, f.k_out, f.v_out, f.workspace]
+            calls.append([f.plan] + [ctypes.c_void_p(t.data_ptr()) if t is not None else None for t in ptrs]
+                         + [ctypes.c_void_p(stream.cuda_stream)])
+        c_burst = []
+        for _ in range(5):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for j in range(8):
+                if L.mustdrop_filter(*calls[j % sets.n]) != 0:
+                    raise RuntimeError("mustdrop_filter refused a call")
+            c_burst.append(1e3 * (time.perf_counter() - t0) / 8)
+        torch.cuda.synchronize()
+        sets.check()
+        host_c_ms = min(c_burst)
 
     # the dominant kernel alone: one call between two events, rotating over the same sets
     t_filter = isolated_call_ms(torch, stream, lambda: sets.step(stream), 50)
@@ -559,7 +583,9 @@ def run_ours(args, w):
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": launches_per_step * K,
             "host_enqueue_ms_per_step": host_call_ms,
-            "host_enqueue_note": "host time of one call, best of 5 bursts of 8 calls on an empty stream; over the timed "
+            "host_enqueue_c_abi_ms_per_step": host_c_ms,
+            "host_enqueue_note": "host time of one call through the Python binding, best of 5 bursts of 8 calls on an empty stream "
+                                 "(host_enqueue_c_abi_ms_per_step: the C-ABI call alone, arguments marshalled once); over the timed "
                                  "rounds the host waits on the stream's queue (%.4f ms per step there)" % host_enqueue_ms,
             "kernel_ms": {"score": t_parts["score"], "select": t_parts["select"], "compact": t_parts["compact"],
                           "filter_call": t_filter,
